@@ -1,0 +1,178 @@
+/*
+ * cdgrab.h -- C ABI of the B200 (sm_100a) PairBalance ordering library for CD-GraB
+ * (Coordinated Distributed Gradient Balancing, arXiv 2302.00845).
+ *
+ * The library plays the paper's order server for m logical workers simulated on one
+ * GPU.  Per epoch it keeps one running sum r in R^d; per step it receives, for every
+ * worker, the two stale gradients of the next pair of its current order, balances the m
+ * pair differences against r in worker order, and records where each pair's two items go
+ * in that worker's next-epoch permutation.  Algorithms are numbered by order of
+ * appearance in the paper: 1 reorder by balanced signs, 2 PairBalance, 3 workers,
+ * 4 parameter server, 5 probabilistic balancing, 6 balancing without normalization,
+ * 7 server-side PairBalance over a set of vectors.
+ *
+ * Conventions
+ *   - Every pointer argument says whether it is a DEVICE or a HOST pointer.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls that take a stream only enqueue work; they do not synchronise the host.
+ *   - All device work of one handle must be issued on one stream (or on streams the
+ *     caller orders itself).  One handle is used by one host thread at a time.
+ *   - Return value: CDGRAB_OK (0) or a negative CDGRAB_ERR_* code.  Argument and state
+ *     errors leave the handle unchanged.  Conditions found on the device (non-finite
+ *     reductions, an expired bounded wait) are written to a device status word and
+ *     reported by cdgrab_status().
+ *   - The library owns r, both permutation buffers, the sign/margin records and all
+ *     scratch; they are allocated once in cdgrab_create and nothing is allocated per
+ *     step.  The caller owns every buffer it passes in.
+ *   - There is no CPU fallback: without a CUDA device of compute capability 10.x the
+ *     create call fails.
+ */
+#ifndef CDGRAB_H_
+#define CDGRAB_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cdgrab_ctx cdgrab_t; /* opaque, library-owned */
+
+enum { CDGRAB_F32 = 0, CDGRAB_BF16 = 1 };
+
+enum {
+  CDGRAB_OK = 0,
+  CDGRAB_ERR_INVALID = -1,   /* bad m/n/d/dtype, NULL pointer, odd n, misaligned buffer  */
+  CDGRAB_ERR_STATE = -2,     /* step outside an epoch, more than n/2 steps, early end    */
+  CDGRAB_ERR_CUDA = -3,      /* a CUDA runtime/driver call failed                        */
+  CDGRAB_ERR_NOMEM = -4,     /* device or host allocation failed                         */
+  CDGRAB_ERR_NONFINITE = -5, /* NaN/Inf met in a reduction (device status word)          */
+  CDGRAB_ERR_TIMEOUT = -6,   /* a bounded device-side wait expired (device status word)  */
+  CDGRAB_ERR_DEVICE = -7     /* no usable sm_100 device                                  */
+};
+
+/* Which code path a handle uses (cdgrab_path / CDGRAB_FORCE_PATH). */
+enum {
+  CDGRAB_PATH_AUTO = 0,
+  CDGRAB_PATH_FUSED = 1, /* one launch per step, whole step on chip (small d)            */
+  CDGRAB_PATH_FMA = 2,   /* two passes, Gram matrix on the fp32 FMA pipe                 */
+  CDGRAB_PATH_UMMA = 3   /* two passes, Gram matrix on tcgen05 tensor cores (bf16)       */
+};
+
+/*
+ * Create an order-server state for m workers with n items each (n even; the paper takes
+ * n even without loss of generality, Appendix B.1, and gives no rule for an unpaired
+ * item, so odd n is CDGRAB_ERR_INVALID) and gradients of dimension d stored as `dtype`.
+ * The current permutation of every worker starts as the identity (the paper leaves the
+ * initial permutations open, Algorithm 4).  Uses the CUDA device current at the call.
+ * Limits: 1 <= m <= 1024, 2 <= n, 1 <= d, m*n < 2^31.
+ * On success *out receives the handle.
+ */
+int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out);
+
+/* Free the handle and everything it owns.  Synchronises the device.  NULL is allowed. */
+int cdgrab_destroy(cdgrab_t *h);
+
+/*
+ * Replace the current permutations before an epoch is opened (Algorithm 4, "send initial
+ * permutations").  perms_in: HOST or DEVICE pointer, int32 [m][n], every row a permutation
+ * of 0..n-1 (validated on the host; anything else is CDGRAB_ERR_INVALID).  Synchronous.
+ */
+int cdgrab_set_perms(cdgrab_t *h, const int32_t *perms_in);
+
+/*
+ * Open an epoch: r <- 0, pair counter <- 0, sign list emptied (Algorithm 4, first line of
+ * the epoch loop).  Asynchronous on `stream`.  CDGRAB_ERR_STATE if an epoch is open.
+ */
+int cdgrab_begin_epoch(cdgrab_t *h, void *stream);
+
+/*
+ * One balancing step: pair index k = number of steps so far in this epoch.
+ *
+ * grads_dev: DEVICE pointer, `dtype` elements, layout [2][m][d] contiguous, 16-byte
+ *   aligned.  Slab 0 row i is the stale gradient worker i produced at position 2k of its
+ *   current order (z1 of Algorithm 2), slab 1 row i the one at position 2k+1 (z2): two
+ *   consecutive gather buffers of the server (Algorithm 4).  Must stay valid and unchanged
+ *   until the work this call enqueued on `stream` has completed.
+ *
+ * Computes, for i = 0..m-1 in this order (Algorithm 7's inner loop): c_i = z1_i - z2_i;
+ * s_i = +1 if ||r + c_i||_2 < ||r - c_i||_2, i.e. <r,c_i> < 0, else -1 (Algorithm 6; a
+ * tie gives -1); r <- r + s_i c_i; and writes the front slot k and the back slot n-1-k of
+ * worker i's next permutation: the item that received +1 goes to the front, the other to
+ * the back (Algorithm 7's pointer updates, equal to Algorithm 1's list form).
+ * r is kept in fp32; reductions accumulate in fp32 partial sums combined in fp64.
+ *
+ * Asynchronous on `stream`.  CDGRAB_ERR_STATE outside an epoch or after n/2 steps.
+ */
+int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream);
+
+/*
+ * Close the epoch after exactly n/2 steps (else CDGRAB_ERR_STATE): the next permutations
+ * become the current ones (Algorithm 4, last lines of the epoch loop) and, if perms_out is
+ * not NULL, are copied there.  perms_out: HOST or DEVICE pointer, int32 [m][n];
+ * perms_out[i][j] = item worker i visits at position j in the next epoch.  The copy is
+ * enqueued on `stream` (pageable host memory makes it synchronous).
+ */
+int cdgrab_end_epoch(cdgrab_t *h, int32_t *perms_out, void *stream);
+
+/* ---- read-back helpers (no semantics of their own; the parity tests need them) ------ */
+
+/* Signs of the current/last epoch: out is HOST or DEVICE int8 [m][n/2], +1/-1, 0 where no
+ * step has been taken yet.  Enqueued on `stream`. */
+int cdgrab_get_signs(cdgrab_t *h, int8_t *out, void *stream);
+
+/* Running sum: out is HOST or DEVICE float [d].  Enqueued on `stream`. */
+int cdgrab_get_r(cdgrab_t *h, float *out, void *stream);
+
+/* Relative margins |<r,c>| / (||r|| ||c||) seen at each decision (0 when r = 0 or c = 0):
+ * out is HOST or DEVICE float [m][n/2].  ||r||^2 is tracked by the recurrence
+ * ||r + s c||^2 = ||r||^2 + 2 s <r,c> + ||c||^2.  Enqueued on `stream`. */
+int cdgrab_get_margins(cdgrab_t *h, float *out, void *stream);
+
+/* Current permutations: out is HOST or DEVICE int32 [m][n].  Enqueued on `stream`. */
+int cdgrab_get_perms(cdgrab_t *h, int32_t *out, void *stream);
+
+/* Next-epoch permutations as far as the open epoch has filled them (front slots 0..k-1 and
+ * back slots n-k..n-1 of every worker; other slots hold stale values): out is HOST or DEVICE
+ * int32 [m][n].  Enqueued on `stream`. */
+int cdgrab_get_next_perms(cdgrab_t *h, int32_t *out, void *stream);
+
+/* Synchronise the device and return the first device-side condition recorded since
+ * creation (CDGRAB_ERR_NONFINITE, CDGRAB_ERR_TIMEOUT, CDGRAB_ERR_CUDA) or CDGRAB_OK. */
+int cdgrab_status(cdgrab_t *h);
+
+/* Code path the handle uses (CDGRAB_PATH_*).  The environment variable
+ * CDGRAB_FORCE_PATH = fused | fma | umma, read at create time, overrides the automatic
+ * choice when the forced path supports the shape; otherwise create fails with
+ * CDGRAB_ERR_INVALID. */
+int cdgrab_path(const cdgrab_t *h);
+
+/* Number of kernels the library has launched through this handle so far. */
+long long cdgrab_launch_count(const cdgrab_t *h);
+
+/* Static message for a CDGRAB_* code. */
+const char *cdgrab_strerror(int code);
+
+/*
+ * Per-example logistic-regression gradients for the current step (the workers' gradient
+ * computation of Algorithm 3 for the logistic-regression task of Section 5), written in
+ * the layout cdgrab_step consumes.  For worker i and slot q in {0,1}: item
+ * j = perm_cur[i][2k+q], z = <w, X[i][j]>, g = (1/(1+exp(-z)) - y[i][j]) * X[i][j].
+ *   X: DEVICE float [m][n][d]; y: DEVICE float [m][n] with values in {0,1};
+ *   w: DEVICE float [d]; grads_out: DEVICE float [2][m][d].  Handle dtype must be F32.
+ * Asynchronous on `stream`.
+ */
+int cdgrab_logreg_grads(cdgrab_t *h, const float *X, const float *y, const float *w,
+                        float *grads_out, void *stream);
+
+/*
+ * Same step with the gradients in HOST memory (pinned memory makes the copy
+ * asynchronous): grads_host [2][m][d] is copied into staging_dev (DEVICE, at least
+ * 2*m*d elements, 16-byte aligned, caller-owned) on `stream`, then cdgrab_step runs on it.
+ */
+int cdgrab_step_host(cdgrab_t *h, const void *grads_host, void *staging_dev, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CDGRAB_H_ */

@@ -1,0 +1,182 @@
+"""ctypes binding of libcdgrab.so: same names as ``include/cdgrab.h``, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  There is no CPU fallback: if the
+shared library has not been built, or no sm_100 device is present, the calls raise.
+PyTorch tensors are used as device buffers; their ``data_ptr()`` and the current CUDA stream
+handle are what crosses the boundary.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libcdgrab.so")
+
+F32, BF16 = 0, 1
+OK = 0
+ERR_INVALID, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_NONFINITE, ERR_TIMEOUT, ERR_DEVICE = -1, -2, -3, -4, -5, -6, -7
+PATH_AUTO, PATH_FUSED, PATH_FMA, PATH_UMMA = 0, 1, 2, 3
+PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma"}
+
+# name -> (restype, argtypes); the single list of what include/cdgrab.h declares
+SIGNATURES = {
+    "cdgrab_create": (C.c_int, [C.c_int, C.c_int, C.c_longlong, C.c_int, C.POINTER(C.c_void_p)]),
+    "cdgrab_destroy": (C.c_int, [C.c_void_p]),
+    "cdgrab_set_perms": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "cdgrab_begin_epoch": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "cdgrab_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_end_epoch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_get_signs": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_get_r": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_get_margins": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_get_perms": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_get_next_perms": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_status": (C.c_int, [C.c_void_p]),
+    "cdgrab_path": (C.c_int, [C.c_void_p]),
+    "cdgrab_launch_count": (C.c_longlong, [C.c_void_p]),
+    "cdgrab_strerror": (C.c_char_p, [C.c_int]),
+    "cdgrab_logreg_grads": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_step_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+}
+
+_lib = None
+
+
+class CdgrabError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().cdgrab_strerror(code).decode() if _lib is not None else str(code)
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+def lib() -> C.CDLL:
+    """Load libcdgrab.so (built in-tree by ``paper_2302_00845_b200.build``); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2302_00845_b200.build` "
+                "(there is no CPU fallback)")
+        l = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = l
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise CdgrabError(code, where)
+
+
+def _stream_ptr(stream=None):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    """Raw pointer of a contiguous torch tensor or numpy array."""
+    if hasattr(t, "data_ptr"):
+        assert t.is_contiguous()
+        return C.c_void_p(t.data_ptr())
+    assert t.flags["C_CONTIGUOUS"]
+    return C.c_void_p(t.ctypes.data)
+
+
+class CdGrab:
+    """Order-server state for m workers x n items in R^d (see ``include/cdgrab.h``)."""
+
+    def __init__(self, m: int, n: int, d: int, dtype: str | int = "f32"):
+        code = {"f32": F32, "bf16": BF16}.get(dtype, dtype)
+        h = C.c_void_p()
+        _check(lib().cdgrab_create(m, n, d, code, C.byref(h)), "cdgrab_create")
+        self._h = h
+        self.m, self.n, self.d, self.dtype = m, n, d, code
+
+    # life cycle -------------------------------------------------------------------------
+    def destroy(self):
+        if getattr(self, "_h", None):
+            lib().cdgrab_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.destroy()
+
+    # the calls of the header ----------------------------------------------------------------
+    def set_perms(self, perms):
+        _check(lib().cdgrab_set_perms(self._h, _ptr(perms)), "cdgrab_set_perms")
+
+    def begin_epoch(self, stream=None):
+        _check(lib().cdgrab_begin_epoch(self._h, _stream_ptr(stream)), "cdgrab_begin_epoch")
+
+    def step(self, grads, stream=None):
+        """grads: CUDA tensor [2][m][d] of the handle's dtype."""
+        _check(lib().cdgrab_step(self._h, _ptr(grads), _stream_ptr(stream)), "cdgrab_step")
+
+    def step_host(self, grads_host, staging, stream=None):
+        """grads_host: pinned host tensor [2][m][d]; staging: CUDA tensor of the same size."""
+        _check(lib().cdgrab_step_host(self._h, _ptr(grads_host), _ptr(staging), _stream_ptr(stream)),
+               "cdgrab_step_host")
+
+    def end_epoch(self, perms_out=None, stream=None):
+        p = _ptr(perms_out) if perms_out is not None else None
+        _check(lib().cdgrab_end_epoch(self._h, p, _stream_ptr(stream)), "cdgrab_end_epoch")
+
+    def logreg_grads(self, X, y, w, grads_out, stream=None):
+        _check(lib().cdgrab_logreg_grads(self._h, _ptr(X), _ptr(y), _ptr(w), _ptr(grads_out),
+                                         _stream_ptr(stream)), "cdgrab_logreg_grads")
+
+    # read-back ------------------------------------------------------------------------------
+    def _fetch(self, name, shape, dtype):
+        import torch
+        out = torch.empty(shape, dtype=dtype, device="cuda")
+        _check(getattr(lib(), name)(self._h, _ptr(out), _stream_ptr()), name)
+        torch.cuda.current_stream().synchronize()
+        return out
+
+    def signs(self):
+        import torch
+        return self._fetch("cdgrab_get_signs", (self.m, self.n // 2), torch.int8)
+
+    def r(self):
+        import torch
+        return self._fetch("cdgrab_get_r", (self.d,), torch.float32)
+
+    def margins(self):
+        import torch
+        return self._fetch("cdgrab_get_margins", (self.m, self.n // 2), torch.float32)
+
+    def perms(self):
+        import torch
+        return self._fetch("cdgrab_get_perms", (self.m, self.n), torch.int32)
+
+    def next_perms(self):
+        import torch
+        return self._fetch("cdgrab_get_next_perms", (self.m, self.n), torch.int32)
+
+    def status(self) -> int:
+        return lib().cdgrab_status(self._h)
+
+    def check_status(self):
+        _check(self.status(), "cdgrab_status")
+
+    @property
+    def path(self) -> str:
+        return PATH_NAMES.get(lib().cdgrab_path(self._h), "?")
+
+    @property
+    def launch_count(self) -> int:
+        return int(lib().cdgrab_launch_count(self._h))

@@ -1,0 +1,311 @@
+// C ABI of libcdgrab.so: handle life cycle, epoch state machine, path dispatch.
+// Every step of the path runs in the kernels; this file only validates and enqueues.
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace {
+
+inline bool valid(const cdgrab_ctx *h) { return h && h->magic == CDG_MAGIC; }
+
+inline size_t elem_size(int dtype) { return dtype == CDGRAB_F32 ? 4 : 2; }
+
+__global__ void iota_perm_kernel(int32_t *p, int m, int n) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < (long long)m * n) p[idx] = (int32_t)(idx % n);
+}
+
+void free_all(cdgrab_ctx *h) {
+  cdg_umma_teardown(h);
+  cudaFree(h->r); cudaFree(h->perm_cur); cudaFree(h->perm_next); cudaFree(h->signs);
+  cudaFree(h->margins); cudaFree(h->rnorm2); cudaFree(h->status); cudaFree(h->gram);
+  cudaFree(h->partials);
+}
+
+int forced_path() {
+  const char *e = getenv("CDGRAB_FORCE_PATH");
+  if (!e || !*e || !strcmp(e, "auto")) return CDGRAB_PATH_AUTO;
+  if (!strcmp(e, "fused")) return CDGRAB_PATH_FUSED;
+  if (!strcmp(e, "fma")) return CDGRAB_PATH_FMA;
+  if (!strcmp(e, "umma")) return CDGRAB_PATH_UMMA;
+  return -1;
+}
+
+inline bool fma_columns_ok(const cdgrab_ctx *h) { return h->m <= 16 && h->d % 4 == 0; }
+
+int copy_out(void *dst, const void *src, size_t bytes, void *stream) {
+  if (!dst) return CDGRAB_ERR_INVALID;
+  if (cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  return CDGRAB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *cdgrab_strerror(int code) {
+  switch (code) {
+    case CDGRAB_OK: return "ok";
+    case CDGRAB_ERR_INVALID: return "invalid argument";
+    case CDGRAB_ERR_STATE: return "call not allowed in the current epoch state";
+    case CDGRAB_ERR_CUDA: return "CUDA call failed";
+    case CDGRAB_ERR_NOMEM: return "out of memory";
+    case CDGRAB_ERR_NONFINITE: return "non-finite value met in a reduction";
+    case CDGRAB_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case CDGRAB_ERR_DEVICE: return "no usable sm_100 CUDA device";
+    default: return "unknown error";
+  }
+}
+
+int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
+  if (!out) return CDGRAB_ERR_INVALID;
+  *out = nullptr;
+  if (m < 1 || m > 1024 || n < 2 || (n & 1) || d < 1) return CDGRAB_ERR_INVALID;
+  if ((long long)m * n >= (1ll << 31)) return CDGRAB_ERR_INVALID;
+  if (dtype != CDGRAB_F32 && dtype != CDGRAB_BF16) return CDGRAB_ERR_INVALID;
+  const int forced = forced_path();
+  if (forced < 0) return CDGRAB_ERR_INVALID;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_DEVICE; }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_DEVICE; }
+  if (prop.major != 10) return CDGRAB_ERR_DEVICE;  // the kernels are built for sm_100a only
+
+  cdgrab_ctx *h = new (std::nothrow) cdgrab_ctx();
+  if (!h) return CDGRAB_ERR_NOMEM;
+  memset(h, 0, sizeof(*h));
+  h->magic = CDG_MAGIC;
+  h->m = m; h->n = n; h->d = d; h->dtype = dtype;
+  h->device = dev; h->num_sms = prop.multiProcessorCount;
+
+  // ---- choose the path ------------------------------------------------------------
+  const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);
+  const bool fused_ok = cdg_fused_supported(m, d, dtype);
+  const bool umma_ok = cdg_umma_supported(m, d, dtype);
+  int path;
+  if (forced == CDGRAB_PATH_AUTO) {
+    if (fused_ok && step_bytes <= (size_t)768 * 1024) path = CDGRAB_PATH_FUSED;
+    else if (umma_ok && !fma_columns_ok(h)) path = CDGRAB_PATH_UMMA;
+    else path = CDGRAB_PATH_FMA;
+  } else {
+    path = forced;
+    if ((path == CDGRAB_PATH_FUSED && !fused_ok) || (path == CDGRAB_PATH_UMMA && !umma_ok)) {
+      delete h;
+      return CDGRAB_ERR_INVALID;
+    }
+  }
+  h->path = path;
+
+  // ---- allocations ----------------------------------------------------------------
+  const size_t np = (size_t)m * (size_t)(n / 2);
+  bool ok = true;
+  ok = ok && cudaMalloc(&h->r, sizeof(float) * (size_t)d) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->perm_cur, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->perm_next, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->signs, np) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->margins, sizeof(float) * np) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->rnorm2, sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->status, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->gram, sizeof(double) * ((size_t)m * m + m)) == cudaSuccess;
+  if (ok && path == CDGRAB_PATH_FMA) {
+    if (fma_columns_ok(h)) {
+      // thread-per-column kernel: one partial vector (<= 152 doubles) per block
+      long long blocks = (d / 4 + 255) / 256;
+      if (blocks > (long long)h->num_sms * 2) blocks = (long long)h->num_sms * 2;
+      h->gram_chunks = (int)blocks;
+      h->partials_bytes = sizeof(double) * 152 * (size_t)blocks;
+    } else {
+      const int ntile = (m + CDG_TM - 1) / CDG_TM;
+      const int npairs = ntile * (ntile + 1) / 2;
+      long long chunks = (d + 256ll * 512 - 1) / (256ll * 512);  // <= 512 columns per thread
+      const long long fill = (2ll * h->num_sms + npairs - 1) / npairs;
+      const long long maxc = (d + 255) / 256;
+      if (chunks < fill) chunks = fill;
+      if (chunks > maxc) chunks = maxc;
+      h->gram_chunks = (int)chunks;
+      h->partials_bytes = sizeof(double) * CDG_TILE_ENTRIES * (size_t)npairs * (size_t)chunks;
+    }
+    ok = ok && cudaMalloc(&h->partials, h->partials_bytes) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaGetLastError();
+    free_all(h);
+    delete h;
+    return CDGRAB_ERR_NOMEM;
+  }
+  if (path == CDGRAB_PATH_UMMA) {
+    const int rc = cdg_umma_setup(h);
+    if (rc != CDGRAB_OK) { free_all(h); delete h; return rc; }
+  }
+
+  const long long tot = (long long)m * n;
+  iota_perm_kernel<<<(unsigned)((tot + 255) / 256), 256>>>(h->perm_cur, m, n);
+  cudaMemset(h->perm_next, 0, sizeof(int32_t) * (size_t)m * n);
+  cudaMemset(h->signs, 0, np);
+  cudaMemset(h->margins, 0, sizeof(float) * np);
+  cudaMemset(h->rnorm2, 0, sizeof(double));
+  cudaMemset(h->status, 0, sizeof(int));
+  cudaMemset(h->r, 0, sizeof(float) * (size_t)d);
+  if (cudaDeviceSynchronize() != cudaSuccess) {
+    cudaGetLastError();
+    free_all(h);
+    delete h;
+    return CDGRAB_ERR_CUDA;
+  }
+  *out = h;
+  return CDGRAB_OK;
+}
+
+int cdgrab_destroy(cdgrab_t *h) {
+  if (!h) return CDGRAB_OK;
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  cudaDeviceSynchronize();
+  free_all(h);
+  h->magic = 0;
+  delete h;
+  return CDGRAB_OK;
+}
+
+int cdgrab_set_perms(cdgrab_t *h, const int32_t *perms_in) {
+  if (!valid(h) || !perms_in) return CDGRAB_ERR_INVALID;
+  if (h->epoch_open) return CDGRAB_ERR_STATE;
+  const size_t cnt = (size_t)h->m * h->n;
+  std::vector<int32_t> host(cnt);
+  if (cudaMemcpy(host.data(), perms_in, cnt * sizeof(int32_t), cudaMemcpyDefault) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  std::vector<char> seen(h->n);
+  for (int i = 0; i < h->m; ++i) {
+    std::fill(seen.begin(), seen.end(), 0);
+    for (int j = 0; j < h->n; ++j) {
+      const int32_t v = host[(size_t)i * h->n + j];
+      if (v < 0 || v >= h->n || seen[v]) return CDGRAB_ERR_INVALID;
+      seen[v] = 1;
+    }
+  }
+  if (cudaMemcpy(h->perm_cur, host.data(), cnt * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  return CDGRAB_OK;
+}
+
+int cdgrab_begin_epoch(cdgrab_t *h, void *stream) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  if (h->epoch_open) return CDGRAB_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(h->r, 0, sizeof(float) * (size_t)h->d, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->rnorm2, 0, sizeof(double), st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->signs, 0, (size_t)h->m * (h->n / 2), st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->margins, 0, sizeof(float) * (size_t)h->m * (h->n / 2), st);
+  if (e == cudaSuccess && h->r_split)
+    e = cudaMemsetAsync(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad, st);
+  if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->k = 0;
+  h->epoch_open = 1;
+  return CDGRAB_OK;
+}
+
+int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
+  if (!valid(h) || !grads_dev) return CDGRAB_ERR_INVALID;
+  if (((uintptr_t)grads_dev & 15) != 0) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+  if (h->path == CDGRAB_PATH_FUSED) {
+    e = cdg_launch_fused(h, grads_dev, st);
+  } else {
+    if (h->path == CDGRAB_PATH_UMMA) e = cdg_launch_gram_umma(h, grads_dev, st);
+    else if (fma_columns_ok(h)) e = cdg_launch_gram_fma(h, grads_dev, st);
+    else e = cdg_launch_gram_generic(h, grads_dev, st);
+    if (e == cudaSuccess) e = cdg_launch_scan(h, st);
+    if (e == cudaSuccess) e = cdg_launch_update(h, grads_dev, st);
+  }
+  if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->k++;
+  return CDGRAB_OK;
+}
+
+int cdgrab_step_host(cdgrab_t *h, const void *grads_host, void *staging_dev, void *stream) {
+  if (!valid(h) || !grads_host || !staging_dev) return CDGRAB_ERR_INVALID;
+  if (((uintptr_t)staging_dev & 15) != 0) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
+  const size_t bytes = 2 * (size_t)h->m * (size_t)h->d * elem_size(h->dtype);
+  if (cudaMemcpyAsync(staging_dev, grads_host, bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  return cdgrab_step(h, staging_dev, stream);
+}
+
+int cdgrab_end_epoch(cdgrab_t *h, int32_t *perms_out, void *stream) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || h->k != h->n / 2) return CDGRAB_ERR_STATE;
+  int32_t *t = h->perm_cur; h->perm_cur = h->perm_next; h->perm_next = t;
+  h->epoch_open = 0;
+  if (perms_out) return copy_out(perms_out, h->perm_cur, sizeof(int32_t) * (size_t)h->m * h->n, stream);
+  return CDGRAB_OK;
+}
+
+int cdgrab_get_signs(cdgrab_t *h, int8_t *out, void *stream) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  return copy_out(out, h->signs, (size_t)h->m * (h->n / 2), stream);
+}
+int cdgrab_get_r(cdgrab_t *h, float *out, void *stream) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  return copy_out(out, h->r, sizeof(float) * (size_t)h->d, stream);
+}
+int cdgrab_get_margins(cdgrab_t *h, float *out, void *stream) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  return copy_out(out, h->margins, sizeof(float) * (size_t)h->m * (h->n / 2), stream);
+}
+int cdgrab_get_perms(cdgrab_t *h, int32_t *out, void *stream) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  return copy_out(out, h->perm_cur, sizeof(int32_t) * (size_t)h->m * h->n, stream);
+}
+int cdgrab_get_next_perms(cdgrab_t *h, int32_t *out, void *stream) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  return copy_out(out, h->perm_next, sizeof(int32_t) * (size_t)h->m * h->n, stream);
+}
+
+int cdgrab_status(cdgrab_t *h) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  int st = 0;
+  if (cudaMemcpy(&st, h->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  if (st & CDG_ST_TIMEOUT) return CDGRAB_ERR_TIMEOUT;
+  if (st & CDG_ST_NONFINITE) return CDGRAB_ERR_NONFINITE;
+  return CDGRAB_OK;
+}
+
+int cdgrab_path(const cdgrab_t *h) { return valid(h) ? h->path : CDGRAB_ERR_INVALID; }
+
+long long cdgrab_launch_count(const cdgrab_t *h) { return valid(h) ? h->launches : -1; }
+
+int cdgrab_logreg_grads(cdgrab_t *h, const float *X, const float *y, const float *w, float *grads_out,
+                        void *stream) {
+  if (!valid(h) || !X || !y || !w || !grads_out) return CDGRAB_ERR_INVALID;
+  if (h->dtype != CDGRAB_F32) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
+  if (cdg_launch_logreg(h, X, y, w, grads_out, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  return CDGRAB_OK;
+}
+
+}  // extern "C"

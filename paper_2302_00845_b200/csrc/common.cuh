@@ -1,0 +1,83 @@
+// Internal declarations shared by the translation units of libcdgrab.so.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cdgrab.h"
+
+#define CDG_MAGIC 0xCD62AB01u
+
+// bits of the device status word
+#define CDG_ST_NONFINITE 1
+#define CDG_ST_TIMEOUT 2
+
+// register tile edge of the generic FMA Gram kernel
+#define CDG_TM 8
+#define CDG_TILE_ENTRIES (CDG_TM * CDG_TM + CDG_TM)
+
+struct cdgrab_ctx {
+  uint32_t magic;
+  int m, n;
+  long long d;
+  int dtype;
+  int device;
+  int num_sms;
+  int path;          // CDGRAB_PATH_*
+  int k;             // pairs consumed in the open epoch
+  int epoch_open;
+  long long launches;
+
+  float *r;              // [d] running sum
+  int32_t *perm_cur;     // [m][n]
+  int32_t *perm_next;    // [m][n]
+  int8_t *signs;         // [m][n/2]
+  float *margins;        // [m][n/2]
+  double *rnorm2;        // [1] tracked ||r||^2
+  int *status;           // [1] device status word
+  double *gram;          // [m*m + m] G (row-major) then b
+  double *partials;      // pass-1 partial sums
+  size_t partials_bytes;
+  int gram_chunks;       // grid.x of the FMA Gram kernels
+
+  // tcgen05 path
+  __nv_bfloat16 *r_split;  // [3][d_pad] hi/mid/lo parts of r
+  long long d_pad;
+  float *umma_partials;    // [ctas][128][ncols]
+  int umma_ctas;
+  int umma_box_rows;       // rows of the gradient TMA box (2m rounded up to 16)
+  int umma_ncols;          // MMA N = box_rows + 16
+  int umma_subs_per_stage;
+  int umma_stages;
+  size_t umma_smem;
+  CUtensorMap tm_r;        // tensor map over r_split
+  const void *tm_g_base;   // gradient buffer the cached map was encoded for
+  CUtensorMap tm_g;
+};
+
+template <typename T>
+__device__ __forceinline__ float cdg_ld(const T *p);
+template <>
+__device__ __forceinline__ float cdg_ld<float>(const float *p) { return *p; }
+template <>
+__device__ __forceinline__ float cdg_ld<__nv_bfloat16>(const __nv_bfloat16 *p) {
+  return __bfloat162float(*p);
+}
+
+// ---- launchers (each returns a cudaError_t and bumps h->launches per kernel) ----------
+cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st);
+cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_gram_fma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,
+                              float *out, cudaStream_t st);
+bool cdg_fused_supported(int m, long long d, int dtype);
+
+// tcgen05 path
+bool cdg_umma_supported(int m, long long d, int dtype);
+int cdg_umma_setup(cdgrab_ctx *h);   // allocations + tensor maps; CDGRAB_* code
+void cdg_umma_teardown(cdgrab_ctx *h);
+cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st);

@@ -1,0 +1,376 @@
+// Generic two-pass path: works for every m, d and dtype the library accepts.
+//
+//   pass 1   gram_tile_kernel      G = C^T C and b = C^T r over the step's m pair
+//                                  differences c_i = z1_i - z2_i, on the fp32 FMA pipe
+//            gram_combine_kernel   fixed-order fp64 sum of the per-block partials
+//   scan     scan_kernel           the m sequential sign decisions of Algorithm 6 in scalar
+//                                  space, signs + next-permutation slots (Algorithm 7)
+//   pass 2   update_kernel         r <- r + sum_i s_i c_i
+//
+// Inside a step r_{i-1} = r_0 + sum_{k<i} s_k c_k, hence
+//   <r_{i-1}, c_i> = b_i + sum_{k<i} s_k G_ki,
+// which is exact in real arithmetic and lets the d-sized work be done in two streaming
+// passes instead of 2m dependent sweeps.
+#include "common.cuh"
+
+// ------------------------------------------------------------------------------------
+// pass 1 (generic): register-tiled Gram on FMA units
+// grid = (chunks, tile pairs (I <= J)); each thread walks columns with a grid stride.
+// ------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+gram_tile_kernel(const T *__restrict__ g, const float *__restrict__ r, int m, long long d,
+                 int ntile, double *__restrict__ partials) {
+  int I = 0, rem = blockIdx.y;
+  while (rem >= ntile - I) { rem -= ntile - I; ++I; }
+  const int J = I + rem;
+  const bool diag = (I == J);
+
+  float acc[CDG_TM][CDG_TM];
+  float bacc[CDG_TM];
+#pragma unroll
+  for (int a = 0; a < CDG_TM; ++a) {
+    bacc[a] = 0.f;
+#pragma unroll
+    for (int b = 0; b < CDG_TM; ++b) acc[a][b] = 0.f;
+  }
+
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const size_t slab = (size_t)m * (size_t)d;
+  for (long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x; x < d; x += stride) {
+    float cI[CDG_TM], cJ[CDG_TM];
+#pragma unroll
+    for (int a = 0; a < CDG_TM; ++a) {
+      const int row = I * CDG_TM + a;
+      cI[a] = 0.f;
+      if (row < m) {
+        const size_t off = (size_t)row * (size_t)d + (size_t)x;
+        cI[a] = cdg_ld(g + off) - cdg_ld(g + slab + off);
+      }
+    }
+    if (diag) {
+      const float rx = r[x];
+#pragma unroll
+      for (int a = 0; a < CDG_TM; ++a) { cJ[a] = cI[a]; bacc[a] = fmaf(rx, cI[a], bacc[a]); }
+    } else {
+#pragma unroll
+      for (int a = 0; a < CDG_TM; ++a) {
+        const int row = J * CDG_TM + a;
+        cJ[a] = 0.f;
+        if (row < m) {
+          const size_t off = (size_t)row * (size_t)d + (size_t)x;
+          cJ[a] = cdg_ld(g + off) - cdg_ld(g + slab + off);
+        }
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < CDG_TM; ++a)
+#pragma unroll
+      for (int b = 0; b < CDG_TM; ++b) acc[a][b] = fmaf(cI[a], cJ[b], acc[a][b]);
+  }
+
+  // block reduction in fp64, fixed tree: lanes by shuffle, warps in index order
+  __shared__ double red[8][CDG_TILE_ENTRIES];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int e = 0; e < CDG_TILE_ENTRIES; ++e) {
+    double v = (e < CDG_TM * CDG_TM) ? (double)acc[e / CDG_TM][e % CDG_TM]
+                                     : (double)bacc[e - CDG_TM * CDG_TM];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+    if (lane == 0) red[warp][e] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < CDG_TILE_ENTRIES) {
+    double v = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) v += red[w][threadIdx.x];
+    partials[((size_t)blockIdx.x * gridDim.y + blockIdx.y) * CDG_TILE_ENTRIES + threadIdx.x] = v;
+  }
+}
+
+// One thread per (tile pair, entry): sum the chunk partials in chunk order, scatter into the
+// symmetric G (row-major [m][m]) and b ([m], stored after G).
+__global__ void gram_combine_kernel(const double *__restrict__ partials, int chunks, int npairs,
+                                    int ntile, int m, double *__restrict__ gram) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= npairs * CDG_TILE_ENTRIES) return;
+  const int p = idx / CDG_TILE_ENTRIES, e = idx % CDG_TILE_ENTRIES;
+  double v = 0.0;
+  for (int c = 0; c < chunks; ++c) v += partials[((size_t)c * npairs + p) * CDG_TILE_ENTRIES + e];
+  int I = 0, rem = p;
+  while (rem >= ntile - I) { rem -= ntile - I; ++I; }
+  const int J = I + rem;
+  if (e < CDG_TM * CDG_TM) {
+    const int row = I * CDG_TM + e / CDG_TM, col = J * CDG_TM + e % CDG_TM;
+    if (row < m && col < m) {
+      gram[(size_t)row * m + col] = v;
+      if (I != J) gram[(size_t)col * m + row] = v;
+    }
+  } else if (I == J) {
+    const int row = I * CDG_TM + (e - CDG_TM * CDG_TM);
+    if (row < m) gram[(size_t)m * m + row] = v;
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// scan: m sequential decisions in scalar space + permutation slots.  One warp.
+//   t_j starts as b_j; after worker i is decided every later t_j gains s_i G_ij, so when
+//   worker j's turn comes t_j = <r_{j-1}, c_j> (summed in the order k = 0..j-1).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32)
+scan_kernel(const double *__restrict__ gram, int m, int n, int k,
+            const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
+            int8_t *__restrict__ signs, float *__restrict__ margins,
+            double *__restrict__ rnorm2, int *__restrict__ status, int use_smem) {
+  extern __shared__ double sh[];
+  double *tsh = sh;            // [m]
+  double *gsh = sh + m;        // [m][m] when use_smem
+  const int lane = threadIdx.x;
+  const double *G = gram;
+  const double *b = gram + (size_t)m * m;
+  for (int j = lane; j < m; j += 32) tsh[j] = b[j];
+  if (use_smem) {
+    for (int e = lane; e < m * m; e += 32) gsh[e] = G[e];
+    G = gsh;
+  }
+  __syncwarp();
+  double rn2 = *rnorm2;
+  const int half = n >> 1;
+  bool bad = false;
+  for (int i = 0; i < m; ++i) {
+    const double ti = tsh[i];
+    const double gii = G[(size_t)i * m + i];
+    // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0; a tie gives -1
+    const int s = (ti < 0.0) ? 1 : -1;
+    bad |= !(isfinite(ti) && isfinite(gii));
+    const double sd = (double)s;
+    for (int j = i + 1 + lane; j < m; j += 32) tsh[j] += sd * G[(size_t)i * m + j];
+    if (lane == 0) {
+      const size_t pos = (size_t)i * half + k;
+      signs[pos] = (int8_t)s;
+      const double den = rn2 * gii;
+      margins[pos] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
+      // Algorithm 7: the item that received +1 goes to the front slot, the other to the back
+      const int32_t first = perm_cur[(size_t)i * n + 2 * k];
+      const int32_t second = perm_cur[(size_t)i * n + 2 * k + 1];
+      perm_next[(size_t)i * n + k] = (s == 1) ? first : second;
+      perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;
+    }
+    rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
+    if (rn2 < 0.0) rn2 = 0.0;
+    __syncwarp();
+  }
+  if (lane == 0) {
+    *rnorm2 = rn2;
+    if (bad) atomicOr(status, CDG_ST_NONFINITE);
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// pass 2: r <- r + sum_i s_i (z1_i - z2_i), i ascending.  VEC columns per thread.
+// AccT is double for fp32 inputs (one rounding of r per step), float for bf16 inputs.
+// ------------------------------------------------------------------------------------
+template <typename T, int VEC>
+struct VecLoad;
+template <>
+struct VecLoad<float, 4> {
+  static __device__ __forceinline__ void ld(const float *p, float (&v)[4]) {
+    const float4 q = __ldg(reinterpret_cast<const float4 *>(p));
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+  }
+};
+template <>
+struct VecLoad<float, 1> {
+  static __device__ __forceinline__ void ld(const float *p, float (&v)[1]) { v[0] = __ldg(p); }
+};
+template <>
+struct VecLoad<__nv_bfloat16, 8> {
+  static __device__ __forceinline__ void ld(const __nv_bfloat16 *p, float (&v)[8]) {
+    const uint4 q = __ldg(reinterpret_cast<const uint4 *>(p));
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[2 * j] = __uint_as_float(w[j] << 16);
+      v[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+  }
+};
+template <>
+struct VecLoad<__nv_bfloat16, 1> {
+  static __device__ __forceinline__ void ld(const __nv_bfloat16 *p, float (&v)[1]) {
+    v[0] = __bfloat162float(*p);
+  }
+};
+
+template <typename T, typename AccT, int VEC, bool SPLIT>
+__global__ void __launch_bounds__(256)
+update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__restrict__ signs,
+              int sign_stride, int m, long long d, __nv_bfloat16 *__restrict__ r_split,
+              long long d_pad) {
+  extern __shared__ float ssh[];  // [m] signs as +-1.0f
+  for (int i = threadIdx.x; i < m; i += blockDim.x) ssh[i] = (float)signs[(size_t)i * sign_stride];
+  __syncthreads();
+  const long long nvec = d / VEC;
+  const size_t slab = (size_t)m * (size_t)d;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+    const size_t x = (size_t)v * VEC;
+    AccT acc[VEC];
+    float rv[VEC];
+    if constexpr (VEC % 4 == 0) {
+#pragma unroll
+      for (int q = 0; q < VEC / 4; ++q) {
+        const float4 f = *reinterpret_cast<const float4 *>(r + x + 4 * q);
+        rv[4 * q] = f.x; rv[4 * q + 1] = f.y; rv[4 * q + 2] = f.z; rv[4 * q + 3] = f.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) rv[j] = r[x + j];
+    }
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) acc[j] = (AccT)rv[j];
+#pragma unroll 4
+    for (int i = 0; i < m; ++i) {
+      float a[VEC], b[VEC];
+      VecLoad<T, VEC>::ld(g + (size_t)i * (size_t)d + x, a);
+      VecLoad<T, VEC>::ld(g + slab + (size_t)i * (size_t)d + x, b);
+      const float s = ssh[i];
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) acc[j] += (AccT)(s * (a[j] - b[j]));
+    }
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) rv[j] = (float)acc[j];
+    if constexpr (VEC % 4 == 0) {
+#pragma unroll
+      for (int q = 0; q < VEC / 4; ++q)
+        *reinterpret_cast<float4 *>(r + x + 4 * q) =
+            make_float4(rv[4 * q], rv[4 * q + 1], rv[4 * q + 2], rv[4 * q + 3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) r[x + j] = rv[j];
+    }
+    if constexpr (SPLIT) {
+      // r = hi + mid + lo exactly (3 x 8 significand bits), consumed by the tensor-core pass
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(rv[j]);
+        const float r1 = rv[j] - __bfloat162float(hi);
+        const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+        const float r2 = r1 - __bfloat162float(mid);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(r2);
+        r_split[x + j] = hi;
+        r_split[(size_t)d_pad + x + j] = mid;
+        r_split[2 * (size_t)d_pad + x + j] = lo;
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// per-example logistic-regression gradient for the current pair of every worker
+// grid = (m, 2): block (i, q) handles item perm_cur[i][2k+q]
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+logreg_kernel(const float *__restrict__ X, const float *__restrict__ y, const float *__restrict__ w,
+              const int32_t *__restrict__ perm_cur, int m, int n, long long d, int k,
+              float *__restrict__ out) {
+  const int i = blockIdx.x, q = blockIdx.y;
+  const int item = perm_cur[(size_t)i * n + 2 * k + q];
+  const float *x = X + ((size_t)i * n + item) * (size_t)d;
+  float part = 0.f;
+  for (long long c = threadIdx.x; c < d; c += blockDim.x) part = fmaf(w[c], x[c], part);
+  __shared__ double red[8];
+  __shared__ float coef;
+  double v = (double)part;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double z = 0.0;
+    for (int wi = 0; wi < 8; ++wi) z += red[wi];
+    const float sig = 1.f / (1.f + expf(-(float)z));
+    coef = sig - y[(size_t)i * n + item];
+  }
+  __syncthreads();
+  const float cf = coef;
+  float *o = out + ((size_t)q * m + i) * (size_t)d;
+  for (long long c = threadIdx.x; c < d; c += blockDim.x) o[c] = cf * x[c];
+}
+
+// ------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------
+cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  const int ntile = (h->m + CDG_TM - 1) / CDG_TM;
+  const int npairs = ntile * (ntile + 1) / 2;
+  dim3 grid(h->gram_chunks, npairs);
+  if (h->dtype == CDGRAB_F32)
+    gram_tile_kernel<float><<<grid, 256, 0, st>>>((const float *)grads, h->r, h->m, h->d, ntile,
+                                                  h->partials);
+  else
+    gram_tile_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)grads, h->r, h->m,
+                                                          h->d, ntile, h->partials);
+  h->launches++;
+  const int total = npairs * CDG_TILE_ENTRIES;
+  gram_combine_kernel<<<(total + 127) / 128, 128, 0, st>>>(h->partials, h->gram_chunks, npairs,
+                                                           ntile, h->m, h->gram);
+  h->launches++;
+  return cudaGetLastError();
+}
+
+cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
+  const int m = h->m;
+  const size_t with_g = ((size_t)m * m + m) * sizeof(double);
+  const int use_smem = with_g <= 160 * 1024;
+  const size_t smem = use_smem ? with_g : (size_t)m * sizeof(double);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         160 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  scan_kernel<<<1, 32, smem, st>>>(h->gram, m, h->n, h->k, h->perm_cur, h->perm_next, h->signs,
+                                   h->margins, h->rnorm2, h->status, use_smem);
+  h->launches++;
+  return cudaGetLastError();
+}
+
+template <typename T, typename AccT, int VEC>
+static void launch_update_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  const long long nvec = h->d / VEC;
+  long long blocks = (nvec + 255) / 256;
+  const long long cap = (long long)h->num_sms * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  const size_t smem = (size_t)h->m * sizeof(float);
+  const int8_t *sg = h->signs + h->k;
+  if (h->r_split)
+    update_kernel<T, AccT, VEC, true><<<(unsigned)blocks, 256, smem, st>>>(
+        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad);
+  else
+    update_kernel<T, AccT, VEC, false><<<(unsigned)blocks, 256, smem, st>>>(
+        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0);
+  h->launches++;
+}
+
+cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  if (h->dtype == CDGRAB_F32) {
+    if (h->d % 4 == 0) launch_update_t<float, double, 4>(h, grads, st);
+    else launch_update_t<float, double, 1>(h, grads, st);
+  } else {
+    if (h->d % 8 == 0) launch_update_t<__nv_bfloat16, float, 8>(h, grads, st);
+    else launch_update_t<__nv_bfloat16, float, 1>(h, grads, st);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,
+                              float *out, cudaStream_t st) {
+  dim3 grid(h->m, 2);
+  logreg_kernel<<<grid, 256, 0, st>>>(X, y, w, h->perm_cur, h->m, h->n, h->d, h->k, out);
+  h->launches++;
+  return cudaGetLastError();
+}
