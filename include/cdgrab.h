@@ -150,6 +150,26 @@ int cdgrab_path(const cdgrab_t *h);
 /* Number of kernels the library has launched through this handle so far. */
 long long cdgrab_launch_count(const cdgrab_t *h);
 
+/* Kernel kinds for the timing hook below. */
+enum {
+  CDGRAB_K_GRAM = 0,    /* pass 1: Gram matrix G = C^T C and b = C^T r                    */
+  CDGRAB_K_COMBINE = 1, /* fixed-order fp64 sum of pass-1 partials                        */
+  CDGRAB_K_SCAN = 2,    /* the m sign decisions + permutation slots                       */
+  CDGRAB_K_UPDATE = 3,  /* pass 2: r <- r + sum_i s_i c_i                                 */
+  CDGRAB_K_FUSED = 4,   /* whole step in one launch                                       */
+  CDGRAB_K_LOGREG = 5,  /* per-example logistic-regression gradients                      */
+  CDGRAB_K_COUNT = 6
+};
+
+/* Timing hook: while on, every kernel the handle launches is bracketed by a pair of CUDA
+ * events recorded on the launching stream (at most 8192 launches are kept; later ones are
+ * not recorded).  Turning it on clears earlier records.  Costs two event records per launch. */
+int cdgrab_profile_enable(cdgrab_t *h, int on);
+
+/* Synchronise the device and report, for kernel kind `kind`, the summed event-to-event
+ * duration in milliseconds and the number of recorded launches.  HOST pointers. */
+int cdgrab_profile_read(cdgrab_t *h, int kind, double *total_ms, long long *launches);
+
 /* Static message for a CDGRAB_* code. */
 const char *cdgrab_strerror(int code);
 

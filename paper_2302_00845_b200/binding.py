@@ -17,6 +17,7 @@ F32, BF16 = 0, 1
 OK = 0
 ERR_INVALID, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_NONFINITE, ERR_TIMEOUT, ERR_DEVICE = -1, -2, -3, -4, -5, -6, -7
 PATH_AUTO, PATH_FUSED, PATH_FMA, PATH_UMMA = 0, 1, 2, 3
+KERNEL_KINDS = ("gram", "combine", "scan", "update", "fused", "logreg")
 PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma"}
 
 # name -> (restype, argtypes); the single list of what include/cdgrab.h declares
@@ -36,6 +37,8 @@ SIGNATURES = {
     "cdgrab_path": (C.c_int, [C.c_void_p]),
     "cdgrab_launch_count": (C.c_longlong, [C.c_void_p]),
     "cdgrab_strerror": (C.c_char_p, [C.c_int]),
+    "cdgrab_profile_enable": (C.c_int, [C.c_void_p, C.c_int]),
+    "cdgrab_profile_read": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]),
     "cdgrab_logreg_grads": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_step_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
 }
@@ -172,6 +175,19 @@ class CdGrab:
 
     def check_status(self):
         _check(self.status(), "cdgrab_status")
+
+    def profile_enable(self, on: bool = True):
+        _check(lib().cdgrab_profile_enable(self._h, int(on)), "cdgrab_profile_enable")
+
+    def profile_read(self) -> dict:
+        """{kernel kind: (total ms, launches)} for the launches recorded since profiling was enabled."""
+        out = {}
+        for kind, name in enumerate(KERNEL_KINDS):
+            ms, cnt = C.c_double(), C.c_longlong()
+            _check(lib().cdgrab_profile_read(self._h, kind, C.byref(ms), C.byref(cnt)), "cdgrab_profile_read")
+            if cnt.value:
+                out[name] = (ms.value, cnt.value)
+        return out
 
     @property
     def path(self) -> str:

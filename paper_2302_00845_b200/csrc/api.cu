@@ -26,6 +26,12 @@ void free_all(cdgrab_ctx *h) {
   cudaFree(h->r); cudaFree(h->perm_cur); cudaFree(h->perm_next); cudaFree(h->signs);
   cudaFree(h->margins); cudaFree(h->rnorm2); cudaFree(h->status); cudaFree(h->gram);
   cudaFree(h->partials);
+  if (h->prof_ev) {
+    for (int i = 0; i < 2 * h->prof_cap; ++i) if (h->prof_ev[i]) cudaEventDestroy(h->prof_ev[i]);
+    free(h->prof_ev);
+    free(h->prof_kind);
+    h->prof_ev = nullptr; h->prof_kind = nullptr;
+  }
 }
 
 int forced_path() {
@@ -289,6 +295,42 @@ int cdgrab_status(cdgrab_t *h) {
   }
   if (st & CDG_ST_TIMEOUT) return CDGRAB_ERR_TIMEOUT;
   if (st & CDG_ST_NONFINITE) return CDGRAB_ERR_NONFINITE;
+  return CDGRAB_OK;
+}
+
+int cdgrab_profile_enable(cdgrab_t *h, int on) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  if (on && !h->prof_ev) {
+    const int cap = 8192;
+    h->prof_ev = (cudaEvent_t *)calloc(2 * (size_t)cap, sizeof(cudaEvent_t));
+    h->prof_kind = (int *)calloc(cap, sizeof(int));
+    if (!h->prof_ev || !h->prof_kind) return CDGRAB_ERR_NOMEM;
+    h->prof_cap = cap;
+    for (int i = 0; i < 2 * cap; ++i)
+      if (cudaEventCreate(&h->prof_ev[i]) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  }
+  if (on) h->prof_n = 0;
+  h->prof_on = on ? 1 : 0;
+  return CDGRAB_OK;
+}
+
+int cdgrab_profile_read(cdgrab_t *h, int kind, double *total_ms, long long *launches) {
+  if (!valid(h) || !total_ms || !launches || kind < 0 || kind >= CDGRAB_K_COUNT) return CDGRAB_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  double tot = 0.0;
+  long long cnt = 0;
+  for (int i = 0; i < h->prof_n; ++i) {
+    if (h->prof_kind[i] != kind) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, h->prof_ev[2 * i], h->prof_ev[2 * i + 1]) != cudaSuccess) {
+      cudaGetLastError();
+      return CDGRAB_ERR_CUDA;
+    }
+    tot += ms;
+    ++cnt;
+  }
+  *total_ms = tot;
+  *launches = cnt;
   return CDGRAB_OK;
 }
 

@@ -42,6 +42,12 @@ struct cdgrab_ctx {
   size_t partials_bytes;
   int gram_chunks;       // grid.x of the FMA Gram kernels
 
+  // optional per-kernel timing (cdgrab_profile_*): event pairs recorded around launches
+  int prof_on;
+  int prof_n, prof_cap;
+  cudaEvent_t *prof_ev;    // [2 * prof_cap]
+  int *prof_kind;          // [prof_cap]
+
   // tcgen05 path
   __nv_bfloat16 *r_split;  // [3][d_pad] hi/mid/lo parts of r
   long long d_pad;
@@ -66,7 +72,21 @@ __device__ __forceinline__ float cdg_ld<__nv_bfloat16>(const __nv_bfloat16 *p) {
   return __bfloat162float(*p);
 }
 
-// ---- launchers (each returns a cudaError_t and bumps h->launches per kernel) ----------
+// Event pair around one launch when profiling is on; a full pool stops recording.
+struct CdgProfScope {
+  cdgrab_ctx *h; cudaStream_t st; int slot;
+  CdgProfScope(cdgrab_ctx *h_, int kind, cudaStream_t st_) : h(h_), st(st_), slot(-1) {
+    h->launches++;
+    if (h->prof_on && h->prof_n < h->prof_cap) {
+      slot = h->prof_n++;
+      h->prof_kind[slot] = kind;
+      cudaEventRecord(h->prof_ev[2 * slot], st);
+    }
+  }
+  ~CdgProfScope() { if (slot >= 0) cudaEventRecord(h->prof_ev[2 * slot + 1], st); }
+};
+
+// ---- launchers (each returns a cudaError_t; every kernel launch sits in a CdgProfScope) ----------
 cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st);
 cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st);

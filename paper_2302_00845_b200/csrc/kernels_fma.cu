@@ -261,10 +261,12 @@ static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, cudaStream_t
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  fused_step_kernel<T, M><<<1, FusedCfg<M>::THREADS, smem, st>>>(
-      (const T *)grads, h->r, h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs,
-      h->margins, h->rnorm2, h->status);
-  h->launches++;
+  {
+    CdgProfScope ps(h, CDGRAB_K_FUSED, st);
+    fused_step_kernel<T, M><<<1, FusedCfg<M>::THREADS, smem, st>>>(
+        (const T *)grads, h->r, h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs,
+        h->margins, h->rnorm2, h->status);
+  }
   return cudaGetLastError();
 }
 
@@ -282,10 +284,14 @@ cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, cudaStream_t st) 
 
 template <typename T, int M>
 static cudaError_t launch_gram_fma_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
-  gram_fma_kernel<T, M><<<h->gram_chunks, 256, 0, st>>>((const T *)grads, h->r, h->m, h->d, h->partials);
-  h->launches++;
-  fma_combine_kernel<M><<<1, 192, 0, st>>>(h->partials, h->gram_chunks, h->m, h->gram);
-  h->launches++;
+  {
+    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
+    gram_fma_kernel<T, M><<<h->gram_chunks, 256, 0, st>>>((const T *)grads, h->r, h->m, h->d, h->partials);
+  }
+  {
+    CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
+    fma_combine_kernel<M><<<1, 192, 0, st>>>(h->partials, h->gram_chunks, h->m, h->gram);
+  }
   return cudaGetLastError();
 }
 

@@ -306,17 +306,21 @@ cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream
   const int ntile = (h->m + CDG_TM - 1) / CDG_TM;
   const int npairs = ntile * (ntile + 1) / 2;
   dim3 grid(h->gram_chunks, npairs);
-  if (h->dtype == CDGRAB_F32)
-    gram_tile_kernel<float><<<grid, 256, 0, st>>>((const float *)grads, h->r, h->m, h->d, ntile,
-                                                  h->partials);
-  else
-    gram_tile_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)grads, h->r, h->m,
-                                                          h->d, ntile, h->partials);
-  h->launches++;
+  {
+    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
+    if (h->dtype == CDGRAB_F32)
+      gram_tile_kernel<float><<<grid, 256, 0, st>>>((const float *)grads, h->r, h->m, h->d, ntile,
+                                                    h->partials);
+    else
+      gram_tile_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)grads, h->r,
+                                                            h->m, h->d, ntile, h->partials);
+  }
   const int total = npairs * CDG_TILE_ENTRIES;
-  gram_combine_kernel<<<(total + 127) / 128, 128, 0, st>>>(h->partials, h->gram_chunks, npairs,
-                                                           ntile, h->m, h->gram);
-  h->launches++;
+  {
+    CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
+    gram_combine_kernel<<<(total + 127) / 128, 128, 0, st>>>(h->partials, h->gram_chunks, npairs,
+                                                             ntile, h->m, h->gram);
+  }
   return cudaGetLastError();
 }
 
@@ -332,9 +336,11 @@ cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  scan_kernel<<<1, 32, smem, st>>>(h->gram, m, h->n, h->k, h->perm_cur, h->perm_next, h->signs,
-                                   h->margins, h->rnorm2, h->status, use_smem);
-  h->launches++;
+  {
+    CdgProfScope ps(h, CDGRAB_K_SCAN, st);
+    scan_kernel<<<1, 32, smem, st>>>(h->gram, m, h->n, h->k, h->perm_cur, h->perm_next, h->signs,
+                                     h->margins, h->rnorm2, h->status, use_smem);
+  }
   return cudaGetLastError();
 }
 
@@ -347,13 +353,13 @@ static void launch_update_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
   if (blocks < 1) blocks = 1;
   const size_t smem = (size_t)h->m * sizeof(float);
   const int8_t *sg = h->signs + h->k;
+  CdgProfScope ps(h, CDGRAB_K_UPDATE, st);
   if (h->r_split)
     update_kernel<T, AccT, VEC, true><<<(unsigned)blocks, 256, smem, st>>>(
         (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad);
   else
     update_kernel<T, AccT, VEC, false><<<(unsigned)blocks, 256, smem, st>>>(
         (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0);
-  h->launches++;
 }
 
 cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
@@ -370,7 +376,9 @@ cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st)
 cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,
                               float *out, cudaStream_t st) {
   dim3 grid(h->m, 2);
-  logreg_kernel<<<grid, 256, 0, st>>>(X, y, w, h->perm_cur, h->m, h->n, h->d, h->k, out);
-  h->launches++;
+  {
+    CdgProfScope ps(h, CDGRAB_K_LOGREG, st);
+    logreg_kernel<<<grid, 256, 0, st>>>(X, y, w, h->perm_cur, h->m, h->n, h->d, h->k, out);
+  }
   return cudaGetLastError();
 }
