@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the PairBalance ordering path.
+
+A step is one balancing step of the whole path (difference forming, balancing core, running-sum
+update, permutation slots) over one batch of synthetic stale gradients [2][m][d].  The default
+workload is the GPT-2-small-sized one (m=64, n=128, d=124,000,000, bf16).
+
+  python bench.py --gpus N --steps K --warmup W          native CUDA path (C ABI)
+  python bench.py --impl reference ...                   the CPU oracle on a bounded sample
+
+Prints ONE JSON line on rank 0.  With N > 1 (torchrun) every rank runs an independent replica
+on its own GPU: the path does not shard (one shared running sum, sequential decisions).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2302_00845_b200 import synth  # noqa: E402
+
+METRIC = "balanced_examples_per_sec"
+UNIT = "examples/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum),
+# keyed by kernel kind and workload; valid only while the kernel source hash matches.
+NCU_TRAFFIC: dict = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="gpt2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-events", action="store_true",
+                    help="do not record per-kernel events inside the timed region")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.lines = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200",
+                 "-i", str(index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.3] or [l for (_, l) in self.lines]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(kind: str, wl: synth.Workload) -> float:
+    """Bytes one launch of a kernel kind must move: inputs once per pass; r read in pass 1,
+    read and written in pass 2 (or once each in the fused step)."""
+    inp = 2.0 * wl.m * wl.d * wl.elem_bytes
+    if kind == "gram":
+        return inp + 4.0 * wl.d
+    if kind in ("update", "fused"):
+        return inp + 8.0 * wl.d
+    return 0.0
+
+
+def source_hash() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2302_00845_b200", "csrc")
+    for f in sorted(os.listdir(csrc)):
+        h.update(open(os.path.join(csrc, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_sample(wl, grads_dev, seconds: float):
+    """The CPU oracle, as it stands, on the first workers of one step (r carried over)."""
+    import oracle
+    t_budget = seconds
+    rows = []
+    o = None
+    done, t_used = 0, 0.0
+    S = 1
+    # size the sample: one position first, then as many as fit the budget (at most m)
+    probe = oracle.PairBalanceOracle(1, 2, wl.d)
+    probe.begin_epoch()
+    gp, gc = synth.to_host(grads_dev[0, 0]), synth.to_host(grads_dev[1, 0])
+    t0 = time.perf_counter()
+    probe.balance_one(0, gp, gc)
+    t_pos = time.perf_counter() - t0
+    probe.close()
+    S = int(max(1, min(wl.m, t_budget / max(t_pos, 1e-6))))
+    o = oracle.PairBalanceOracle(S, 2, wl.d)
+    o.begin_epoch()
+    host = [(synth.to_host(grads_dev[0, i]), synth.to_host(grads_dev[1, i])) for i in range(S)]
+    t0 = time.perf_counter()
+    for i in range(S):
+        o.balance_one(i, host[i][0], host[i][1])
+    t_used = time.perf_counter() - t0
+    o.close()
+    return {"value": 2.0 * S / t_used, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"first {S} of {wl.m} workers of one step at full d={wl.d} "
+                      f"({2 * S} examples, {t_used:.2f} s)"}
+
+
+def run_reference(args):
+    """The oracle timed on the host cores: each step is a bounded sample of a balancing step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    wl = synth.WORKLOADS[args.workload]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    # sample: S workers per step, sized from one probe so the whole run ends within minutes
+    S_cap = min(wl.m, 4)
+    sub = wl.scaled(m=S_cap)
+    gs = synth.GradientStream(sub, device=dev)
+    g = gs.step(0)
+    host = [(synth.to_host(g[0, i]), synth.to_host(g[1, i])) for i in range(S_cap)]
+    probe = oracle.PairBalanceOracle(1, 2, wl.d)
+    probe.begin_epoch()
+    t0 = time.perf_counter()
+    probe.balance_one(0, host[0][0], host[0][1])
+    t_pos = time.perf_counter() - t0
+    probe.close()
+    total_steps = args.steps + args.warmup
+    S = int(max(1, min(S_cap, 120.0 / max(t_pos * total_steps, 1e-9))))
+    n_o = 2 * total_steps
+    o = oracle.PairBalanceOracle(S, n_o, wl.d)
+    o.begin_epoch()
+    for _ in range(args.warmup):
+        for i in range(S):
+            o.balance_one(i, host[i][0], host[i][1])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        for i in range(S):
+            o.balance_one(i, host[i][0], host[i][1])
+    dt = time.perf_counter() - t0
+    o.close()
+    value = 2.0 * S * args.steps / dt
+    sample = (f"each step balances the first {S} of {wl.m} workers' pairs at full d={wl.d} "
+              f"({wl.dtype}); same rows every step, running sum carried")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": wl.name, "m": wl.m, "n": wl.n, "d": wl.d,
+                                        "storage": wl.dtype, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+def run_native(args):
+    from paper_2302_00845_b200 import binding, build
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    wl = synth.WORKLOADS[args.workload]
+    if wl.kind == "logreg":
+        raise SystemExit("bench.py: the logistic-regression workload is covered by the parity tests")
+    m, n, d = wl.m, wl.n, wl.d
+    step_bytes = 2 * m * d * wl.elem_bytes
+    total_mem = torch.cuda.get_device_properties(local).total_memory
+    nbuf = 2 if 2 * step_bytes < 0.5 * total_mem else 1
+    flush_mode = "inputs_larger_than_l2" if step_bytes >= 4 * L2_BYTES else "l2_flush_between_steps"
+
+    gs = synth.GradientStream(wl, device="cuda")
+    bufs = [gs.step(k) for k in range(nbuf)]
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if flush_mode != "inputs_larger_than_l2" else None
+    h = binding.CdGrab(m, n, d, wl.dtype)
+    stream = torch.cuda.current_stream()
+
+    state = {"step": 0}
+
+    def one_step():
+        if state["step"] % (n // 2) == 0:
+            if state["step"]:
+                h.end_epoch()
+            h.begin_epoch()
+        h.step(bufs[state["step"] % nbuf])
+        state["step"] += 1
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        one_step()
+    barrier()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = h.launch_count
+    if not args.no_kernel_events:
+        h.profile_enable(True)
+    t_wall0 = time.time()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            one_step()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+    else:
+        evs = []
+        barrier()
+        for _ in range(args.steps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            one_step()
+            b.record(stream)
+            evs.append((a, b))
+        barrier()
+        ms = sum(a.elapsed_time(b) for a, b in evs)
+    t_wall1 = time.time()
+    launches = h.launch_count - launches0
+    prof = h.profile_read() if not args.no_kernel_events else {}
+    h.profile_enable(False)
+    h.check_status()
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+
+    if world > 1:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    examples = 2 * m * args.steps * world
+    value = examples / (ms * 1e-3)
+
+    # ---- roofline of the dominant kernel ---------------------------------------------------
+    peak, peak_kind = peaks()
+    roof = None
+    if prof:
+        dom = max(prof, key=lambda kname: prof[kname][0])
+        tot_ms, cnt = prof[dom]
+        avg_ms = tot_ms / cnt
+        ab = algorithmic_bytes(dom, wl)
+        achieved = ab / (avg_ms * 1e-3) / 1e9
+        tr = NCU_TRAFFIC.get((dom, wl.name))
+        traffic = tr["bytes"] if tr and tr.get("source") == source_hash() else None
+        roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
+                "avg_launch_ms": avg_ms, "algorithmic_bytes_per_launch": ab,
+                "kernels": {kname: {"ms_total": v[0], "launches": v[1],
+                                    "share": v[0] / sum(x[0] for x in prof.values())}
+                            for kname, v in prof.items()}}
+    step_model_b2 = 2.0 * step_bytes + 12.0 * d
+    step_model_b1 = 1.0 * step_bytes + 8.0 * d
+    model = step_model_b1 if h.path == "fused" else step_model_b2
+    step_gbs = model / (ms / args.steps * 1e-3) / 1e9 * (1 if world == 1 else 1)
+
+    # ---- end to end through the host-buffer call ----------------------------------------------
+    e2e = None
+    if not args.no_e2e and world == 1:
+        e2e = run_e2e(h, wl, bufs[0], state, one_step)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        torch.cuda.synchronize()
+        cpu = oracle_sample(wl, bufs[0], args.cpu_seconds)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "m": m, "n": n, "d": d, "storage": wl.dtype,
+                       "path": h.path, "step_input_bytes": step_bytes, "input_buffers": nbuf,
+                       "cache": flush_mode, "parallelism": "replicas" if world > 1 else "single",
+                       "step_model_bytes": model, "step_model_gbs": step_gbs,
+                       "step_model_frac_of_peak": step_gbs / peak},
+            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    h.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(h, wl, dev_buf, state, one_step):
+    """Same metric through cdgrab_step_host: every step copies its [2][m][d] input from pinned host
+    memory and reads the sign table back."""
+    import psutil
+    from paper_2302_00845_b200 import binding  # noqa: F401
+    step_bytes = 2 * wl.m * wl.d * wl.elem_bytes
+    if psutil.virtual_memory().available < 2.5 * step_bytes:
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": step_bytes, "d2h_bytes_per_step": 0,
+                "note": "not enough host memory for a pinned copy of one step"}
+    host = torch.empty(dev_buf.shape, dtype=dev_buf.dtype, pin_memory=True)
+    host.copy_(dev_buf)
+    staging = torch.empty_like(dev_buf)
+    signs_host = torch.empty(wl.m, wl.n // 2, dtype=torch.int8, pin_memory=True)
+    stream = torch.cuda.current_stream()
+    lib = binding.lib()
+    steps = 3 if step_bytes > (1 << 30) else 10
+
+    def e2e_step():
+        if state["step"] % (wl.n // 2) == 0:
+            if state["step"]:
+                h.end_epoch()
+            h.begin_epoch()
+        h.step_host(host, staging)
+        state["step"] += 1
+        rc = lib.cdgrab_get_signs(h._h, signs_host.data_ptr(), stream.cuda_stream)
+        assert rc == 0
+        stream.synchronize()  # the caller reads the step's result
+
+    e2e_step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    return {"value": 2.0 * wl.m * steps / dt, "unit": UNIT, "h2d_bytes_per_step": step_bytes,
+            "d2h_bytes_per_step": wl.m * (wl.n // 2), "steps": steps, "ms_per_step": 1e3 * dt / steps}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()
