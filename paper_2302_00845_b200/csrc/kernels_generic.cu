@@ -290,8 +290,10 @@ logreg_kernel(const float *__restrict__ X, const float *__restrict__ y, const fl
   if (threadIdx.x == 0) {
     double z = 0.0;
     for (int wi = 0; wi < 8; ++wi) z += red[wi];
-    const float sig = 1.f / (1.f + expf(-(float)z));
-    coef = sig - y[(size_t)i * n + item];
+    // sigma(z) - y without cancellation for y in {0,1}: sigma(z) - 1 = -sigma(-z)
+    const float zf = (float)z;
+    const float yv = y[(size_t)i * n + item];
+    coef = (yv > 0.5f) ? -1.f / (1.f + expf(zf)) : 1.f / (1.f + expf(-zf));
   }
   __syncthreads();
   const float cf = coef;
