@@ -1,7 +1,364 @@
-// tcgen05 Gram path (placeholder until the tensor-core kernel lands).
+// Pass 1 on the 5th-generation tensor cores (tcgen05) for bf16 gradients, m <= 64.
+//
+// The 2m gradient rows of a step ([2][m][d], K-major exactly as they lie in HBM) are the
+// operand A of  H = A A^T  (2m x 2m); every bf16 x bf16 product is exact in the fp32
+// accumulator, so no difference has to be rounded to bf16.  The Gram matrix of the pair
+// differences c_i = z1_i - z2_i follows afterwards in fp64:
+//     G_ki = H[k][i] - H[k][m+i] - H[m+k][i] + H[m+k][m+i].
+// The running sum r (fp32) is kept as three bf16 rows hi + mid + lo = r exactly (3 x 8
+// significand bits), written by pass 2; they are appended to operand B, so
+//     b_i = <r, c_i> = sum_j (H[i][R+j] - H[m+i][R+j])
+// falls out of the same MMA.
+//
+// One persistent CTA per SM owns a contiguous K range (split-K).  Per 64-column block the TMA
+// engine lands a [box_rows x 64] gradient box and a [16 x 64] box of the r rows (rows past
+// the tensor are zero-filled) back to back in 128-byte-swizzled shared memory; the same bytes
+// serve as operand A (rows 0..127 from the block base) and operand B (the first N =
+// box_rows + 16 rows).  Roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner,
+// warps 2..5 read the accumulator back (tcgen05.ld) and write the CTA's partial H.
+// Every wait is bounded: on expiry the CTA raises the time-out bit of the status word,
+// drains the copies it has in flight, frees its TMEM and returns.
+#include <cudaTypedefs.h>
+
 #include "common.cuh"
 
-bool cdg_umma_supported(int, long long, int) { return false; }
-int cdg_umma_setup(cdgrab_ctx *) { return CDGRAB_ERR_INVALID; }
-void cdg_umma_teardown(cdgrab_ctx *) {}
-cudaError_t cdg_launch_gram_umma(cdgrab_ctx *, const void *, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr int kSubCols = 64;             // bf16 columns per TMA box = one 128-byte swizzle row
+constexpr int kRBoxRows = 16;
+constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
+
+struct UmmaParams {
+  int box_rows;        // rows of the gradient box (2m rounded up to 16)
+  int ncols;           // MMA N = box_rows + 16
+  int rows_used;       // 2m
+  int subs_per_stage;
+  int stages;
+  uint32_t sub_bytes;  // ncols * 128
+  long long total_sub; // ceil(d / 64)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// bounded wait; false when the deadline passed
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long deadline) {
+  while (true) {
+    uint32_t done;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    if (clock64() > deadline) return false;
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// K-major, 128-byte swizzle: rows 128 B apart, 8-row groups 1024 B apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address
+  d |= (uint64_t)1 << 16;                          // leading byte offset (unused for this layout)
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                          // descriptor version
+  d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+  return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
+                 const UmmaParams p, float *__restrict__ partials, int *__restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[kMaxStages];
+  __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
+  __shared__ __align__(8) uint64_t bar_accum;
+  __shared__ uint32_t tmem_base_sh;
+  __shared__ int abort_sh;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-B alignment
+  const uint32_t stage_bytes = p.sub_bytes * p.subs_per_stage;
+
+  // this CTA's K range, in 64-column blocks
+  const long long sub_lo = p.total_sub * (long long)blockIdx.x / gridDim.x;
+  const long long sub_hi = p.total_sub * (long long)(blockIdx.x + 1) / gridDim.x;
+  const long long nsub = sub_hi - sub_lo;
+  const int n_iter = (int)((nsub + p.subs_per_stage - 1) / p.subs_per_stage);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&bar_accum), 1);
+    abort_sh = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_sh)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = tmem_base_sh;
+  const long long deadline = clock64() + kWaitCycles;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int s = it % p.stages;
+        if (it >= p.stages) ok = mbar_wait(smem_u32(&bar_empty[s]), ((it / p.stages) - 1) & 1, deadline);
+        if (!ok) break;
+        const long long first = sub_lo + (long long)it * p.subs_per_stage;
+        const int cnt = (int)min((long long)p.subs_per_stage, sub_hi - first);
+        const uint32_t full = smem_u32(&bar_full[s]);
+        mbar_expect_tx(full, cnt * p.sub_bytes);
+        for (int q = 0; q < cnt; ++q) {
+          const uint32_t dst = tiles + s * stage_bytes + q * p.sub_bytes;
+          const int col = (int)((first + q) * kSubCols);  // 64 bf16 = 128 bytes: 16-byte aligned
+          tma_load_2d(dst, &tm_g, col, 0, full);
+          tma_load_2d(dst + (uint32_t)p.box_rows * 128u, &tm_r, col, 0, full);
+        }
+        issued = it + 1;
+      }
+      if (!ok) {
+        atomicOr(status, CDG_ST_TIMEOUT);
+        atomicExch(&abort_sh, 1);
+        // let the copies already issued land before the CTA gives up its shared memory
+        for (int it = max(0, issued - p.stages); it < issued; ++it)
+          mbar_wait(smem_u32(&bar_full[it % p.stages]), (it / p.stages) & 1, clock64() + kWaitCycles);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = ncols
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.ncols >> 3) << 17) |
+                             ((128u >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int s = it % p.stages;
+        ok = mbar_wait(smem_u32(&bar_full[s]), (it / p.stages) & 1, deadline);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const long long first = sub_lo + (long long)it * p.subs_per_stage;
+        const int cnt = (int)min((long long)p.subs_per_stage, sub_hi - first);
+        for (int q = 0; q < cnt; ++q) {
+          const uint64_t desc = umma_desc(tiles + s * stage_bytes + q * p.sub_bytes);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4) {
+            // 16 bf16 = 32 bytes further along K inside the swizzle row
+            const uint64_t dk = desc + (uint64_t)(k4 * 2);
+            umma_bf16(tmem_acc, dk, dk, idesc, (it | q | k4) != 0);
+          }
+        }
+        umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
+      }
+      if (ok) {
+        umma_commit(smem_u32(&bar_accum));     // accumulator complete
+      } else {
+        atomicOr(status, CDG_ST_TIMEOUT);
+        atomicExch(&abort_sh, 1);
+      }
+    }
+  } else {
+    // ---------------- accumulator read-back: TMEM -> partial H ----------------
+    const bool ok = (n_iter == 0) ? true : mbar_wait(smem_u32(&bar_accum), 0, deadline);
+    if (!ok) {
+      if (lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+    } else if (n_iter > 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int lg = warp & 3;                 // TMEM lane group this warp may read
+      const int row = lg * 32 + lane;
+      float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.ncols;
+      for (int c0 = 0; c0 < p.ncols; c0 += 16) {
+        uint32_t v[16];
+        const uint32_t taddr = tmem_acc + ((uint32_t)(lg * 32) << 16) + (uint32_t)c0;
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+              "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+              "=r"(v[14]), "=r"(v[15])
+            : "r"(taddr) : "memory");
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < p.rows_used) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4 *>(dst + c0 + j) =
+                make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                            __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+        }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(256u) : "memory");
+  }
+}
+
+// G and b from the per-CTA partial H, summed over CTAs in index order in fp64.
+// thread e < m*m: (k, i) = (e / m, e % m);  m*m <= e < m*m + m: b_i
+__global__ void umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows,
+                                    int m, double *__restrict__ gram) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= m * m + m) return;
+  double acc = 0.0;
+  if (e < m * m) {
+    const int k = e / m, i = e % m;
+    for (int c = 0; c < ctas; ++c) {
+      const float *P = partials + (size_t)c * 128 * ncols;
+      acc += ((double)P[(size_t)k * ncols + i] - (double)P[(size_t)k * ncols + m + i]) -
+             ((double)P[(size_t)(m + k) * ncols + i] - (double)P[(size_t)(m + k) * ncols + m + i]);
+    }
+  } else {
+    const int i = e - m * m;
+    for (int c = 0; c < ctas; ++c) {
+      const float *P = partials + (size_t)c * 128 * ncols;
+      double t = 0.0;
+      for (int j = 0; j < 3; ++j)
+        t += (double)P[(size_t)i * ncols + box_rows + j] - (double)P[(size_t)(m + i) * ncols + box_rows + j];
+      acc += t;
+    }
+  }
+  gram[e] = acc;
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+// 2-D bf16 map over `rows` rows of `d` columns, row pitch `pitch_elems`, box [box_rows][64]
+bool encode_map(CUtensorMap *map, const void *base, long long d, int rows, long long pitch_elems, int box_rows) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kSubCols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool cdg_umma_supported(int m, long long d, int dtype) {
+  // bf16 rows whose pitch is a multiple of 16 bytes; 2m rows fit one 128-row MMA tile
+  return dtype == CDGRAB_BF16 && m <= 64 && d % 8 == 0 && d >= 4096 && encode_fn() != nullptr;
+}
+
+int cdg_umma_setup(cdgrab_ctx *h) {
+  const int box_rows = ((2 * h->m + 15) / 16) * 16;
+  h->umma_box_rows = box_rows;
+  h->umma_ncols = box_rows + kRBoxRows;
+  h->umma_subs_per_stage = 4;
+  const size_t sub_bytes = (size_t)h->umma_ncols * 128;
+  const size_t stage_bytes = sub_bytes * h->umma_subs_per_stage;
+  const size_t slack = (128 * 128 > sub_bytes) ? 128 * 128 - sub_bytes : 0;  // operand A reads 128 rows
+  const size_t budget = 226 * 1024 - 1024 - slack;
+  int stages = (int)(budget / stage_bytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return CDGRAB_ERR_INVALID;
+  h->umma_stages = stages;
+  h->umma_smem = stages * stage_bytes + slack + 1024;
+  const long long total_sub = (h->d + kSubCols - 1) / kSubCols;
+  h->umma_ctas = (int)((total_sub < h->num_sms) ? total_sub : h->num_sms);
+  h->d_pad = total_sub * kSubCols;
+  if (cudaMalloc(&h->r_split, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
+      cudaMalloc(&h->umma_partials, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_NOMEM;
+  }
+  if (cudaMemset(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
+      cudaMemset(h->umma_partials, 0, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess)
+    return CDGRAB_ERR_CUDA;
+  if (!encode_map(&h->tm_r, h->r_split, h->d, 3, h->d_pad, kRBoxRows)) return CDGRAB_ERR_CUDA;
+  if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->umma_smem) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  h->tm_g_base = nullptr;
+  return CDGRAB_OK;
+}
+
+void cdg_umma_teardown(cdgrab_ctx *h) {
+  cudaFree(h->r_split);
+  cudaFree(h->umma_partials);
+  h->r_split = nullptr;
+  h->umma_partials = nullptr;
+}
+
+cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  if (grads != h->tm_g_base) {
+    if (!encode_map(&h->tm_g, grads, h->d, 2 * h->m, h->d, h->umma_box_rows)) return cudaErrorInvalidValue;
+    h->tm_g_base = grads;
+  }
+  UmmaParams p;
+  p.box_rows = h->umma_box_rows;
+  p.ncols = h->umma_ncols;
+  p.rows_used = 2 * h->m;
+  p.subs_per_stage = h->umma_subs_per_stage;
+  p.stages = h->umma_stages;
+  p.sub_bytes = (uint32_t)h->umma_ncols * 128u;
+  p.total_sub = (h->d + kSubCols - 1) / kSubCols;
+  {
+    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
+    gram_umma_kernel<<<h->umma_ctas, kThreads, h->umma_smem, st>>>(h->tm_g, h->tm_r, p, h->umma_partials, h->status);
+  }
+  {
+    CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
+    const int total = h->m * h->m + h->m;
+    umma_combine_kernel<<<(total + 127) / 128, 128, 0, st>>>(h->umma_partials, h->umma_ctas, h->umma_ncols,
+                                                             h->umma_box_rows, h->m, h->gram);
+  }
+  return cudaGetLastError();
+}

@@ -1,0 +1,64 @@
+"""Parity of the tensor-core (tcgen05) Gram path against the CPU oracle, bf16 inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2302_00845_b200 import binding
+from parity import Pair
+
+pytestmark = pytest.mark.gpu
+
+
+def grads(m, d, seed, mean=0.0, scale=1.0):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return (torch.randn(2, m, d, generator=g, device="cuda") * scale + mean).to(torch.bfloat16)
+
+
+def run(m, n, d, seed, mean=0.0, scale=1.0):
+    pr = Pair(m, n, d, "bf16")
+    try:
+        assert pr.gpu.path == "umma"
+        pr.begin()
+        for k in range(n // 2):
+            pr.step(grads(m, d, seed * 100 + k, mean, scale))
+        return pr.end()
+    finally:
+        pr.close()
+
+
+@pytest.mark.parametrize("m,n,d", [
+    (4, 4, 4096),          # one 16-row box, few K blocks: fewer CTAs than SMs
+    (64, 4, 8192),         # full 128-row tile
+    (32, 4, 64 * 148 * 3 + 8),   # every SM busy, ragged last K block
+    (17, 6, 100_000),      # 2m not a multiple of 16
+    (64, 4, 1_000_000),    # many pipeline turns per CTA
+])
+def test_umma_shapes(m, n, d, monkeypatch):
+    monkeypatch.setenv("CDGRAB_FORCE_PATH", "umma")
+    rep = run(m, n, d, seed=m + d % 7)
+    print(f"umma m={m} n={n} d={d}:", rep)
+    assert rep.raw_agreement > 0.9
+
+
+def test_umma_with_common_mean(monkeypatch):
+    """A shared mean ten times the noise: the raw-gradient Gram cancels in four terms."""
+    monkeypatch.setenv("CDGRAB_FORCE_PATH", "umma")
+    rep = run(16, 6, 262_144, seed=3, mean=1.0, scale=0.1)
+    print("umma common mean:", rep)
+
+
+def test_umma_matches_fma_path_signs(monkeypatch):
+    m, n, d = 8, 6, 65536
+    out = {}
+    for path in ("umma", "fma"):
+        monkeypatch.setenv("CDGRAB_FORCE_PATH", path)
+        with binding.CdGrab(m, n, d, "bf16") as h:
+            assert h.path == path
+            h.begin_epoch()
+            for k in range(n // 2):
+                h.step(grads(m, d, 500 + k, mean=0.2))
+            out[path] = (h.signs().cpu(), h.r().cpu(), h.margins().cpu())
+            assert h.status() == binding.OK
+    assert torch.equal(out["umma"][0], out["fma"][0])
+    assert torch.equal(out["umma"][1], out["fma"][1])   # same signs -> same fp32 update order
+    np.testing.assert_allclose(out["umma"][2].numpy(), out["fma"][2].numpy(), rtol=1e-3, atol=1e-6)
