@@ -53,7 +53,18 @@ def parse_args():
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="do not record per-kernel events inside the timed region")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--d", type=int, default=0, help="override d (smaller cases for profiler captures)")
+    ap.add_argument("--m", type=int, default=0, help="override m")
     return ap.parse_args()
+
+
+def pick_workload(args) -> synth.Workload:
+    wl = synth.WORKLOADS[args.workload]
+    if args.d:
+        wl = wl.scaled(d=args.d, name=f"{wl.name}@d={args.d}")
+    if args.m:
+        wl = wl.scaled(m=args.m, name=f"{wl.name}@m={args.m}")
+    return wl
 
 
 # ------------------------------------------------------------------------------------------
@@ -169,7 +180,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    wl = synth.WORKLOADS[args.workload]
+    wl = pick_workload(args)
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     # sample: S workers per step, sized from one probe so the whole run ends within minutes
     S_cap = min(wl.m, 4)
@@ -231,7 +242,7 @@ def run_native(args):
     if world > 1:
         dist.barrier()
 
-    wl = synth.WORKLOADS[args.workload]
+    wl = pick_workload(args)
     if wl.kind == "logreg":
         raise SystemExit("bench.py: the logistic-regression workload is covered by the parity tests")
     m, n, d = wl.m, wl.n, wl.d
