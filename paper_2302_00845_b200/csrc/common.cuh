@@ -58,9 +58,11 @@ struct cdgrab_ctx {
   int umma_subs_per_stage;
   int umma_stages;
   size_t umma_smem;
-  CUtensorMap tm_r;        // tensor map over r_split
-  const void *tm_g_base;   // gradient buffer the cached map was encoded for
-  CUtensorMap tm_g;
+  CUtensorMap tm_r;        // 3-D tensor map over r_split
+  CUtensorMap tm_r2;       // 2-D map over r_split (ragged last block)
+  const void *tm_g_base;   // gradient buffer the cached maps were encoded for
+  CUtensorMap tm_g;        // 3-D map over the gradient rows
+  CUtensorMap tm_g2;       // 2-D map over the gradient rows (ragged last block)
 };
 
 template <typename T>

@@ -10,15 +10,22 @@
 //     b_i = <r, c_i> = sum_j (H[i][R+j] - H[m+i][R+j])
 // falls out of the same MMA.
 //
-// One persistent CTA per SM owns a contiguous K range (split-K).  Per 64-column block the TMA
-// engine lands a [box_rows x 64] gradient box and a [16 x 64] box of the r rows (rows past
-// the tensor are zero-filled) back to back in 128-byte-swizzled shared memory; the same bytes
-// serve as operand A (rows 0..127 from the block base) and operand B (the first N =
-// box_rows + 16 rows).  Roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner,
-// warps 2..5 read the accumulator back (tcgen05.ld) and write the CTA's partial H.
+// One persistent CTA per SM owns a contiguous K range (split-K) in blocks of 64 columns.
+// A pipeline stage holds `subs` consecutive blocks.  Rows are loaded in groups of 8 by 3-D TMA
+// boxes {64 columns, 8 rows, subs blocks}: one instruction touches only 8 rows and
+// subs*128 contiguous bytes of each, which keeps address translation and DRAM pages local
+// even though consecutive rows lie hundreds of megabytes apart.  In shared memory a stage is
+// [row group][block][8 rows][128 B, 128-byte swizzle]; the MMA descriptors walk row groups
+// with a stride of subs*1024 bytes.  Row groups 0..box_rows/8-1 hold gradient rows (rows past
+// 2m are zero-filled by TMA), the next group holds the three r rows, and one more group of
+// zeros (written once) pads N to a multiple of 16.  The same bytes serve as operand A (16
+// row groups from the block base) and operand B (the first N = box_rows + 16 rows).  A ragged
+// last block (d not a multiple of 64) is loaded with 2-D boxes of 8 rows into the same layout.
+// Roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2..5 read the accumulator back (tcgen05.ld) and write the CTA's partial H.
 // Every wait is bounded: on expiry the CTA raises the time-out bit of the status word,
 // drains the copies it has in flight, frees its TMEM and returns.
 #include <cudaTypedefs.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -31,13 +38,13 @@ constexpr int kRBoxRows = 16;
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
 
 struct UmmaParams {
-  int box_rows;        // rows of the gradient box (2m rounded up to 16)
+  int box_rows;        // gradient rows held per block (2m rounded up to 16)
   int ncols;           // MMA N = box_rows + 16
   int rows_used;       // 2m
-  int subs_per_stage;
+  int subs;            // 64-column blocks per stage
   int stages;
-  uint32_t sub_bytes;  // ncols * 128
-  long long total_sub; // ceil(d / 64)
+  long long nblk_full; // d / 64: blocks loaded by the 3-D maps
+  int tail;            // 1 when d % 64 != 0: one more, ragged block
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -69,13 +76,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
 
-// K-major, 128-byte swizzle: rows 128 B apart, 8-row groups 1024 B apart
-__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+// K-major, 128-byte swizzle: rows 128 B apart, 8-row groups `sbo` bytes apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t sbo) {
   uint64_t d = 0;
   d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address
   d |= (uint64_t)1 << 16;                          // leading byte offset (unused for this layout)
-  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+  d |= (uint64_t)(sbo >> 4) << 32;                 // stride byte offset between 8-row groups
   d |= (uint64_t)1 << 46;                          // descriptor version
   d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
   return d;
@@ -92,24 +104,27 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
+gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constant__ CUtensorMap tm_r3,
+                 const __grid_constant__ CUtensorMap tm_g2, const __grid_constant__ CUtensorMap tm_r2,
                  const UmmaParams p, float *__restrict__ partials, int *__restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
   __shared__ __align__(8) uint64_t bar_accum;
   __shared__ uint32_t tmem_base_sh;
-  __shared__ int abort_sh;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-B alignment
-  const uint32_t stage_bytes = p.sub_bytes * p.subs_per_stage;
+  const uint32_t group_bytes = (uint32_t)p.subs * 1024u;         // one row group of a stage
+  const int ngroups = p.ncols >> 3;
+  const int ggroups = p.box_rows >> 3;                           // gradient row groups
+  const uint32_t stage_bytes = group_bytes * ngroups;
 
-  // this CTA's K range, in 64-column blocks
-  const long long sub_lo = p.total_sub * (long long)blockIdx.x / gridDim.x;
-  const long long sub_hi = p.total_sub * (long long)(blockIdx.x + 1) / gridDim.x;
-  const long long nsub = sub_hi - sub_lo;
-  const int n_iter = (int)((nsub + p.subs_per_stage - 1) / p.subs_per_stage);
+  // this CTA's K range in full blocks; the last CTA also owns the ragged block, taken first
+  const long long blk_lo = p.nblk_full * (long long)blockIdx.x / gridDim.x;
+  const long long blk_hi = p.nblk_full * (long long)(blockIdx.x + 1) / gridDim.x;
+  const int has_tail = (p.tail && blockIdx.x == gridDim.x - 1) ? 1 : 0;
+  const int n_iter = has_tail + (int)((blk_hi - blk_lo + p.subs - 1) / p.subs);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -117,9 +132,20 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
     mbar_init(smem_u32(&bar_accum), 1);
-    abort_sh = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // row groups that are never loaded (gradient groups wholly past row 2m, and the padding
+  // group after the r rows) are zeroed once
+  const int lgroups = (p.rows_used + 7) >> 3;                    // gradient row groups that get loaded
+  for (int s = 0; s < p.stages; ++s) {
+    for (int g = lgroups; g < ngroups; ++g) {
+      if (g == ggroups) continue;                                // the r rows
+      uint8_t *z = smem_raw + (tiles - smem_u32(smem_raw)) + (size_t)s * stage_bytes + (size_t)g * group_bytes;
+      for (uint32_t o = threadIdx.x * 16; o < group_bytes; o += kThreads * 16)
+        *reinterpret_cast<uint4 *>(z + o) = make_uint4(0, 0, 0, 0);
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // visible to the MMA's smem reads
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(&tmem_base_sh)), "r"(256u) : "memory");
@@ -140,21 +166,24 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant
         const int s = it % p.stages;
         if (it >= p.stages) ok = mbar_wait(smem_u32(&bar_empty[s]), ((it / p.stages) - 1) & 1, deadline);
         if (!ok) break;
-        const long long first = sub_lo + (long long)it * p.subs_per_stage;
-        const int cnt = (int)min((long long)p.subs_per_stage, sub_hi - first);
         const uint32_t full = smem_u32(&bar_full[s]);
-        mbar_expect_tx(full, cnt * p.sub_bytes);
-        for (int q = 0; q < cnt; ++q) {
-          const uint32_t dst = tiles + s * stage_bytes + q * p.sub_bytes;
-          const int col = (int)((first + q) * kSubCols);  // 64 bf16 = 128 bytes: 16-byte aligned
-          tma_load_2d(dst, &tm_g, col, 0, full);
-          tma_load_2d(dst + (uint32_t)p.box_rows * 128u, &tm_r, col, 0, full);
+        const uint32_t base = tiles + s * stage_bytes;
+        if (has_tail && it == 0) {
+          // ragged block: 8-row 2-D boxes into block slot 0 of every loaded row group
+          const int col = (int)(p.nblk_full * kSubCols);   // 128-byte aligned
+          mbar_expect_tx(full, (uint32_t)(lgroups + 1) * 1024u);
+          for (int g = 0; g < lgroups; ++g) tma_load_2d(base + g * group_bytes, &tm_g2, col, g * 8, full);
+          tma_load_2d(base + ggroups * group_bytes, &tm_r2, col, 0, full);
+        } else {
+          const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
+          mbar_expect_tx(full, (uint32_t)(lgroups + 1) * group_bytes);
+          for (int g = 0; g < lgroups; ++g) tma_load_3d(base + g * group_bytes, &tm_g3, 0, g * 8, (int)first, full);
+          tma_load_3d(base + ggroups * group_bytes, &tm_r3, 0, 0, (int)first, full);
         }
         issued = it + 1;
       }
       if (!ok) {
         atomicOr(status, CDG_ST_TIMEOUT);
-        atomicExch(&abort_sh, 1);
         // let the copies already issued land before the CTA gives up its shared memory
         for (int it = max(0, issued - p.stages); it < issued; ++it)
           mbar_wait(smem_u32(&bar_full[it % p.stages]), (it / p.stages) & 1, clock64() + kWaitCycles);
@@ -172,10 +201,13 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant
         ok = mbar_wait(smem_u32(&bar_full[s]), (it / p.stages) & 1, deadline);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const long long first = sub_lo + (long long)it * p.subs_per_stage;
-        const int cnt = (int)min((long long)p.subs_per_stage, sub_hi - first);
+        int cnt = 1;
+        if (!(has_tail && it == 0)) {
+          const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
+          cnt = (int)min((long long)p.subs, blk_hi - first);   // blocks past blk_hi belong to the next CTA
+        }
         for (int q = 0; q < cnt; ++q) {
-          const uint64_t desc = umma_desc(tiles + s * stage_bytes + q * p.sub_bytes);
+          const uint64_t desc = umma_desc(tiles + s * stage_bytes + q * 1024u, group_bytes);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4) {
             // 16 bf16 = 32 bytes further along K inside the swizzle row
@@ -185,34 +217,35 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant
         }
         umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
       }
-      if (ok) {
-        umma_commit(smem_u32(&bar_accum));     // accumulator complete
-      } else {
-        atomicOr(status, CDG_ST_TIMEOUT);
-        atomicExch(&abort_sh, 1);
-      }
+      if (ok) umma_commit(smem_u32(&bar_accum));  // accumulator complete
+      else atomicOr(status, CDG_ST_TIMEOUT);
     }
   } else {
     // ---------------- accumulator read-back: TMEM -> partial H ----------------
     const bool ok = (n_iter == 0) ? true : mbar_wait(smem_u32(&bar_accum), 0, deadline);
     if (!ok) {
       if (lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
-    } else if (n_iter > 0) {
+    } else {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int lg = warp & 3;                 // TMEM lane group this warp may read
       const int row = lg * 32 + lane;
       float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.ncols;
       for (int c0 = 0; c0 < p.ncols; c0 += 16) {
         uint32_t v[16];
-        const uint32_t taddr = tmem_acc + ((uint32_t)(lg * 32) << 16) + (uint32_t)c0;
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
-              "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
-              "=r"(v[14]), "=r"(v[15])
-            : "r"(taddr) : "memory");
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (n_iter > 0) {
+          const uint32_t taddr = tmem_acc + ((uint32_t)(lg * 32) << 16) + (uint32_t)c0;
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+              "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+                "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+                "=r"(v[14]), "=r"(v[15])
+              : "r"(taddr) : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0u;
+        }
         if (row < p.rows_used) {
 #pragma unroll
           for (int j = 0; j < 16; j += 4)
@@ -275,15 +308,29 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-// 2-D bf16 map over `rows` rows of `d` columns, row pitch `pitch_elems`, box [box_rows][64]
-bool encode_map(CUtensorMap *map, const void *base, long long d, int rows, long long pitch_elems, int box_rows) {
+// 2-D bf16 map over `rows` rows of `d` columns, row pitch `pitch_elems`, box [8 rows][64]
+bool encode_map_2d(CUtensorMap *map, const void *base, long long d, int rows, long long pitch_elems) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 2};
-  cuuint32_t box[2] = {(cuuint32_t)kSubCols, (cuuint32_t)box_rows};
+  cuuint32_t box[2] = {(cuuint32_t)kSubCols, 8};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 3-D view {64 columns, rows, nblk blocks of 64 columns} of the same memory (block pitch 128 bytes),
+// box {64, 8 rows, subs blocks}
+bool encode_map_3d(CUtensorMap *map, const void *base, long long nblk, int rows, long long pitch_elems, int subs) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)kSubCols, (cuuint64_t)rows, (cuuint64_t)nblk};
+  cuuint64_t strides[2] = {(cuuint64_t)pitch_elems * 2, (cuuint64_t)kSubCols * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kSubCols, 8, (cuuint32_t)subs};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -299,18 +346,25 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   const int box_rows = ((2 * h->m + 15) / 16) * 16;
   h->umma_box_rows = box_rows;
   h->umma_ncols = box_rows + kRBoxRows;
-  h->umma_subs_per_stage = 4;
-  const size_t sub_bytes = (size_t)h->umma_ncols * 128;
-  const size_t stage_bytes = sub_bytes * h->umma_subs_per_stage;
-  const size_t slack = (128 * 128 > sub_bytes) ? 128 * 128 - sub_bytes : 0;  // operand A reads 128 rows
+  int subs = 4;
+  if (const char *e = getenv("CDGRAB_UMMA_SUBS")) {   // tuning knob: 64-column blocks per stage
+    const int v = atoi(e);
+    if (v >= 1 && v <= 8) subs = v;
+  }
+  h->umma_subs_per_stage = subs;
+  const size_t group_bytes = (size_t)subs * 1024;
+  const size_t stage_bytes = group_bytes * (h->umma_ncols / 8);
+  const int ngroups = h->umma_ncols / 8;
+  const size_t slack = (ngroups < 16) ? (16 - ngroups) * group_bytes : 0;  // operand A spans 16 row groups
   const size_t budget = 226 * 1024 - 1024 - slack;
   int stages = (int)(budget / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return CDGRAB_ERR_INVALID;
   h->umma_stages = stages;
   h->umma_smem = stages * stage_bytes + slack + 1024;
+  const long long nblk_full = h->d / kSubCols;
   const long long total_sub = (h->d + kSubCols - 1) / kSubCols;
-  h->umma_ctas = (int)((total_sub < h->num_sms) ? total_sub : h->num_sms);
+  h->umma_ctas = (int)((nblk_full < h->num_sms) ? (nblk_full > 0 ? nblk_full : 1) : h->num_sms);
   h->d_pad = total_sub * kSubCols;
   if (cudaMalloc(&h->r_split, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
       cudaMalloc(&h->umma_partials, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess) {
@@ -320,7 +374,8 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   if (cudaMemset(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
       cudaMemset(h->umma_partials, 0, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess)
     return CDGRAB_ERR_CUDA;
-  if (!encode_map(&h->tm_r, h->r_split, h->d, 3, h->d_pad, kRBoxRows)) return CDGRAB_ERR_CUDA;
+  if (!encode_map_3d(&h->tm_r, h->r_split, nblk_full, 3, h->d_pad, subs)) return CDGRAB_ERR_CUDA;
+  if (!encode_map_2d(&h->tm_r2, h->r_split, h->d, 3, h->d_pad)) return CDGRAB_ERR_CUDA;
   if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->umma_smem) !=
       cudaSuccess) {
     cudaGetLastError();
@@ -338,21 +393,25 @@ void cdg_umma_teardown(cdgrab_ctx *h) {
 }
 
 cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  const long long nblk_full = h->d / kSubCols;
   if (grads != h->tm_g_base) {
-    if (!encode_map(&h->tm_g, grads, h->d, 2 * h->m, h->d, h->umma_box_rows)) return cudaErrorInvalidValue;
+    if (!encode_map_3d(&h->tm_g, grads, nblk_full, 2 * h->m, h->d, h->umma_subs_per_stage) ||
+        !encode_map_2d(&h->tm_g2, grads, h->d, 2 * h->m, h->d))
+      return cudaErrorInvalidValue;
     h->tm_g_base = grads;
   }
   UmmaParams p;
   p.box_rows = h->umma_box_rows;
   p.ncols = h->umma_ncols;
   p.rows_used = 2 * h->m;
-  p.subs_per_stage = h->umma_subs_per_stage;
+  p.subs = h->umma_subs_per_stage;
   p.stages = h->umma_stages;
-  p.sub_bytes = (uint32_t)h->umma_ncols * 128u;
-  p.total_sub = (h->d + kSubCols - 1) / kSubCols;
+  p.nblk_full = nblk_full;
+  p.tail = (h->d % kSubCols) ? 1 : 0;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
-    gram_umma_kernel<<<h->umma_ctas, kThreads, h->umma_smem, st>>>(h->tm_g, h->tm_r, p, h->umma_partials, h->status);
+    gram_umma_kernel<<<h->umma_ctas, kThreads, h->umma_smem, st>>>(h->tm_g, h->tm_r, h->tm_g2, h->tm_r2, p,
+                                                                   h->umma_partials, h->status);
   }
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
