@@ -48,7 +48,8 @@ enum {
   CDGRAB_ERR_NOMEM = -4,     /* device or host allocation failed                         */
   CDGRAB_ERR_NONFINITE = -5, /* NaN/Inf met in a reduction (device status word)          */
   CDGRAB_ERR_TIMEOUT = -6,   /* a bounded device-side wait expired (device status word)  */
-  CDGRAB_ERR_DEVICE = -7     /* no usable sm_100 device                                  */
+  CDGRAB_ERR_DEVICE = -7,    /* no usable sm_100 device                                  */
+  CDGRAB_ERR_TOO_LARGE = -8  /* size beyond the fixed scratch of cdgrab_step_noalloc        */
 };
 
 /* Which code path a handle uses (cdgrab_path / CDGRAB_FORCE_PATH). */
@@ -191,6 +192,43 @@ int cdgrab_logreg_grads(cdgrab_t *h, const float *X, const float *y, const float
  * 2*m*d elements, 16-byte aligned, caller-owned) on `stream`, then cdgrab_step runs on it.
  */
 int cdgrab_step_host(cdgrab_t *h, const void *grads_host, void *staging_dev, void *stream);
+
+/*
+ * One balancing step that allocates nothing (the paper has no counterpart: this is a
+ * packaging of cdgrab_step for a restricted kind of caller).
+ *
+ * Some callers cannot call cudaMalloc: plug-ins that are handed buffers and a stream and
+ * nothing else, code inside a framework's caching allocator whose pool a raw allocation
+ * would fragment or overrun, loops that cannot afford the device-wide synchronisation an
+ * allocation or a free implies.  They cannot use cdgrab_create either.  This call keeps no
+ * handle: the caller owns the running sum and the signs, and the scratch of the two-pass
+ * formulation (block partial sums, Gram matrix, a few bookkeeping words) lives in one fixed
+ * array of 625,152 bytes in the library's device image, which every GPU that loads the
+ * library holds until the process exits.
+ *
+ *   m          workers, 1 <= m <= 16; more is CDGRAB_ERR_TOO_LARGE (the fixed scratch and the
+ *              register-resident kernels behind this call stop there)
+ *   d          gradient dimension, a multiple of 4, d >= 4 (else CDGRAB_ERR_INVALID)
+ *   dtype      CDGRAB_F32 or CDGRAB_BF16
+ *   grads_dev  DEVICE, [2][m][d] as for cdgrab_step, 16-byte aligned, caller-owned
+ *   r_dev      DEVICE, float [d], 16-byte aligned, caller-owned: the running sum, read and
+ *              updated in place (zero it yourself at the start of an epoch)
+ *   signs_out_dev  DEVICE, int8 [m], caller-owned: receives the m signs of this step
+ *
+ * Same arithmetic as cdgrab_step on the FMA path: for i = 0..m-1, s_i = +1 iff <r,c_i> < 0
+ * with c_i = z1_i - z2_i, then r <- r + s_i c_i.  The caller applies the signs to its own
+ * permutations (item with +1 to the front slot, the other to the back slot).
+ *
+ * The first call on a device resolves the scratch array's device address and writes its
+ * constant part; that call is synchronous and should be made before any stream capture is
+ * begun.  Later calls only enqueue work on `stream`.  No call allocates or frees memory.
+ * All calls on a device share the scratch, which keeps the previous call's contents; the
+ * words that must start at zero are cleared on `stream` at every call.  Two calls whose
+ * device work may overlap (different streams without ordering, or several host threads)
+ * race on the scratch: order them.
+ */
+int cdgrab_step_noalloc(int m, long long d, int dtype, const void *grads_dev, float *r_dev,
+                        int8_t *signs_out_dev, void *stream);
 
 #ifdef __cplusplus
 }

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(HERE, "libcdgrab.so")
 F32, BF16 = 0, 1
 OK = 0
 ERR_INVALID, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_NONFINITE, ERR_TIMEOUT, ERR_DEVICE = -1, -2, -3, -4, -5, -6, -7
+ERR_TOO_LARGE = -8
 PATH_AUTO, PATH_FUSED, PATH_FMA, PATH_UMMA = 0, 1, 2, 3
 KERNEL_KINDS = ("gram", "combine", "scan", "update", "fused", "logreg")
 PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma"}
@@ -41,6 +42,8 @@ SIGNATURES = {
     "cdgrab_profile_read": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]),
     "cdgrab_logreg_grads": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_step_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_step_noalloc": (C.c_int, [C.c_int, C.c_longlong, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p]),
 }
 
 _lib = None
@@ -196,3 +199,13 @@ class CdGrab:
     @property
     def launch_count(self) -> int:
         return int(lib().cdgrab_launch_count(self._h))
+
+
+def step_noalloc(grads, r, signs_out, stream=None):
+    """cdgrab_step_noalloc on torch tensors: grads [2][m][d] (f32 or bf16), r float32 [d] updated in
+    place, signs_out int8 [m].  Allocates nothing on the device."""
+    import torch
+    m, d = int(grads.shape[1]), int(grads.shape[2])
+    code = F32 if grads.dtype == torch.float32 else BF16
+    _check(lib().cdgrab_step_noalloc(m, d, code, _ptr(grads), _ptr(r), _ptr(signs_out), _stream_ptr(stream)),
+           "cdgrab_step_noalloc")

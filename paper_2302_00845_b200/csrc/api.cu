@@ -68,6 +68,7 @@ const char *cdgrab_strerror(int code) {
     case CDGRAB_ERR_NONFINITE: return "non-finite value met in a reduction";
     case CDGRAB_ERR_TIMEOUT: return "bounded device-side wait expired";
     case CDGRAB_ERR_DEVICE: return "no usable sm_100 CUDA device";
+    case CDGRAB_ERR_TOO_LARGE: return "size beyond the fixed scratch of the no-allocation entry point";
     default: return "unknown error";
   }
 }

@@ -40,11 +40,11 @@ def test_the_five_named_calls_exist():
 
 def test_strerror_covers_all_codes(lib):
     seen = set()
-    for code in range(0, -8, -1):
+    for code in range(0, -9, -1):
         msg = lib.cdgrab_strerror(code).decode()
         assert msg and msg != "unknown error"
         seen.add(msg)
-    assert len(seen) == 8
+    assert len(seen) == 9
     assert lib.cdgrab_strerror(-99).decode() == "unknown error"
 
 
