@@ -133,13 +133,22 @@ gram_fma_kernel(const T *__restrict__ g, const float *__restrict__ r, int m, lon
   if (threadIdx.x < Tri<M>::NACC) partials[(size_t)blockIdx.x * Tri<M>::NACC + threadIdx.x] = v;
 }
 
+// 6 slices of the block list are summed side by side (slice p takes blocks p, p+6, ...), then
+// the slices are added in index order: fixed order for a fixed grid.
 template <int M>
-__global__ void fma_combine_kernel(const double *__restrict__ partials, int blocks, int m,
-                                   double *__restrict__ gram) {
-  const int e = threadIdx.x;
-  if (e >= Tri<M>::NACC) return;
+__global__ void __launch_bounds__(6 * Tri<M>::NPAD)
+fma_combine_kernel(const double *__restrict__ partials, int blocks, int m, double *__restrict__ gram) {
+  __shared__ double part[6][Tri<M>::NPAD];
+  const int e = threadIdx.x % Tri<M>::NPAD, slice = threadIdx.x / Tri<M>::NPAD;
   double v = 0.0;
-  for (int b = 0; b < blocks; ++b) v += partials[(size_t)b * Tri<M>::NACC + e];
+  if (e < Tri<M>::NACC)
+    for (int b = slice; b < blocks; b += 6) v += partials[(size_t)b * Tri<M>::NACC + e];
+  part[slice][e] = v;
+  __syncthreads();
+  if (slice != 0 || e >= Tri<M>::NACC) return;
+  v = 0.0;
+#pragma unroll
+  for (int p = 0; p < 6; ++p) v += part[p][e];
   if (e < Tri<M>::NPAIR) {
     int a = 0, rem = e;
     while (rem >= M - a) { rem -= M - a; ++a; }
@@ -290,7 +299,7 @@ static cudaError_t launch_gram_fma_t(cdgrab_ctx *h, const void *grads, cudaStrea
   }
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
-    fma_combine_kernel<M><<<1, 192, 0, st>>>(h->partials, h->gram_chunks, h->m, h->gram);
+    fma_combine_kernel<M><<<1, 6 * Tri<M>::NPAD, 0, st>>>(h->partials, h->gram_chunks, h->m, h->gram);
   }
   return cudaGetLastError();
 }

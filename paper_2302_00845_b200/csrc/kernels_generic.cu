@@ -114,56 +114,72 @@ __global__ void gram_combine_kernel(const double *__restrict__ partials, int chu
 }
 
 // ------------------------------------------------------------------------------------
-// scan: m sequential decisions in scalar space + permutation slots.  One warp.
+// scan: m sequential decisions in scalar space + permutation slots.  The block stages G, b
+// and the current pairs in shared memory, warp 0 takes the decisions, the block writes out.
 //   t_j starts as b_j; after worker i is decided every later t_j gains s_i G_ij, so when
 //   worker j's turn comes t_j = <r_{j-1}, c_j> (summed in the order k = 0..j-1).
 // ------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(32)
+__global__ void __launch_bounds__(256)
 scan_kernel(const double *__restrict__ gram, int m, int n, int k,
             const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
             int8_t *__restrict__ signs, float *__restrict__ margins,
             double *__restrict__ rnorm2, int *__restrict__ status, int use_smem) {
   extern __shared__ double sh[];
-  double *tsh = sh;            // [m]
-  double *gsh = sh + m;        // [m][m] when use_smem
-  const int lane = threadIdx.x;
+  double *tsh = sh;                                   // [m]
+  float *msh = reinterpret_cast<float *>(sh + m);     // [m] margins
+  int *ssh = reinterpret_cast<int *>(msh + m);        // [m] signs
+  int *psh = ssh + m;                                 // [2m] the current pair of every worker
+  double *gsh = sh + 3 * m;                           // [m][m] when use_smem (4m words = 2m doubles above)
+  const int tid = threadIdx.x;
   const double *G = gram;
   const double *b = gram + (size_t)m * m;
-  for (int j = lane; j < m; j += 32) tsh[j] = b[j];
+  for (int j = tid; j < m; j += blockDim.x) {
+    tsh[j] = b[j];
+    psh[2 * j] = perm_cur[(size_t)j * n + 2 * k];
+    psh[2 * j + 1] = perm_cur[(size_t)j * n + 2 * k + 1];
+  }
   if (use_smem) {
-    for (int e = lane; e < m * m; e += 32) gsh[e] = G[e];
+    for (int e = tid; e < m * m; e += blockDim.x) gsh[e] = G[e];
     G = gsh;
   }
-  __syncwarp();
-  double rn2 = *rnorm2;
-  const int half = n >> 1;
-  bool bad = false;
-  for (int i = 0; i < m; ++i) {
-    const double ti = tsh[i];
-    const double gii = G[(size_t)i * m + i];
-    // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0; a tie gives -1
-    const int s = (ti < 0.0) ? 1 : -1;
-    bad |= !(isfinite(ti) && isfinite(gii));
-    const double sd = (double)s;
-    for (int j = i + 1 + lane; j < m; j += 32) tsh[j] += sd * G[(size_t)i * m + j];
-    if (lane == 0) {
-      const size_t pos = (size_t)i * half + k;
-      signs[pos] = (int8_t)s;
-      const double den = rn2 * gii;
-      margins[pos] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
-      // Algorithm 7: the item that received +1 goes to the front slot, the other to the back
-      const int32_t first = perm_cur[(size_t)i * n + 2 * k];
-      const int32_t second = perm_cur[(size_t)i * n + 2 * k + 1];
-      perm_next[(size_t)i * n + k] = (s == 1) ? first : second;
-      perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;
+  __syncthreads();
+  if (tid < 32) {
+    const int lane = tid;
+    double rn2 = *rnorm2;
+    bool bad = false;
+    for (int i = 0; i < m; ++i) {
+      const double ti = tsh[i];
+      const double gii = G[(size_t)i * m + i];
+      // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0; a tie gives -1
+      const int s = (ti < 0.0) ? 1 : -1;
+      bad |= !(isfinite(ti) && isfinite(gii));
+      const double sd = (double)s;
+      for (int j = i + 1 + lane; j < m; j += 32) tsh[j] += sd * G[(size_t)i * m + j];
+      if (lane == 0) {
+        ssh[i] = s;
+        const double den = rn2 * gii;
+        msh[i] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
+      }
+      rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
+      if (rn2 < 0.0) rn2 = 0.0;
+      __syncwarp();
     }
-    rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
-    if (rn2 < 0.0) rn2 = 0.0;
-    __syncwarp();
+    if (lane == 0) {
+      *rnorm2 = rn2;
+      if (bad) atomicOr(status, CDG_ST_NONFINITE);
+    }
   }
-  if (lane == 0) {
-    *rnorm2 = rn2;
-    if (bad) atomicOr(status, CDG_ST_NONFINITE);
+  __syncthreads();
+  const int half = n >> 1;
+  for (int i = tid; i < m; i += blockDim.x) {
+    const int s = ssh[i];
+    const size_t pos = (size_t)i * half + k;
+    signs[pos] = (int8_t)s;
+    margins[pos] = msh[i];
+    // Algorithm 7: the item that received +1 goes to the front slot, the other to the back
+    const int32_t first = psh[2 * i], second = psh[2 * i + 1];
+    perm_next[(size_t)i * n + k] = (s == 1) ? first : second;
+    perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;
   }
 }
 
@@ -194,6 +210,33 @@ struct VecLoad<__nv_bfloat16, 8> {
       v[2 * j] = __uint_as_float(w[j] << 16);
       v[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
     }
+  }
+};
+// 256-bit loads (sm_100): one 32-byte request per row and thread
+__device__ __forceinline__ void ld256(const void *p, uint32_t (&w)[8]) {
+  asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+               : "l"(p));
+}
+template <>
+struct VecLoad<__nv_bfloat16, 16> {
+  static __device__ __forceinline__ void ld(const __nv_bfloat16 *p, float (&v)[16]) {
+    uint32_t w[8];
+    ld256(p, w);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      v[2 * j] = __uint_as_float(w[j] << 16);
+      v[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+  }
+};
+template <>
+struct VecLoad<float, 8> {
+  static __device__ __forceinline__ void ld(const float *p, float (&v)[8]) {
+    uint32_t w[8];
+    ld256(p, w);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(w[j]);
   }
 };
 template <>
@@ -230,7 +273,7 @@ update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__re
     }
 #pragma unroll
     for (int j = 0; j < VEC; ++j) acc[j] = (AccT)rv[j];
-#pragma unroll 4
+#pragma unroll 2
     for (int i = 0; i < m; ++i) {
       float a[VEC], b[VEC];
       VecLoad<T, VEC>::ld(g + (size_t)i * (size_t)d + x, a);
@@ -252,16 +295,29 @@ update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__re
     }
     if constexpr (SPLIT) {
       // r = hi + mid + lo exactly (3 x 8 significand bits), consumed by the tensor-core pass
+      __nv_bfloat16 hi[VEC], mid[VEC], lo[VEC];
 #pragma unroll
       for (int j = 0; j < VEC; ++j) {
-        const __nv_bfloat16 hi = __float2bfloat16_rn(rv[j]);
-        const float r1 = rv[j] - __bfloat162float(hi);
-        const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-        const float r2 = r1 - __bfloat162float(mid);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(r2);
-        r_split[x + j] = hi;
-        r_split[(size_t)d_pad + x + j] = mid;
-        r_split[2 * (size_t)d_pad + x + j] = lo;
+        hi[j] = __float2bfloat16_rn(rv[j]);
+        const float r1 = rv[j] - __bfloat162float(hi[j]);
+        mid[j] = __float2bfloat16_rn(r1);
+        lo[j] = __float2bfloat16_rn(r1 - __bfloat162float(mid[j]));
+      }
+      if constexpr (VEC % 8 == 0) {
+        // d_pad is a multiple of 64, x of 8: 16-byte aligned vector stores
+#pragma unroll
+        for (int q = 0; q < VEC / 8; ++q) {
+          *reinterpret_cast<uint4 *>(r_split + x + 8 * q) = *reinterpret_cast<const uint4 *>(hi + 8 * q);
+          *reinterpret_cast<uint4 *>(r_split + (size_t)d_pad + x + 8 * q) = *reinterpret_cast<const uint4 *>(mid + 8 * q);
+          *reinterpret_cast<uint4 *>(r_split + 2 * (size_t)d_pad + x + 8 * q) = *reinterpret_cast<const uint4 *>(lo + 8 * q);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+          r_split[x + j] = hi[j];
+          r_split[(size_t)d_pad + x + j] = mid[j];
+          r_split[2 * (size_t)d_pad + x + j] = lo[j];
+        }
       }
     }
   }
@@ -328,9 +384,10 @@ cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream
 
 cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
   const int m = h->m;
-  const size_t with_g = ((size_t)m * m + m) * sizeof(double);
+  const size_t small = (size_t)3 * m * sizeof(double);  // t, then margins/signs/pairs (4m words)
+  const size_t with_g = small + (size_t)m * m * sizeof(double);
   const int use_smem = with_g <= 160 * 1024;
-  const size_t smem = use_smem ? with_g : (size_t)m * sizeof(double);
+  const size_t smem = use_smem ? with_g : small;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -340,7 +397,7 @@ cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
   }
   {
     CdgProfScope ps(h, CDGRAB_K_SCAN, st);
-    scan_kernel<<<1, 32, smem, st>>>(h->gram, m, h->n, h->k, h->perm_cur, h->perm_next, h->signs,
+    scan_kernel<<<1, 256, smem, st>>>(h->gram, m, h->n, h->k, h->perm_cur, h->perm_next, h->signs,
                                      h->margins, h->rnorm2, h->status, use_smem);
   }
   return cudaGetLastError();
@@ -350,7 +407,7 @@ template <typename T, typename AccT, int VEC>
 static void launch_update_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
   const long long nvec = h->d / VEC;
   long long blocks = (nvec + 255) / 256;
-  const long long cap = (long long)h->num_sms * 16;
+  const long long cap = (long long)h->num_sms * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   const size_t smem = (size_t)h->m * sizeof(float);
@@ -365,11 +422,14 @@ static void launch_update_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
 }
 
 cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  const bool al32 = ((uintptr_t)grads & 31) == 0;   // 256-bit loads need 32-byte aligned rows
   if (h->dtype == CDGRAB_F32) {
-    if (h->d % 4 == 0) launch_update_t<float, double, 4>(h, grads, st);
+    if (al32 && h->d % 8 == 0) launch_update_t<float, double, 8>(h, grads, st);
+    else if (h->d % 4 == 0) launch_update_t<float, double, 4>(h, grads, st);
     else launch_update_t<float, double, 1>(h, grads, st);
   } else {
-    if (h->d % 8 == 0) launch_update_t<__nv_bfloat16, float, 8>(h, grads, st);
+    if (al32 && h->d % 16 == 0) launch_update_t<__nv_bfloat16, float, 16>(h, grads, st);
+    else if (h->d % 8 == 0) launch_update_t<__nv_bfloat16, float, 8>(h, grads, st);
     else launch_update_t<__nv_bfloat16, float, 1>(h, grads, st);
   }
   return cudaGetLastError();

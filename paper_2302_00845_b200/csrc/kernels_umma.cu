@@ -271,24 +271,32 @@ __global__ void umma_combine_kernel(const float *__restrict__ partials, int ctas
                                     int m, double *__restrict__ gram) {
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= m * m + m) return;
-  double acc = 0.0;
+  // CTAs taken four at a time with independent sums (loads stay in flight); fixed order
+  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+  const size_t cs = (size_t)128 * ncols;   // one CTA's partial H
   if (e < m * m) {
     const int k = e / m, i = e % m;
-    for (int c = 0; c < ctas; ++c) {
-      const float *P = partials + (size_t)c * 128 * ncols;
-      acc += ((double)P[(size_t)k * ncols + i] - (double)P[(size_t)k * ncols + m + i]) -
-             ((double)P[(size_t)(m + k) * ncols + i] - (double)P[(size_t)(m + k) * ncols + m + i]);
-    }
+    const size_t o00 = (size_t)k * ncols + i, o01 = o00 + m, o10 = (size_t)(m + k) * ncols + i, o11 = o10 + m;
+    auto term = [&](int c) {
+      const float *P = partials + (size_t)c * cs;
+      return ((double)P[o00] - (double)P[o01]) - ((double)P[o10] - (double)P[o11]);
+    };
+    int c = 0;
+    for (; c + 4 <= ctas; c += 4) { a0 += term(c); a1 += term(c + 1); a2 += term(c + 2); a3 += term(c + 3); }
+    for (; c < ctas; ++c) a0 += term(c);
   } else {
     const int i = e - m * m;
-    for (int c = 0; c < ctas; ++c) {
-      const float *P = partials + (size_t)c * 128 * ncols;
-      double t = 0.0;
-      for (int j = 0; j < 3; ++j)
-        t += (double)P[(size_t)i * ncols + box_rows + j] - (double)P[(size_t)(m + i) * ncols + box_rows + j];
-      acc += t;
-    }
+    const size_t o0 = (size_t)i * ncols + box_rows, o1 = (size_t)(m + i) * ncols + box_rows;
+    auto term = [&](int c) {
+      const float *P = partials + (size_t)c * cs;
+      return (((double)P[o0] - (double)P[o1]) + ((double)P[o0 + 1] - (double)P[o1 + 1])) +
+             ((double)P[o0 + 2] - (double)P[o1 + 2]);
+    };
+    int c = 0;
+    for (; c + 4 <= ctas; c += 4) { a0 += term(c); a1 += term(c + 1); a2 += term(c + 2); a3 += term(c + 3); }
+    for (; c < ctas; ++c) a0 += term(c);
   }
+  const double acc = (a0 + a1) + (a2 + a3);
   gram[e] = acc;
 }
 
