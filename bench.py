@@ -140,6 +140,19 @@ def algorithmic_bytes(kind: str, wl: synth.Workload) -> float:
     return 0.0
 
 
+def aggregate_replicas(ms_local: float, examples_local: int, world: int, device: str):
+    """Whole-job throughput of `world` independent replicas: every rank processed
+    `examples_local` examples; the job's time is the slowest rank's (max over ranks).
+    Returns (examples per second over all ranks, that time in ms)."""
+    ms = ms_local
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_local], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return examples_local * world / (ms * 1e-3), ms
+
+
 def source_hash() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2302_00845_b200", "csrc")
@@ -310,12 +323,7 @@ def run_native(args):
     h.check_status()
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
 
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    examples = 2 * m * args.steps * world
-    value = examples / (ms * 1e-3)
+    value, ms = aggregate_replicas(ms, 2 * m * args.steps, world, "cuda")
 
     # ---- roofline of the dominant kernel ---------------------------------------------------
     peak, peak_kind = peaks()

@@ -1,0 +1,84 @@
+"""Host-side logic of bench.py without a GPU: the N > 1 aggregation over independent replicas
+(world size 2, gloo), the reference arm's line, and the rank rule of the reference arm."""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    # rank 1 is the slower replica: the job's time is its time, the work is the sum
+    value, ms = bench.aggregate_replicas(10.0 * (rank + 1), 128, world, "cpu")
+    out[rank] = (value, ms)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_replica_aggregation_world_size_2_gloo():
+    ctx = mp.get_context("spawn")
+    out = ctx.Manager().dict()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    for r in range(2):
+        value, ms = out[r]
+        assert ms == 20.0
+        assert abs(value - 2 * 128 / 0.020) < 1e-6
+
+
+def test_single_rank_aggregation_is_identity():
+    sys.path.insert(0, ROOT)
+    import bench
+    value, ms = bench.aggregate_replicas(4.0, 128, 1, "cpu")
+    assert ms == 4.0 and abs(value - 32000.0) < 1e-9
+
+
+def _run_bench(extra_env, *args):
+    env = dict(os.environ, **extra_env)
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], env=env,
+                          capture_output=True, text=True, timeout=600)
+
+
+def test_reference_arm_prints_one_json_line_with_the_contract_keys():
+    res = _run_bench({"RANK": "0", "WORLD_SIZE": "1"}, "--impl", "reference", "--workload", "tiny",
+                     "--steps", "3", "--warmup", "1")
+    assert res.returncode == 0, res.stderr
+    lines = [l for l in res.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["metric"] == "balanced_examples_per_sec"
+    assert d["unit"] == "examples/s" and d["higher_is_better"] is True
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
+    assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0,
+                        "d2h_bytes_per_step": 0}
+    assert d["config"]["workload"] == "tiny"
+
+
+def test_reference_arm_other_ranks_exit_quietly():
+    res = _run_bench({"RANK": "1", "WORLD_SIZE": "2"}, "--impl", "reference", "--workload", "tiny")
+    assert res.returncode == 0 and res.stdout.strip() == ""
+
+
+def test_algorithmic_bytes_model():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2302_00845_b200 import synth
+    wl = synth.WORKLOADS["gpt2"]
+    inp = 2 * 64 * 124_000_000 * 2
+    assert bench.algorithmic_bytes("gram", wl) == inp + 4 * 124_000_000
+    assert bench.algorithmic_bytes("update", wl) == inp + 8 * 124_000_000
+    assert inp == 31_744_000_000
