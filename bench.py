@@ -38,7 +38,11 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by kernel kind and workload; valid only while the kernel source hash matches.
-NCU_TRAFFIC: dict = {}
+NCU_TRAFFIC: dict = {
+    # captured at d = 8,000,000 (profiles/*_gpt2_d8m.md), scaled by d to a full-size launch
+    ("gram", "gpt2"): {"bytes": 2.105445e9 * 15.5, "source": "8fbf93204aa13d41"},
+    ("update", "gpt2"): {"bytes": 2.156762e9 * 15.5, "source": "8fbf93204aa13d41"},
+}
 
 
 def parse_args():
