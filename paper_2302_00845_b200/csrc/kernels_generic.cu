@@ -125,11 +125,11 @@ scan_kernel(const double *__restrict__ gram, int m, int n, int k,
             int8_t *__restrict__ signs, float *__restrict__ margins,
             double *__restrict__ rnorm2, int *__restrict__ status, int use_smem) {
   extern __shared__ double sh[];
-  double *tsh = sh;                                   // [m]
-  float *msh = reinterpret_cast<float *>(sh + m);     // [m] margins
-  int *ssh = reinterpret_cast<int *>(msh + m);        // [m] signs
+  double *tsh = sh;                                   // [m] t_j; entry i is final once worker i is decided
+  double *rnsh = sh + m;                              // [m] ||r||^2 seen by worker i
+  int *ssh = reinterpret_cast<int *>(sh + 2 * m);     // [m] signs
   int *psh = ssh + m;                                 // [2m] the current pair of every worker
-  double *gsh = sh + 3 * m;                           // [m][m] when use_smem (4m words = 2m doubles above)
+  double *gsh = sh + 4 * m;                           // [m][m] when use_smem (3m words above, padded)
   const int tid = threadIdx.x;
   const double *G = gram;
   const double *b = gram + (size_t)m * m;
@@ -155,11 +155,7 @@ scan_kernel(const double *__restrict__ gram, int m, int n, int k,
       bad |= !(isfinite(ti) && isfinite(gii));
       const double sd = (double)s;
       for (int j = i + 1 + lane; j < m; j += 32) tsh[j] += sd * G[(size_t)i * m + j];
-      if (lane == 0) {
-        ssh[i] = s;
-        const double den = rn2 * gii;
-        msh[i] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
-      }
+      if (lane == 0) { ssh[i] = s; rnsh[i] = rn2; }
       rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
       if (rn2 < 0.0) rn2 = 0.0;
       __syncwarp();
@@ -175,7 +171,8 @@ scan_kernel(const double *__restrict__ gram, int m, int n, int k,
     const int s = ssh[i];
     const size_t pos = (size_t)i * half + k;
     signs[pos] = (int8_t)s;
-    margins[pos] = msh[i];
+    const double den = rnsh[i] * G[(size_t)i * m + i];
+    margins[pos] = (den > 0.0) ? (float)(fabs(tsh[i]) / sqrt(den)) : 0.f;
     // Algorithm 7: the item that received +1 goes to the front slot, the other to the back
     const int32_t first = psh[2 * i], second = psh[2 * i + 1];
     perm_next[(size_t)i * n + k] = (s == 1) ? first : second;
@@ -384,7 +381,7 @@ cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream
 
 cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
   const int m = h->m;
-  const size_t small = (size_t)3 * m * sizeof(double);  // t, then margins/signs/pairs (4m words)
+  const size_t small = (size_t)4 * m * sizeof(double);  // t, ||r||^2, then signs/pairs (3m words, padded)
   const size_t with_g = small + (size_t)m * m * sizeof(double);
   const int use_smem = with_g <= 160 * 1024;
   const size_t smem = use_smem ? with_g : small;

@@ -265,39 +265,44 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   }
 }
 
-// G and b from the per-CTA partial H, summed over CTAs in index order in fp64.
-// thread e < m*m: (k, i) = (e / m, e % m);  m*m <= e < m*m + m: b_i
-__global__ void umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows,
-                                    int m, double *__restrict__ gram) {
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= m * m + m) return;
-  // CTAs taken four at a time with independent sums (loads stay in flight); fixed order
-  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+// G and b from the per-CTA partial H in fp64.  A block handles 32 consecutive entries
+// (e < m*m: (k, i) = (e / m, e % m);  m*m <= e < m*m + m: b_i); warp w sums the CTAs
+// w, w+8, w+16, ... in that order, the eight warp sums are then added in warp order.
+__global__ void __launch_bounds__(256)
+umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows, int m,
+                    double *__restrict__ gram) {
+  __shared__ double part[8][32];
+  const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+  const int total = m * m + m;
+  const int e = blockIdx.x * 32 + lane;
   const size_t cs = (size_t)128 * ncols;   // one CTA's partial H
+  double acc = 0.0;
   if (e < m * m) {
     const int k = e / m, i = e % m;
     const size_t o00 = (size_t)k * ncols + i, o01 = o00 + m, o10 = (size_t)(m + k) * ncols + i, o11 = o10 + m;
-    auto term = [&](int c) {
+#pragma unroll 4
+    for (int c = slice; c < ctas; c += 8) {
       const float *P = partials + (size_t)c * cs;
-      return ((double)P[o00] - (double)P[o01]) - ((double)P[o10] - (double)P[o11]);
-    };
-    int c = 0;
-    for (; c + 4 <= ctas; c += 4) { a0 += term(c); a1 += term(c + 1); a2 += term(c + 2); a3 += term(c + 3); }
-    for (; c < ctas; ++c) a0 += term(c);
-  } else {
+      acc += ((double)P[o00] - (double)P[o01]) - ((double)P[o10] - (double)P[o11]);
+    }
+  } else if (e < total) {
     const int i = e - m * m;
     const size_t o0 = (size_t)i * ncols + box_rows, o1 = (size_t)(m + i) * ncols + box_rows;
-    auto term = [&](int c) {
+#pragma unroll 4
+    for (int c = slice; c < ctas; c += 8) {
       const float *P = partials + (size_t)c * cs;
-      return (((double)P[o0] - (double)P[o1]) + ((double)P[o0 + 1] - (double)P[o1 + 1])) +
+      acc += (((double)P[o0] - (double)P[o1]) + ((double)P[o0 + 1] - (double)P[o1 + 1])) +
              ((double)P[o0 + 2] - (double)P[o1 + 2]);
-    };
-    int c = 0;
-    for (; c + 4 <= ctas; c += 4) { a0 += term(c); a1 += term(c + 1); a2 += term(c + 2); a3 += term(c + 3); }
-    for (; c < ctas; ++c) a0 += term(c);
+    }
   }
-  const double acc = (a0 + a1) + (a2 + a3);
-  gram[e] = acc;
+  part[slice][lane] = acc;
+  __syncthreads();
+  if (slice == 0 && e < total) {
+    double v = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) v += part[w][lane];
+    gram[e] = v;
+  }
 }
 
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
@@ -424,7 +429,7 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
     const int total = h->m * h->m + h->m;
-    umma_combine_kernel<<<(total + 127) / 128, 128, 0, st>>>(h->umma_partials, h->umma_ctas, h->umma_ncols,
+    umma_combine_kernel<<<(total + 31) / 32, 256, 0, st>>>(h->umma_partials, h->umma_ctas, h->umma_ncols,
                                                              h->umma_box_rows, h->m, h->gram);
   }
   return cudaGetLastError();
