@@ -26,6 +26,7 @@ void free_all(cdgrab_ctx *h) {
   cudaFree(h->r); cudaFree(h->perm_cur); cudaFree(h->perm_next); cudaFree(h->signs);
   cudaFree(h->margins); cudaFree(h->rnorm2); cudaFree(h->status); cudaFree(h->gram);
   cudaFree(h->partials);
+  cudaFree(h->ticket);
   if (h->prof_ev) {
     for (int i = 0; i < 2 * h->prof_cap; ++i) if (h->prof_ev[i]) cudaEventDestroy(h->prof_ev[i]);
     free(h->prof_ev);
@@ -124,6 +125,8 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
   ok = ok && cudaMalloc(&h->rnorm2, sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&h->status, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMalloc(&h->gram, sizeof(double) * ((size_t)m * m + m)) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->ticket, sizeof(unsigned)) == cudaSuccess;
+  ok = ok && cudaMemset(h->ticket, 0, sizeof(unsigned)) == cudaSuccess;
   if (ok && path == CDGRAB_PATH_FMA) {
     if (fma_columns_ok(h)) {
       // thread-per-column kernel: one partial vector (<= 152 doubles) per block
@@ -153,6 +156,14 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
   if (path == CDGRAB_PATH_UMMA) {
     const int rc = cdg_umma_setup(h);
     if (rc != CDGRAB_OK) { free_all(h); delete h; return rc; }
+  }
+  if (path == CDGRAB_PATH_FMA && fma_columns_ok(h) && cdg_fma_tma_supported(m, d, dtype)) {
+    // CDGRAB_FMA_TMA=0 keeps the load-from-registers Gram kernel (diagnostic knob)
+    const char *e = getenv("CDGRAB_FMA_TMA");
+    if (!(e && e[0] == '0')) {
+      const int rc = cdg_fma_tma_setup(h);
+      if (rc != CDGRAB_OK) { free_all(h); delete h; return rc; }
+    }
   }
 
   const long long tot = (long long)m * n;
@@ -234,9 +245,10 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
     e = cdg_launch_fused(h, grads_dev, st);
   } else {
     if (h->path == CDGRAB_PATH_UMMA) e = cdg_launch_gram_umma(h, grads_dev, st);
+    else if (h->fma_tma) e = cdg_launch_gram_fma_tma(h, grads_dev, st);
     else if (fma_columns_ok(h)) e = cdg_launch_gram_fma(h, grads_dev, st);
     else e = cdg_launch_gram_generic(h, grads_dev, st);
-    if (e == cudaSuccess) e = cdg_launch_scan(h, st);
+    if (e == cudaSuccess && !(h->fma_tma && h->fma_tma_fused)) e = cdg_launch_scan(h, st);
     if (e == cudaSuccess) e = cdg_launch_update(h, grads_dev, st);
   }
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }

@@ -42,6 +42,18 @@ struct cdgrab_ctx {
   size_t partials_bytes;
   int gram_chunks;       // grid.x of the FMA Gram kernels
 
+  // TMA-pipelined FMA Gram
+  int fma_tma;             // 1 when that kernel serves pass 1
+  int fma_tma_stages;
+  int fma_tma_boxrows;     // rows per bulk-tensor copy
+  int fma_tma_contig;      // 1: each CTA owns a contiguous range of tiles
+  int fma_tma_fused;       // 1: the last CTA of pass 1 also combines and decides (no scan launch)
+  unsigned *ticket;        // [1] arrival counter of that hand-over, zero between launches
+  size_t fma_tma_smem;
+  CUtensorMap tm_fr;       // 2-D map over r (one row)
+  const void *tm_fg_base;
+  CUtensorMap tm_fg;       // 2-D map over the gradient rows
+
   // optional per-kernel timing (cdgrab_profile_*): event pairs recorded around launches
   int prof_on;
   int prof_n, prof_cap;
@@ -97,6 +109,14 @@ cudaError_t cdg_launch_gram_fma(cdgrab_ctx *h, const void *grads, cudaStream_t s
 cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,
                               float *out, cudaStream_t st);
 bool cdg_fused_supported(int m, long long d, int dtype);
+
+// cuTensorMapEncodeTiled looked up through the runtime (NULL when the driver lacks it)
+void *cdg_tensor_map_encoder();
+
+// TMA-pipelined FMA Gram (m <= 16)
+bool cdg_fma_tma_supported(int m, long long d, int dtype);
+int cdg_fma_tma_setup(cdgrab_ctx *h);
+cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 
 // tcgen05 path
 bool cdg_umma_supported(int m, long long d, int dtype);

@@ -315,3 +315,376 @@ cudaError_t cdg_launch_gram_fma(cdgrab_ctx *h, const void *grads, cudaStream_t s
   if (M == 8) return launch_gram_fma_t<__nv_bfloat16, 8>(h, grads, st);
   return launch_gram_fma_t<__nv_bfloat16, 16>(h, grads, st);
 }
+
+// ------------------------------------------------------------------------------------
+// TMA-pipelined pass 1 for m <= 16 and long rows.
+//
+// The thread-per-column Gram above keeps ~250 registers per thread, so only 8 warps fit on
+// an SM and their own loads cannot cover the HBM latency.  Here the loads are taken off the
+// compute warps: warp 8 (one lane) streams tiles of [2m rows x 256 columns] plus the
+// matching 256 entries of r through a ring of shared-memory stages with bulk-tensor copies
+// and mbarriers; the 256 compute threads each own one column of the tile, read its 2m
+// values from shared memory (consecutive threads, consecutive words: no bank conflicts),
+// form c = z1 - z2 and feed the same register-resident triangle of accumulators.
+// Persistent CTAs take tiles blockIdx.x, blockIdx.x + gridDim.x, ...
+// Waits are bounded; on expiry the CTA raises the time-out bit and stops consuming.
+// ------------------------------------------------------------------------------------
+#include <stdlib.h>
+
+#include <type_traits>
+
+#include "ptx.cuh"
+#include "scan.cuh"
+
+constexpr int kFtCols = 256;       // columns per tile
+constexpr int kFtMaxStages = 8;
+constexpr int kFtThreads = 2 * kFtCols + 32;   // two compute groups + the producer warp
+
+template <typename T>
+__device__ __forceinline__ float ft_widen(T v);
+template <>
+__device__ __forceinline__ float ft_widen<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float ft_widen<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <int I, int N, typename F>
+__device__ __forceinline__ void static_for(F &&f) {
+  if constexpr (I < N) {
+    f(std::integral_constant<int, I>{});
+    static_for<I + 1, N>(f);
+  }
+}
+
+// The triangle of accumulators is shared out between two groups of 256 threads so that each
+// thread needs about half the registers and twice as many warps fit: pair (a, b) belongs to
+// group (a + b) & 1, the b-vector to group 1.  Local indices are compile-time constants.
+template <int M>
+struct Split {
+  __host__ __device__ static constexpr int owner(int a, int b) { return (a + b) & 1; }
+  __host__ __device__ static constexpr int count(int g) {
+    int n = 0;
+    for (int x = 0; x < M; ++x)
+      for (int y = x; y < M; ++y) n += owner(x, y) == g;
+    return n;
+  }
+  __host__ __device__ static constexpr int lidx(int a, int b) {
+    int n = 0;
+    for (int x = 0; x < M; ++x)
+      for (int y = x; y < M; ++y) {
+        if (x == a && y == b) return n;
+        n += owner(x, y) == owner(a, b);
+      }
+    return n;
+  }
+  static constexpr int N0 = count(0);
+  static constexpr int N1 = count(1) + M;       // odd pairs, then b
+  static constexpr int NL = N0 > N1 ? N0 : N1;
+  static constexpr int QL = (NL + 31) / 32;
+  static constexpr int NLPAD = 32 * QL;
+};
+
+template <typename T, int M, int G>
+__device__ __forceinline__ void ft_consume(const T *gt, const float *rt, int m, int col, float (&acc)[Split<M>::NLPAD]) {
+  float c[M];
+#pragma unroll
+  for (int i = 0; i < M; ++i) {
+    c[i] = 0.f;
+    if (i < m)   // c = z1 - z2; columns past d were zero-filled by the copy
+      c[i] = ft_widen<T>(gt[(size_t)i * kFtCols + col]) - ft_widen<T>(gt[(size_t)(m + i) * kFtCols + col]);
+  }
+  static_for<0, M>([&](auto A) {
+    static_for<A.value, M>([&](auto B) {
+      constexpr int a = A.value, b = B.value;
+      if constexpr (Split<M>::owner(a, b) == G) {
+        constexpr int l = Split<M>::lidx(a, b);
+        acc[l] = fmaf(c[a], c[b], acc[l]);
+      }
+    });
+  });
+  if constexpr (G == 1) {
+    const float rv = rt[col];
+    static_for<0, M>([&](auto A) {
+      constexpr int l = Split<M>::count(1) + A.value;
+      acc[l] = fmaf(rv, c[A.value], acc[l]);
+    });
+  }
+}
+
+// When enabled, the last CTA to finish also runs the scalar part of the step.
+struct FtTail {
+  int enabled;
+  int n, k;
+  unsigned *ticket;          // zero between launches
+  const int32_t *perm_cur;
+  int32_t *perm_next;
+  int8_t *signs;
+  float *margins;
+  double *rnorm2;
+};
+
+template <typename T, int M>
+__global__ void __launch_bounds__(kFtThreads, 1)
+gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
+                    int m, long long d, int stages, int box_rows, int contiguous,
+                    double *__restrict__ partials, int *__restrict__ status, const FtTail tail) {
+  extern __shared__ uint8_t ft_smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[kFtMaxStages];
+  __shared__ __align__(8) uint64_t bar_empty[kFtMaxStages];
+  __shared__ double red[16 * Split<M>::NLPAD];      // [warp][local entry]
+  __shared__ short lmap[2][Split<M>::NLPAD];        // local entry -> entry of the full triangle (-1: padding)
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group = warp >> 3;                       // 0, 1: compute groups; 2: producer
+  const uint32_t base = (smem_u32(ft_smem_raw) + 127u) & ~127u;
+  uint8_t *base_ptr = ft_smem_raw + (base - smem_u32(ft_smem_raw));
+  const int nbox = (2 * m + box_rows - 1) / box_rows;             // row boxes per tile
+  const uint32_t box_bytes = (uint32_t)box_rows * kFtCols * (uint32_t)sizeof(T);
+  const uint32_t g_bytes = (uint32_t)nbox * box_bytes;            // rows past 2m are zero-filled
+  const uint32_t stage_bytes = g_bytes + kFtCols * (uint32_t)sizeof(float);   // rows, then the r tile
+  const long long ntiles = (d + kFtCols - 1) / kFtCols;
+  // tiles of this CTA: a contiguous range, or every gridDim.x-th tile
+  const long long t_lo = contiguous ? ntiles * blockIdx.x / gridDim.x : blockIdx.x;
+  const long long t_hi = contiguous ? ntiles * (blockIdx.x + 1) / gridDim.x : ntiles;
+  const long long t_step = contiguous ? 1 : gridDim.x;
+  const int n_iter = (int)((t_hi - t_lo + t_step - 1) / t_step);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 16);  // one arrival per compute warp
+    }
+    mbar_init_fence();
+  }
+  if (threadIdx.x < 2 * Split<M>::NLPAD) (&lmap[0][0])[threadIdx.x] = -1;
+  __syncthreads();
+  if (threadIdx.x < Tri<M>::NACC) {
+    // entry e of the triangle -> (group, local index): count the same-group entries before it
+    const int e = threadIdx.x;
+    if (e < Tri<M>::NPAIR) {
+      int a = 0, rem = e;
+      while (rem >= M - a) { rem -= M - a; ++a; }
+      const int b = a + rem, g = Split<M>::owner(a, b);
+      int l = 0;
+      for (int x = 0; x < M; ++x)
+        for (int y = x; y < M; ++y)
+          if ((x < a || (x == a && y < b)) && Split<M>::owner(x, y) == g) ++l;
+      lmap[g][l] = (short)e;
+    } else {
+      lmap[1][Split<M>::count(1) + (e - Tri<M>::NPAIR)] = (short)e;
+    }
+  }
+  __syncthreads();
+  const long long deadline = clock64() + kCdgWaitCycles;
+
+  float acc[Split<M>::NLPAD];
+#pragma unroll
+  for (int e = 0; e < Split<M>::NLPAD; ++e) acc[e] = 0.f;
+
+  if (group == 2) {
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int it = 0; it < n_iter; ++it) {
+        const int s = it % stages;
+        if (it >= stages) ok = mbar_wait(smem_u32(&bar_empty[s]), ((it / stages) - 1) & 1, deadline);
+        if (!ok) break;
+        const long long tile = t_lo + (long long)it * t_step;
+        const int col = (int)(tile * kFtCols);            // 256 elements: 16-byte aligned for both types
+        const uint32_t full = smem_u32(&bar_full[s]);
+        const uint32_t dst = base + s * stage_bytes;
+        mbar_expect_tx(full, stage_bytes);
+        for (int q = 0; q < nbox; ++q) tma_load_2d(dst + q * box_bytes, &tm_g, col, q * box_rows, full);
+        tma_load_2d(dst + g_bytes, &tm_r, col, 0, full);
+        issued = it + 1;
+      }
+      if (!ok) {
+        atomicOr(status, CDG_ST_TIMEOUT);
+        for (int it = max(0, issued - stages); it < issued; ++it)
+          mbar_wait(smem_u32(&bar_full[it % stages]), (it / stages) & 1, clock64() + kCdgWaitCycles);
+      }
+    }
+  } else {
+    const int col = threadIdx.x & (kFtCols - 1);
+    bool ok = true;
+    for (int it = 0; it < n_iter && ok; ++it) {
+      const int s = it % stages;
+      ok = mbar_wait(smem_u32(&bar_full[s]), (it / stages) & 1, deadline);
+      if (!ok) break;
+      const T *gt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes);
+      const float *rt = reinterpret_cast<const float *>(base_ptr + (size_t)s * stage_bytes + g_bytes);
+      if (group == 0) ft_consume<T, M, 0>(gt, rt, m, col, acc);
+      else ft_consume<T, M, 1>(gt, rt, m, col, acc);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));   // this warp is done with the stage
+    }
+    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+    // warp totals of the local entries, as doubles
+    warp_reduce_vec<Split<M>::NLPAD>(acc, lane);
+#pragma unroll
+    for (int q = 0; q < Split<M>::QL; ++q)
+      red[warp * Split<M>::NLPAD + q + Split<M>::QL * lane] = (double)acc[q];
+  }
+  __syncthreads();
+  // thread (g, l): add the 8 warps of group g in warp order, store under the triangle's entry
+  if (threadIdx.x < 2 * Split<M>::NLPAD) {
+    const int g = threadIdx.x / Split<M>::NLPAD, l = threadIdx.x % Split<M>::NLPAD;
+    const int e = lmap[g][l];
+    if (e >= 0) {
+      double v = 0.0;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) v += red[(g * 8 + w) * Split<M>::NLPAD + l];
+      partials[(size_t)blockIdx.x * Tri<M>::NACC + e] = v;
+    }
+  }
+  if (!tail.enabled) return;
+
+  // ---- the CTA that takes the last ticket finishes the step: combine, decide, write ----
+  // (no waiting: a CTA either is last and sees every partial, or leaves)
+  __shared__ int is_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned t = atomicAdd(tail.ticket, 1u);
+    is_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // the stage ring is idle now; reuse it (all copies were consumed before the partials went out)
+  double *sh = reinterpret_cast<double *>(base_ptr);
+  const ScanSmem S = scan_smem(sh, m);
+  double *slices = S.g + (size_t)m * m;                       // [3][NPAD] block-list slices
+  constexpr int NP = Tri<M>::NPAD;
+  if (threadIdx.x < 3 * NP) {
+    // slice p adds blocks p, p+3, ... in that order; the slices are then added in order
+    const int e = threadIdx.x % NP, p = threadIdx.x / NP;
+    double v = 0.0;
+    if (e < Tri<M>::NACC)
+      for (int b = p; b < (int)gridDim.x; b += 3) v += __ldcg(partials + (size_t)b * Tri<M>::NACC + e);
+    slices[p * NP + e] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < Tri<M>::NACC) {
+    const int e = threadIdx.x;
+    const double v = (slices[e] + slices[NP + e]) + slices[2 * NP + e];
+    if (e < Tri<M>::NPAIR) {
+      int a = 0, rem = e;
+      while (rem >= M - a) { rem -= M - a; ++a; }
+      const int b = a + rem;
+      if (a < m && b < m) { S.g[a * m + b] = v; S.g[b * m + a] = v; }
+    } else {
+      const int a = e - Tri<M>::NPAIR;
+      if (a < m) S.t[a] = v;
+    }
+  }
+  scan_load_pairs(S, tail.perm_cur, m, tail.n, tail.k);
+  if (threadIdx.x == 0) *tail.ticket = 0u;                    // ready for the next launch
+  __syncthreads();
+  scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status);
+}
+
+bool cdg_fma_tma_supported(int m, long long d, int dtype) {
+  const int align = (dtype == CDGRAB_F32) ? 4 : 8;   // row pitch must be a multiple of 16 bytes
+  return m <= 16 && d % align == 0 && d >= 65536 && cdg_tensor_map_encoder() != nullptr;
+}
+
+static bool ft_encode(CUtensorMap *map, const void *base, long long d, int rows, int box_rows, int elem_bytes) {
+  typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                               const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  EncodeFn fn = (EncodeFn)cdg_tensor_map_encoder();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)d * elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)kFtCols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE,
+            getenv("CDGRAB_FT_L2P") ? (CUtensorMapL2promotion)atoi(getenv("CDGRAB_FT_L2P")) : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename T, int M>
+static cudaError_t ft_set_smem(size_t smem) {
+  return cudaFuncSetAttribute(gram_fma_tma_kernel<T, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+int cdg_fma_tma_setup(cdgrab_ctx *h) {
+  const size_t esz = h->dtype == CDGRAB_F32 ? 4 : 2;
+  int box_rows = 8;   // few distinct rows per copy keeps the far-apart rows' pages local
+  if (const char *e = getenv("CDGRAB_FT_BOXROWS")) {
+    const int v = atoi(e);
+    if (v >= 1 && v <= 32) box_rows = v;
+  }
+  h->fma_tma_boxrows = box_rows;
+  h->fma_tma_contig = 1;
+  h->fma_tma_fused = 1;      // CDGRAB_FT_FUSE_TAIL=0: separate combine and scan launches
+  if (const char *e = getenv("CDGRAB_FT_FUSE_TAIL")) h->fma_tma_fused = atoi(e) ? 1 : 0;
+  if (const char *e = getenv("CDGRAB_FT_CONTIG")) h->fma_tma_contig = atoi(e) ? 1 : 0;
+  const int nbox = (2 * h->m + box_rows - 1) / box_rows;
+  const size_t stage = (size_t)nbox * box_rows * kFtCols * esz + kFtCols * sizeof(float);
+  int stages = (int)((200 * 1024) / stage);
+  if (const char *e = getenv("CDGRAB_FT_STAGES")) {
+    const int v = atoi(e);
+    if (v >= 2 && v < stages) stages = v;
+  }
+  if (stages > kFtMaxStages) stages = kFtMaxStages;
+  if (stages < 2) return CDGRAB_ERR_INVALID;
+  h->fma_tma_stages = stages;
+  h->fma_tma_smem = stages * stage + 128;
+  const long long ntiles = (h->d + kFtCols - 1) / kFtCols;
+  h->gram_chunks = (int)(ntiles < h->num_sms ? ntiles : h->num_sms);
+  if (!ft_encode(&h->tm_fr, h->r, h->d, 1, 1, 4)) return CDGRAB_ERR_CUDA;
+  const int M = pick_M(h->m);
+  cudaError_t e;
+  if (h->dtype == CDGRAB_F32)
+    e = M == 4 ? ft_set_smem<float, 4>(h->fma_tma_smem) : M == 8 ? ft_set_smem<float, 8>(h->fma_tma_smem)
+                                                                  : ft_set_smem<float, 16>(h->fma_tma_smem);
+  else
+    e = M == 4 ? ft_set_smem<__nv_bfloat16, 4>(h->fma_tma_smem)
+               : M == 8 ? ft_set_smem<__nv_bfloat16, 8>(h->fma_tma_smem)
+                        : ft_set_smem<__nv_bfloat16, 16>(h->fma_tma_smem);
+  if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->tm_fg_base = nullptr;
+  h->fma_tma = 1;
+  return CDGRAB_OK;
+}
+
+template <typename T, int M>
+static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, cudaStream_t st) {
+  FtTail tail;
+  tail.enabled = h->fma_tma_fused;
+  tail.n = h->n; tail.k = h->k;
+  tail.ticket = h->ticket;
+  tail.perm_cur = h->perm_cur; tail.perm_next = h->perm_next;
+  tail.signs = h->signs; tail.margins = h->margins; tail.rnorm2 = h->rnorm2;
+  {
+    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
+    gram_fma_tma_kernel<T, M><<<h->gram_chunks, kFtThreads, h->fma_tma_smem, st>>>(
+        h->tm_fg, h->tm_fr, h->m, h->d, h->fma_tma_stages, h->fma_tma_boxrows, h->fma_tma_contig, h->partials,
+        h->status, tail);
+  }
+  if (!h->fma_tma_fused) {
+    CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
+    fma_combine_kernel<M><<<1, 6 * Tri<M>::NPAD, 0, st>>>(h->partials, h->gram_chunks, h->m, h->gram);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  if (grads != h->tm_fg_base) {
+    if (!ft_encode(&h->tm_fg, grads, h->d, 2 * h->m, h->fma_tma_boxrows, h->dtype == CDGRAB_F32 ? 4 : 2))
+      return cudaErrorInvalidValue;
+    h->tm_fg_base = grads;
+  }
+  const int M = pick_M(h->m);
+  if (h->dtype == CDGRAB_F32) {
+    if (M == 4) return launch_gram_fma_tma_t<float, 4>(h, st);
+    if (M == 8) return launch_gram_fma_tma_t<float, 8>(h, st);
+    return launch_gram_fma_tma_t<float, 16>(h, st);
+  }
+  if (M == 4) return launch_gram_fma_tma_t<__nv_bfloat16, 4>(h, st);
+  if (M == 8) return launch_gram_fma_tma_t<__nv_bfloat16, 8>(h, st);
+  return launch_gram_fma_tma_t<__nv_bfloat16, 16>(h, st);
+}

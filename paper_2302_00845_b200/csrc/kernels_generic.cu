@@ -12,6 +12,7 @@
 // which is exact in real arithmetic and lets the d-sized work be done in two streaming
 // passes instead of 2m dependent sweeps.
 #include "common.cuh"
+#include "scan.cuh"
 
 // ------------------------------------------------------------------------------------
 // pass 1 (generic): register-tiled Gram on FMA units
@@ -125,59 +126,16 @@ scan_kernel(const double *__restrict__ gram, int m, int n, int k,
             int8_t *__restrict__ signs, float *__restrict__ margins,
             double *__restrict__ rnorm2, int *__restrict__ status, int use_smem) {
   extern __shared__ double sh[];
-  double *tsh = sh;                                   // [m] t_j; entry i is final once worker i is decided
-  double *rnsh = sh + m;                              // [m] ||r||^2 seen by worker i
-  int *ssh = reinterpret_cast<int *>(sh + 2 * m);     // [m] signs
-  int *psh = ssh + m;                                 // [2m] the current pair of every worker
-  double *gsh = sh + 4 * m;                           // [m][m] when use_smem (3m words above, padded)
-  const int tid = threadIdx.x;
+  const ScanSmem S = scan_smem(sh, m);
   const double *G = gram;
-  const double *b = gram + (size_t)m * m;
-  for (int j = tid; j < m; j += blockDim.x) {
-    tsh[j] = b[j];
-    psh[2 * j] = perm_cur[(size_t)j * n + 2 * k];
-    psh[2 * j + 1] = perm_cur[(size_t)j * n + 2 * k + 1];
-  }
+  for (int j = threadIdx.x; j < m; j += blockDim.x) S.t[j] = gram[(size_t)m * m + j];
   if (use_smem) {
-    for (int e = tid; e < m * m; e += blockDim.x) gsh[e] = G[e];
-    G = gsh;
+    for (int e = threadIdx.x; e < m * m; e += blockDim.x) S.g[e] = gram[e];
+    G = S.g;
   }
+  scan_load_pairs(S, perm_cur, m, n, k);
   __syncthreads();
-  if (tid < 32) {
-    const int lane = tid;
-    double rn2 = *rnorm2;
-    bool bad = false;
-    for (int i = 0; i < m; ++i) {
-      const double ti = tsh[i];
-      const double gii = G[(size_t)i * m + i];
-      // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0; a tie gives -1
-      const int s = (ti < 0.0) ? 1 : -1;
-      bad |= !(isfinite(ti) && isfinite(gii));
-      const double sd = (double)s;
-      for (int j = i + 1 + lane; j < m; j += 32) tsh[j] += sd * G[(size_t)i * m + j];
-      if (lane == 0) { ssh[i] = s; rnsh[i] = rn2; }
-      rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
-      if (rn2 < 0.0) rn2 = 0.0;
-      __syncwarp();
-    }
-    if (lane == 0) {
-      *rnorm2 = rn2;
-      if (bad) atomicOr(status, CDG_ST_NONFINITE);
-    }
-  }
-  __syncthreads();
-  const int half = n >> 1;
-  for (int i = tid; i < m; i += blockDim.x) {
-    const int s = ssh[i];
-    const size_t pos = (size_t)i * half + k;
-    signs[pos] = (int8_t)s;
-    const double den = rnsh[i] * G[(size_t)i * m + i];
-    margins[pos] = (den > 0.0) ? (float)(fabs(tsh[i]) / sqrt(den)) : 0.f;
-    // Algorithm 7: the item that received +1 goes to the front slot, the other to the back
-    const int32_t first = psh[2 * i], second = psh[2 * i + 1];
-    perm_next[(size_t)i * n + k] = (s == 1) ? first : second;
-    perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;
-  }
+  scan_decide_and_write(S, G, m, n, k, perm_next, signs, margins, rnorm2, status);
 }
 
 // ------------------------------------------------------------------------------------
@@ -381,8 +339,8 @@ cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream
 
 cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
   const int m = h->m;
-  const size_t small = (size_t)4 * m * sizeof(double);  // t, ||r||^2, then signs/pairs (3m words, padded)
-  const size_t with_g = small + (size_t)m * m * sizeof(double);
+  const size_t small = scan_smem_bytes(m, false);
+  const size_t with_g = scan_smem_bytes(m, true);
   const int use_smem = with_g <= 160 * 1024;
   const size_t smem = use_smem ? with_g : small;
   static bool attr_set = false;

@@ -28,6 +28,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace {
 
@@ -35,7 +36,7 @@ constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr int kSubCols = 64;             // bf16 columns per TMA box = one 128-byte swizzle row
 constexpr int kRBoxRows = 16;
-constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
+constexpr long long kWaitCycles = kCdgWaitCycles;
 
 struct UmmaParams {
   int box_rows;        // gradient rows held per block (2m rounded up to 16)
@@ -46,41 +47,6 @@ struct UmmaParams {
   long long nblk_full; // d / 64: blocks loaded by the 3-D maps
   int tail;            // 1 when d % 64 != 0: one more, ragged block
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// bounded wait; false when the deadline passed
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long deadline) {
-  while (true) {
-    uint32_t done;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    if (done) return true;
-    if (clock64() > deadline) return false;
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
 
 // K-major, 128-byte swizzle: rows 128 B apart, 8-row groups `sbo` bytes apart
 __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t sbo) {
@@ -132,7 +98,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
     mbar_init(smem_u32(&bar_accum), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
   }
   // row groups that are never loaded (gradient groups wholly past row 2m, and the padding
   // group after the r rows) are zeroed once
@@ -349,6 +315,8 @@ bool encode_map_3d(CUtensorMap *map, const void *base, long long nblk, int rows,
 }
 
 }  // namespace
+
+void *cdg_tensor_map_encoder() { return (void *)encode_fn(); }
 
 bool cdg_umma_supported(int m, long long d, int dtype) {
   // bf16 rows whose pitch is a multiple of 16 bytes; 2m rows fit one 128-row MMA tile

@@ -1,0 +1,83 @@
+// The scalar part of a balancing step, shared by the stand-alone scan kernel and by Gram
+// kernels that finish the step themselves: m sequential sign decisions (Algorithm 6) on
+//   t_i = b_i + sum_{k<i} s_k G_ki
+// and the two permutation slots per worker (Algorithm 7).  Block-wide routines: every thread
+// of the block must call them; shared memory is handed in by the caller.
+#pragma once
+
+#include "common.cuh"
+
+struct ScanSmem {
+  double *t;     // [m]  starts as b; entry i is <r_{i-1}, c_i> once worker i is decided
+  double *rn;    // [m]  ||r||^2 seen by worker i
+  int *s;        // [m]  signs
+  int *p;        // [2m] the current pair of every worker
+  double *g;     // [m][m] optional copy of G
+};
+
+// (4m + m*m) doubles
+__device__ __forceinline__ ScanSmem scan_smem(double *sh, int m) {
+  ScanSmem S;
+  S.t = sh;
+  S.rn = sh + m;
+  S.s = reinterpret_cast<int *>(sh + 2 * m);
+  S.p = S.s + m;
+  S.g = sh + 4 * m;
+  return S;
+}
+__host__ __device__ inline size_t scan_smem_bytes(int m, bool with_g) {
+  return ((size_t)4 * m + (with_g ? (size_t)m * m : 0)) * sizeof(double);
+}
+
+__device__ __forceinline__ void scan_load_pairs(const ScanSmem &S, const int32_t *__restrict__ perm_cur, int m,
+                                                int n, int k) {
+  for (int j = threadIdx.x; j < m; j += blockDim.x) {
+    S.p[2 * j] = perm_cur[(size_t)j * n + 2 * k];
+    S.p[2 * j + 1] = perm_cur[(size_t)j * n + 2 * k + 1];
+  }
+}
+
+// S.t = b, S.p = pairs and G (shared or global, row-major [m][m]) must be ready and visible
+// to the block (barrier before the call).  Warp 0 decides, the block writes out.
+__device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const double *G, int m, int n, int k,
+                                                      int32_t *__restrict__ perm_next, int8_t *__restrict__ signs,
+                                                      float *__restrict__ margins, double *__restrict__ rnorm2,
+                                                      int *__restrict__ status) {
+  const int tid = threadIdx.x;
+  if (tid < 32) {
+    const int lane = tid;
+    double rn2 = *rnorm2;
+    bool bad = false;
+    for (int i = 0; i < m; ++i) {
+      const double ti = S.t[i];
+      const double gii = G[(size_t)i * m + i];
+      // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0; a tie gives -1
+      const int s = (ti < 0.0) ? 1 : -1;
+      bad |= !(isfinite(ti) && isfinite(gii));
+      const double sd = (double)s;
+      // every later t_j gains s_i G_ij, summed in the order i = 0, 1, ...
+      for (int j = i + 1 + lane; j < m; j += 32) S.t[j] += sd * G[(size_t)i * m + j];
+      if (lane == 0) { S.s[i] = s; S.rn[i] = rn2; }
+      rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
+      if (rn2 < 0.0) rn2 = 0.0;
+      __syncwarp();
+    }
+    if (lane == 0) {
+      *rnorm2 = rn2;
+      if (bad) atomicOr(status, CDG_ST_NONFINITE);
+    }
+  }
+  __syncthreads();
+  const int half = n >> 1;
+  for (int i = tid; i < m; i += blockDim.x) {
+    const int s = S.s[i];
+    const size_t pos = (size_t)i * half + k;
+    signs[pos] = (int8_t)s;
+    const double den = S.rn[i] * G[(size_t)i * m + i];
+    margins[pos] = (den > 0.0) ? (float)(fabs(S.t[i]) / sqrt(den)) : 0.f;
+    // Algorithm 7: the item that received +1 goes to the front slot, the other to the back
+    const int32_t first = S.p[2 * i], second = S.p[2 * i + 1];
+    perm_next[(size_t)i * n + k] = (s == 1) ? first : second;
+    perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;
+  }
+}

@@ -267,3 +267,29 @@ def test_step_host_matches_step():
             torch.cuda.synchronize()
         assert torch.equal(a.signs(), b.signs())
         assert torch.equal(a.r(), b.r())
+
+
+@pytest.mark.parametrize("m,d,dtype", [(16, 65536 * 5 + 4 * 33, "f32"), (7, 148 * 256 * 3, "f32"),
+                                       (12, 70_000 + 8 * 11, "bf16"), (3, 65536 * 3, "bf16")])
+def test_tma_pipelined_fma_gram(m, d, dtype):
+    """Long rows with m <= 16: pass 1 runs the TMA-fed FMA kernel (several ring turns per CTA,
+    ragged last tile); the same shapes with that kernel switched off must agree."""
+    rep = run_random_epoch(m, 6, d, dtype, seed=m + 3)
+    assert rep.path == "fma"
+    print(f"tma-fma m={m} d={d} {dtype}:", rep)
+
+
+def test_tma_fma_gram_matches_register_kernel(monkeypatch):
+    m, n, d = 16, 4, 1_000_000
+    out = []
+    for knob in ("1", "0"):
+        monkeypatch.setenv("CDGRAB_FMA_TMA", knob)
+        with binding.CdGrab(m, n, d, "f32") as h:
+            h.begin_epoch()
+            for k in range(n // 2):
+                h.step(random_grads(m, d, "f32", 900 + k, mean=0.1))
+            out.append((h.signs().cpu(), h.r().cpu(), h.margins().cpu()))
+            assert h.status() == binding.OK
+    assert torch.equal(out[0][0], out[1][0])
+    assert torch.equal(out[0][1], out[1][1])
+    np.testing.assert_allclose(out[0][2].numpy(), out[1][2].numpy(), rtol=1e-4, atol=1e-7)

@@ -26,7 +26,8 @@ def _grads(m, d, dtype, seed):
 @pytest.mark.parametrize("m,d,dtype", [(8, 65536 + 12, torch.float32), (16, 300_000, torch.float32),
                                        (3, 4096, torch.bfloat16)])
 def test_two_calls_match_the_handle_based_step(m, d, dtype, monkeypatch):
-    monkeypatch.setenv("CDGRAB_FORCE_PATH", "fma")   # the handle runs the same two-pass kernels
+    monkeypatch.setenv("CDGRAB_FORCE_PATH", "fma")   # the handle runs the same two-pass kernels,
+    monkeypatch.setenv("CDGRAB_FMA_TMA", "0")        # with the same summation order in pass 1
     steps = [_grads(m, d, dtype, 7 * m + k) for k in range(2)]
     name = "f32" if dtype == torch.float32 else "bf16"
     with binding.CdGrab(m, 4, d, name) as h:
