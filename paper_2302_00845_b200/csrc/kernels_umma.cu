@@ -327,8 +327,11 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   const int box_rows = ((2 * h->m + 15) / 16) * 16;
   h->umma_box_rows = box_rows;
   h->umma_ncols = box_rows + kRBoxRows;
-  int subs = 4;
-  if (const char *e = getenv("CDGRAB_UMMA_SUBS")) {   // tuning knob: 64-column blocks per stage
+  // 64-column blocks per stage: stages of roughly 70-80 KB measured best (4 blocks at m = 64,
+  // 6-8 at m = 32); CDGRAB_UMMA_SUBS overrides
+  int subs = 76 / (h->umma_ncols / 8);
+  subs = subs < 2 ? 2 : (subs > 8 ? 8 : subs);
+  if (const char *e = getenv("CDGRAB_UMMA_SUBS")) {
     const int v = atoi(e);
     if (v >= 1 && v <= 8) subs = v;
   }
