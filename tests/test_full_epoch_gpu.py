@@ -1,0 +1,72 @@
+"""Whole-epoch parity at the full sizes of the large workloads (opt-in: several minutes each).
+
+Run with CDGRAB_LONG_TESTS=1.  Every step of one epoch is balanced on the GPU (through the C
+ABI) and replayed by the CPU oracle on the same bytes, streamed to the host through a pinned
+buffer one worker pair at a time; signs (outside the tie band), the final running sum and the
+next-epoch permutations are compared."""
+import os
+import time
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import PairBalanceOracle
+from paper_2302_00845_b200 import binding, synth
+from parity import TAU, R_TOL, rel_l2
+
+pytestmark = [pytest.mark.gpu, pytest.mark.slow,
+              pytest.mark.skipif(os.environ.get("CDGRAB_LONG_TESTS") != "1",
+                                 reason="set CDGRAB_LONG_TESTS=1 to run whole epochs at full size")]
+
+
+def run_epoch(name):
+    wl = synth.WORKLOADS[name]
+    m, n, d = wl.m, wl.n, wl.d
+    gs = synth.GradientStream(wl, device="cuda")
+    gpu = binding.CdGrab(m, n, d, wl.dtype)
+    cpu = PairBalanceOracle(m, n, d)
+    pin = torch.empty(2, d, dtype=wl.torch_dtype, pin_memory=True)
+    view = pin.view(torch.int16).numpy().view(np.uint16) if wl.dtype == "bf16" else pin.numpy()
+    raw = 0
+    t0 = time.time()
+    try:
+        gpu.begin_epoch(); cpu.begin_epoch()
+        buf = None
+        for k in range(n // 2):
+            buf = gs.step(k, out=buf)
+            gpu.step(buf)
+            s = gpu.signs()[:, k].cpu().numpy()
+            for i in range(m):
+                pin[0].copy_(buf[0, i], non_blocking=True)
+                pin[1].copy_(buf[1, i], non_blocking=True)
+                torch.cuda.synchronize()
+                cpu.balance_one(i, view[0], view[1], replay=int(s[i]), tau=TAU[wl.dtype])
+            raw += int((cpu.own_signs()[:, k] == s).sum())
+        assert cpu.mismatches == 0
+        err = rel_l2(gpu.r().cpu().numpy().astype(np.float64), cpu.r())
+        assert err <= R_TOL[wl.dtype], err
+        out = torch.empty(m, n, dtype=torch.int32, device="cuda")
+        gpu.end_epoch(out)
+        torch.cuda.synchronize()
+        want = cpu.end_epoch()
+        assert np.array_equal(out.cpu().numpy(), want)
+        assert gpu.status() == binding.OK
+        marg = gpu.margins().cpu().numpy()
+        print(f"FULL EPOCH {name}: m={m} n={n} d={d} {wl.dtype} path={gpu.path} positions={m * n // 2} "
+              f"near_ties={cpu.near_ties} raw_agree={raw / (m * n // 2):.6f} r_rel_err={err:.3e} "
+              f"median_margin={np.median(marg):.3e} perms=bit-exact wall={time.time() - t0:.0f}s")
+    finally:
+        gpu.destroy(); cpu.close()
+
+
+def test_mid_full_epoch():
+    run_epoch("mid")
+
+
+def test_lstm_full_epoch():
+    run_epoch("lstm")
+
+
+def test_gpt2_full_epoch():
+    run_epoch("gpt2")
