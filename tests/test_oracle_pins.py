@@ -408,3 +408,48 @@ def test_logistic_gradient_matches_finite_differences():
             e = np.zeros(d); e[a] = 1e-6
             fd = (loss(w + e) - loss(w - e)) / 2e-6
             assert abs(fd - g[a]) < 1e-8
+
+
+# --------------------------------------------------------------------------------------
+# Parallel herding objective, Eq. (7): hand-computed examples and invariants.
+# --------------------------------------------------------------------------------------
+def load_herding_cases():
+    out = []
+    for line in open(os.path.join(GOLDEN, "herding_objective_examples.txt")):
+        if not line.startswith("case"):
+            continue
+        head, zs, ps, want = [t.strip() for t in line.split("|")]
+        _, name, m, n, d = head.split()
+        m, n, d = int(m), int(n), int(d)
+        z = np.array([float(v) for v in zs.split()]).reshape(m, n, d)
+        perms = np.array([int(v) for v in ps.split()]).reshape(m, n)
+        out.append((name, z, perms, float(want)))
+    return out
+
+
+def test_herding_objective_hand_examples():
+    cases = load_herding_cases()
+    assert len(cases) == 7
+    for name, z, perms, want in cases:
+        assert oracle.herding_objective(z, perms) == want, name
+
+
+def test_herding_objective_invariants():
+    rng = np.random.default_rng(21)
+    m, n, d = 3, 17, 5
+    z = rng.standard_normal((m, n, d))
+    perms = np.stack([rng.permutation(n) for _ in range(m)])
+    base = oracle.herding_objective(z, perms)
+    # cumulative-sum formulation with a library routine
+    zbar = z.reshape(-1, d).mean(axis=0)
+    steps = sum(z[i, perms[i]] for i in range(m)) - m * zbar            # [n][d]
+    assert abs(np.abs(np.cumsum(steps, axis=0)).max() - base) < 1e-12
+    # the centred vectors sum to zero, so walking every order backwards gives the same bound
+    assert abs(oracle.herding_objective(z, perms[:, ::-1]) - base) < 1e-12
+    # relabelling the workers changes nothing; a constant shift of all vectors changes nothing
+    assert abs(oracle.herding_objective(z[::-1], perms[::-1]) - base) < 1e-12
+    assert abs(oracle.herding_objective(z + 3.5, perms) - base) < 1e-10
+    # scaling scales the bound
+    assert abs(oracle.herding_objective(2 * z, perms) - 2 * base) < 1e-12
+    # identical vectors: nothing to balance
+    assert oracle.herding_objective(np.ones((2, 4, 3)), np.tile(np.arange(4), (2, 1))) == 0.0
