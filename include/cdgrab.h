@@ -194,6 +194,22 @@ int cdgrab_logreg_grads(cdgrab_t *h, const float *X, const float *y, const float
 int cdgrab_step_host(cdgrab_t *h, const void *grads_host, void *staging_dev, void *stream);
 
 /*
+ * Parallel herding objective, Eq. (7) of the paper -- the bound PairBalance is meant to shrink:
+ *   max over k in [n] of || sum_{j<=k} sum_{i<m} ( z[i][perms[i][j]] - zbar ) ||_inf ,
+ * zbar = mean of all m*n vectors.  Stand-alone (no handle), fp64 sums in a fixed order.
+ *   z_dev      DEVICE float [m][n][d], vectors indexed by item id
+ *   perms_dev  DEVICE int32 [m][n], row i = the order in which worker i visits its items
+ *   workspace_dev  DEVICE, 8-byte aligned, at least cdgrab_herding_workspace_bytes(m, n, d) bytes,
+ *              caller-owned scratch (contents undefined afterwards)
+ *   out_dev    DEVICE double [1], receives the objective
+ * Asynchronous on `stream`.  CDGRAB_ERR_INVALID for NULL pointers, non-positive sizes, a
+ * workspace that is too small or misaligned.
+ */
+long long cdgrab_herding_workspace_bytes(int m, int n, long long d);
+int cdgrab_herding_objective(const float *z_dev, const int32_t *perms_dev, int m, int n, long long d,
+                             void *workspace_dev, long long workspace_bytes, double *out_dev, void *stream);
+
+/*
  * One balancing step that allocates nothing (the paper has no counterpart: this is a
  * packaging of cdgrab_step for a restricted kind of caller).
  *

@@ -42,6 +42,9 @@ SIGNATURES = {
     "cdgrab_profile_read": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]),
     "cdgrab_logreg_grads": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_step_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_herding_workspace_bytes": (C.c_longlong, [C.c_int, C.c_int, C.c_longlong]),
+    "cdgrab_herding_objective": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_longlong, C.c_void_p,
+                                           C.c_longlong, C.c_void_p, C.c_void_p]),
     "cdgrab_step_noalloc": (C.c_int, [C.c_int, C.c_longlong, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p]),
 }
@@ -209,3 +212,15 @@ def step_noalloc(grads, r, signs_out, stream=None):
     code = F32 if grads.dtype == torch.float32 else BF16
     _check(lib().cdgrab_step_noalloc(m, d, code, _ptr(grads), _ptr(r), _ptr(signs_out), _stream_ptr(stream)),
            "cdgrab_step_noalloc")
+
+
+def herding_objective(z, perms, stream=None) -> float:
+    """Eq. (7) on the device: z CUDA float32 [m][n][d] (by item id), perms CUDA int32 [m][n]."""
+    import torch
+    m, n, d = (int(v) for v in z.shape)
+    nbytes = int(lib().cdgrab_herding_workspace_bytes(m, n, d))
+    ws = torch.empty(nbytes // 8, dtype=torch.float64, device=z.device)
+    out = torch.empty(1, dtype=torch.float64, device=z.device)
+    _check(lib().cdgrab_herding_objective(_ptr(z), _ptr(perms), m, n, d, _ptr(ws), nbytes, _ptr(out),
+                                          _stream_ptr(stream)), "cdgrab_herding_objective")
+    return float(out.item())
