@@ -108,6 +108,16 @@ int cdgrab_begin_epoch(cdgrab_t *h, void *stream);
 int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream);
 
 /*
+ * cdgrab_step that also returns what the paper's parameter server sends back to the workers
+ * (Algorithm 4, "compute avg. gradient ... send to all the workers"): the average of each of
+ * the two gather buffers, mean_out_dev[q][x] = (1/m) sum_i grads_dev[q][i][x] for q = 0, 1.
+ * mean_out_dev: DEVICE float [2][d], 16-byte aligned, caller-owned.  The rows are summed in
+ * fp32 in worker order while pass 2 has them in registers, so the average costs no extra read
+ * of the inputs.  Otherwise identical to cdgrab_step (same errors, same asynchrony).
+ */
+int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, void *stream);
+
+/*
  * Close the epoch after exactly n/2 steps (else CDGRAB_ERR_STATE): the next permutations
  * become the current ones (Algorithm 4, last lines of the epoch loop) and, if perms_out is
  * not NULL, are copied there.  perms_out: HOST or DEVICE pointer, int32 [m][n];

@@ -28,6 +28,7 @@ SIGNATURES = {
     "cdgrab_set_perms": (C.c_int, [C.c_void_p, C.c_void_p]),
     "cdgrab_begin_epoch": (C.c_int, [C.c_void_p, C.c_void_p]),
     "cdgrab_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_step_mean": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_end_epoch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_get_signs": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_get_r": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -134,6 +135,11 @@ class CdGrab:
     def step(self, grads, stream=None):
         """grads: CUDA tensor [2][m][d] of the handle's dtype."""
         _check(lib().cdgrab_step(self._h, _ptr(grads), _stream_ptr(stream)), "cdgrab_step")
+
+    def step_mean(self, grads, mean_out, stream=None):
+        """step() that also writes the average of each gather buffer into mean_out (CUDA float32 [2][d])."""
+        _check(lib().cdgrab_step_mean(self._h, _ptr(grads), _ptr(mean_out), _stream_ptr(stream)),
+               "cdgrab_step_mean")
 
     def step_host(self, grads_host, staging, stream=None):
         """grads_host: pinned host tensor [2][m][d]; staging: CUDA tensor of the same size."""

@@ -133,7 +133,9 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
       long long blocks = (d / 4 + 255) / 256;
       if (blocks > (long long)h->num_sms * 2) blocks = (long long)h->num_sms * 2;
       h->gram_chunks = (int)blocks;
-      h->partials_bytes = sizeof(double) * 152 * (size_t)blocks;
+      // sized for the larger of the two grids that may write it: this kernel's (<= 2 per SM)
+      // and the TMA-fed kernel's (one CTA per SM whatever the row length)
+      h->partials_bytes = sizeof(double) * 152 * (size_t)h->num_sms * 2;
     } else {
       const int ntile = (m + CDG_TM - 1) / CDG_TM;
       const int npairs = ntile * (ntile + 1) / 2;
@@ -254,6 +256,18 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   h->k++;
   return CDGRAB_OK;
+}
+
+int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, void *stream) {
+  if (!valid(h) || !mean_out_dev) return CDGRAB_ERR_INVALID;
+  h->mean_out = mean_out_dev;
+  int rc = cdgrab_step(h, grads_dev, stream);
+  if (rc == CDGRAB_OK && h->path == CDGRAB_PATH_FUSED) {
+    // the single-launch step has no separate pass 2 to fold the average into
+    if (cdg_launch_mean(h, grads_dev, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); rc = CDGRAB_ERR_CUDA; }
+  }
+  h->mean_out = nullptr;
+  return rc;
 }
 
 int cdgrab_step_host(cdgrab_t *h, const void *grads_host, void *staging_dev, void *stream) {

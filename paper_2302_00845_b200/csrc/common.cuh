@@ -39,6 +39,7 @@ struct cdgrab_ctx {
   int *status;           // [1] device status word
   double *gram;          // [m*m + m] G (row-major) then b
   double *partials;      // pass-1 partial sums
+  float *mean_out;       // [2][d] destination of the averaged gather buffers for the step being enqueued, or NULL
   size_t partials_bytes;
   int gram_chunks;       // grid.x of the FMA Gram kernels
 
@@ -104,6 +105,7 @@ struct CdgProfScope {
 cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st);
 cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_mean(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_gram_fma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,

@@ -201,11 +201,14 @@ struct VecLoad<__nv_bfloat16, 1> {
   }
 };
 
-template <typename T, typename AccT, int VEC, bool SPLIT>
+// MEAN: also write the parameter-server average of each gather buffer (Algorithm 4,
+// "compute avg. gradient"): mean_out[q][x] = (1/m) sum_i grads[q][i][x], from the rows already
+// in registers.
+template <typename T, typename AccT, int VEC, bool SPLIT, bool MEAN>
 __global__ void __launch_bounds__(256)
 update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__restrict__ signs,
               int sign_stride, int m, long long d, __nv_bfloat16 *__restrict__ r_split,
-              long long d_pad) {
+              long long d_pad, float *__restrict__ mean_out) {
   extern __shared__ float ssh[];  // [m] signs as +-1.0f
   for (int i = threadIdx.x; i < m; i += blockDim.x) ssh[i] = (float)signs[(size_t)i * sign_stride];
   __syncthreads();
@@ -228,6 +231,11 @@ update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__re
     }
 #pragma unroll
     for (int j = 0; j < VEC; ++j) acc[j] = (AccT)rv[j];
+    float sa[MEAN ? VEC : 1], sb[MEAN ? VEC : 1];
+    if constexpr (MEAN) {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) { sa[j] = 0.f; sb[j] = 0.f; }
+    }
 #pragma unroll 2
     for (int i = 0; i < m; ++i) {
       float a[VEC], b[VEC];
@@ -236,6 +244,28 @@ update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__re
       const float s = ssh[i];
 #pragma unroll
       for (int j = 0; j < VEC; ++j) acc[j] += (AccT)(s * (a[j] - b[j]));
+      if constexpr (MEAN) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) { sa[j] += a[j]; sb[j] += b[j]; }
+      }
+    }
+    if constexpr (MEAN) {
+      const float inv_m = 1.f / (float)m;
+      if constexpr (VEC % 4 == 0) {   // d is a multiple of VEC here: 16-byte aligned in both slabs
+#pragma unroll
+        for (int q = 0; q < VEC / 4; ++q) {
+          *reinterpret_cast<float4 *>(mean_out + x + 4 * q) =
+              make_float4(sa[4 * q] * inv_m, sa[4 * q + 1] * inv_m, sa[4 * q + 2] * inv_m, sa[4 * q + 3] * inv_m);
+          *reinterpret_cast<float4 *>(mean_out + (size_t)d + x + 4 * q) =
+              make_float4(sb[4 * q] * inv_m, sb[4 * q + 1] * inv_m, sb[4 * q + 2] * inv_m, sb[4 * q + 3] * inv_m);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+          mean_out[x + j] = sa[j] * inv_m;
+          mean_out[(size_t)d + x + j] = sb[j] * inv_m;
+        }
+      }
     }
 #pragma unroll
     for (int j = 0; j < VEC; ++j) rv[j] = (float)acc[j];
@@ -368,12 +398,20 @@ static void launch_update_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
   const size_t smem = (size_t)h->m * sizeof(float);
   const int8_t *sg = h->signs + h->k;
   CdgProfScope ps(h, CDGRAB_K_UPDATE, st);
-  if (h->r_split)
-    update_kernel<T, AccT, VEC, true><<<(unsigned)blocks, 256, smem, st>>>(
-        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad);
-  else
-    update_kernel<T, AccT, VEC, false><<<(unsigned)blocks, 256, smem, st>>>(
-        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0);
+  if (h->mean_out) {
+    if (h->r_split)
+      update_kernel<T, AccT, VEC, true, true><<<(unsigned)blocks, 256, smem, st>>>(
+          (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad, h->mean_out);
+    else
+      update_kernel<T, AccT, VEC, false, true><<<(unsigned)blocks, 256, smem, st>>>(
+          (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0, h->mean_out);
+  } else if (h->r_split) {
+    update_kernel<T, AccT, VEC, true, false><<<(unsigned)blocks, 256, smem, st>>>(
+        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad, nullptr);
+  } else {
+    update_kernel<T, AccT, VEC, false, false><<<(unsigned)blocks, 256, smem, st>>>(
+        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0, nullptr);
+  }
 }
 
 cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
@@ -387,6 +425,28 @@ cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st)
     else if (h->d % 8 == 0) launch_update_t<__nv_bfloat16, float, 8>(h, grads, st);
     else launch_update_t<__nv_bfloat16, float, 1>(h, grads, st);
   }
+  return cudaGetLastError();
+}
+
+// stand-alone average of both gather buffers (used where pass 2 is part of a fused kernel)
+template <typename T>
+__global__ void mean_kernel(const T *__restrict__ g, int m, long long d, float *__restrict__ mean_out) {
+  const long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (x >= 2 * d) return;
+  const int q = (int)(x / d);
+  const long long col = x % d;
+  float acc = 0.f;
+  for (int i = 0; i < m; ++i) acc += cdg_ld(g + ((size_t)q * m + i) * (size_t)d + col);
+  mean_out[x] = acc * (1.f / (float)m);
+}
+
+cudaError_t cdg_launch_mean(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  const unsigned blocks = (unsigned)((2 * h->d + 255) / 256);
+  CdgProfScope ps(h, CDGRAB_K_UPDATE, st);
+  if (h->dtype == CDGRAB_F32)
+    mean_kernel<float><<<blocks, 256, 0, st>>>((const float *)grads, h->m, h->d, h->mean_out);
+  else
+    mean_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16 *)grads, h->m, h->d, h->mean_out);
   return cudaGetLastError();
 }
 

@@ -293,3 +293,27 @@ def test_tma_fma_gram_matches_register_kernel(monkeypatch):
     assert torch.equal(out[0][0], out[1][0])
     assert torch.equal(out[0][1], out[1][1])
     np.testing.assert_allclose(out[0][2].numpy(), out[1][2].numpy(), rtol=1e-4, atol=1e-7)
+
+
+@pytest.mark.parametrize("m,d,dtype", [(16, 100_000, "f32"), (8, 65_536, "bf16"), (32, 50_048, "bf16")])
+def test_handles_side_by_side_do_not_disturb_each_other(m, d, dtype):
+    """Three handles of the same shape alive at once, stepped in turn on the same inputs: each
+    owns its scratch, so all must agree bit for bit (a scratch buffer sized for the wrong grid
+    once let one handle write into its neighbour's memory)."""
+    n = 6
+    hs = [binding.CdGrab(m, n, d, dtype) for _ in range(3)]
+    try:
+        for h in hs:
+            h.begin_epoch()
+        for k in range(n // 2):
+            g = random_grads(m, d, dtype, 7000 + k, mean=0.2)
+            for h in hs:
+                h.step(g)
+        ref = (hs[0].signs(), hs[0].r(), hs[0].margins())
+        assert float(ref[2].max()) > 0
+        for h in hs[1:]:
+            assert torch.equal(h.signs(), ref[0]) and torch.equal(h.r(), ref[1]) and torch.equal(h.margins(), ref[2])
+            assert h.status() == binding.OK
+    finally:
+        for h in hs:
+            h.destroy()
