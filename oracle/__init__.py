@@ -49,6 +49,10 @@ def _load():
         lib.cdo_begin_epoch.argtypes = [C.c_void_p]
         lib.cdo_balance_one.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int,
                                         C.c_int, C.c_double]
+        lib.cdo_balance_one_randomized.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int,
+                                                   C.c_double, C.c_double, C.c_int, C.c_double]
+        lib.cdo_out_of_bound.restype = C.c_longlong
+        lib.cdo_out_of_bound.argtypes = [C.c_void_p]
         lib.cdo_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_double]
         lib.cdo_end_epoch.argtypes = [C.c_void_p, C.c_void_p]
         for name in ("cdo_get_r", "cdo_get_signs", "cdo_get_own_signs", "cdo_get_perm_cur",
@@ -119,6 +123,31 @@ class PairBalanceOracle:
         if s == 0:
             raise RuntimeError("oracle: balance_one out of order or outside an epoch")
         return s
+
+    def balance_one_randomized(self, i: int, g_prev: np.ndarray, g_cur: np.ndarray, u: float, w: float,
+                               replay: int = 0, tau: float = 0.0) -> int:
+        """RandomizedBalance (Algorithm 2's subroutine with Algorithm 5's bound w) for worker i:
+        p = 1/2 - <r,c>/(2w), sign +1 iff u < p."""
+        gp, dt = _as_rows(g_prev)
+        gc, dt2 = _as_rows(g_cur)
+        assert dt == dt2 and gp.size == self.d and gc.size == self.d
+        s = _load().cdo_balance_one_randomized(self._h, i, gp.ctypes.data, gc.ctypes.data, dt, float(u),
+                                               float(w), int(replay), float(tau))
+        if s == 0:
+            raise RuntimeError("oracle: randomized balance out of order, outside an epoch, or w <= 0")
+        return s
+
+    def step_randomized(self, grads: np.ndarray, u: np.ndarray, w: float, replay: np.ndarray | None = None,
+                        tau: float = 0.0):
+        g, _ = _as_rows(grads)
+        assert g.shape == (2, self.m, self.d) and len(u) == self.m
+        for i in range(self.m):
+            self.balance_one_randomized(i, g[0, i], g[1, i], float(u[i]), w,
+                                        0 if replay is None else int(replay[i]), tau)
+
+    @property
+    def out_of_bound(self) -> int:
+        return int(_load().cdo_out_of_bound(self._h))
 
     def step(self, grads: np.ndarray, replay: np.ndarray | None = None, tau: float = 0.0):
         """grads: [2][m][d]; slab 0 holds the earlier vector of every worker's pair."""

@@ -30,6 +30,11 @@
  *     appends pi(j);
  *   - each worker's reorder sees only that worker's own signs.
  *
+ * A second rule is offered beside the greedy one: RandomizedBalance (Algorithm 2's subroutine,
+ * with the bound w of Algorithm 5), p = 1/2 - <r,c>/(2w), s = +1 with probability p.  The
+ * uniform draw is an input, so the oracle stays deterministic.  Algorithm 5's second stopping
+ * condition (||r||_inf > w) is not evaluated.
+ *
  * Replay mode (tolerance rule of the parity tests): when the caller hands in a sign
  * for a position and |t| <= tau * ||r|| * ||c||, the position is a near-tie, the
  * handed-in sign is adopted and counted; outside that band the oracle keeps its own
@@ -72,6 +77,7 @@ typedef struct {
   double *rn;         /* [m][n/2] ||r|| before the update */
   double *cn;         /* [m][n/2] ||c|| */
   long long near_ties, mismatches;
+  long long out_of_bound; /* randomized rule: positions with |<r,c>| > w */
 } cdo_t;
 
 static double widen(const void *p, long long x, int dtype) {
@@ -126,7 +132,7 @@ int cdo_begin_epoch(cdo_t *s) {
   if (!s || s->epoch_open) return -1;
   memset(s->r, 0, sizeof(double) * (size_t)s->d);
   s->k = 0; s->i_next = 0; s->epoch_open = 1;
-  s->near_ties = 0; s->mismatches = 0;
+  s->near_ties = 0; s->mismatches = 0; s->out_of_bound = 0;
   return 0;
 }
 
@@ -137,8 +143,8 @@ int cdo_begin_epoch(cdo_t *s) {
  * replay = 0: no replay; replay = +1/-1: sign seen elsewhere, adopted inside the tie
  * band given by tau.  Returns the adopted sign, or 0 on misuse.
  */
-int cdo_balance_one(cdo_t *s, int i, const void *g_prev, const void *g_cur, int dtype,
-                    int replay, double tau) {
+static int balance_core(cdo_t *s, int i, const void *g_prev, const void *g_cur, int dtype,
+                        int replay, double tau, int randomized, double u, double w) {
   if (!s || !s->epoch_open || i != s->i_next || s->k >= s->n / 2) return 0;
   const long long d = s->d;
   const long long nchunk = s->nchunk;
@@ -166,7 +172,25 @@ int cdo_balance_one(cdo_t *s, int i, const void *g_prev, const void *g_cur, int 
   int own = (t < 0.0) ? +1 : -1;
   int sgn = own;
   double rn = sqrt(rr), cn = sqrt(cc);
-  if (replay == 1 || replay == -1) {
+  if (randomized) {
+    /* Algorithm 2's subroutine with the bound w of Algorithm 5 made explicit:
+     * p = 1/2 - <r,c>/(2w); +1 with probability p, drawn as "u < p" from the uniform u handed in.
+     * |<r,c>| > w is where Algorithm 5 would stop; here p leaves [0,1], the draw becomes
+     * deterministic (and equal to the greedy sign) and the event is counted. */
+    const double p = 0.5 - t / (2.0 * w);
+    own = (u < p) ? +1 : -1;
+    sgn = own;
+    if (fabs(t) > w) s->out_of_bound++;
+    if (replay == 1 || replay == -1) {
+      /* an error dt in <r,c> moves p by dt/(2w): the tie band in terms of u - p */
+      if (fabs(u - p) > tau * rn * cn / (2.0 * w)) {
+        if (replay != own) s->mismatches++;
+      } else {
+        s->near_ties++;
+        sgn = replay;
+      }
+    }
+  } else if (replay == 1 || replay == -1) {
     if (fabs(t) > tau * rn * cn) {
       if (replay != own) s->mismatches++;
     } else {
@@ -192,6 +216,19 @@ int cdo_balance_one(cdo_t *s, int i, const void *g_prev, const void *g_cur, int 
   s->i_next++;
   if (s->i_next == s->m) { s->i_next = 0; s->k++; }
   return sgn;
+}
+
+int cdo_balance_one(cdo_t *s, int i, const void *g_prev, const void *g_cur, int dtype,
+                    int replay, double tau) {
+  return balance_core(s, i, g_prev, g_cur, dtype, replay, tau, 0, 0.0, 1.0);
+}
+
+/* RandomizedBalance for worker i: as cdo_balance_one, with the sign drawn from the uniform u
+ * in [0,1) and the bound w > 0. */
+int cdo_balance_one_randomized(cdo_t *s, int i, const void *g_prev, const void *g_cur, int dtype,
+                               double u, double w, int replay, double tau) {
+  if (!(w > 0.0)) return 0;
+  return balance_core(s, i, g_prev, g_cur, dtype, replay, tau, 1, u, w);
 }
 
 /*
@@ -233,6 +270,7 @@ void cdo_get_trace(const cdo_t *s, double *t, double *rn, double *cn) {
 }
 long long cdo_near_ties(const cdo_t *s) { return s->near_ties; }
 long long cdo_mismatches(const cdo_t *s) { return s->mismatches; }
+long long cdo_out_of_bound(const cdo_t *s) { return s->out_of_bound; }
 int cdo_pairs_done(const cdo_t *s) { return s->k; }
 int cdo_threads(void) {
 #ifdef _OPENMP

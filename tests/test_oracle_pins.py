@@ -453,3 +453,75 @@ def test_herding_objective_invariants():
     assert abs(oracle.herding_objective(2 * z, perms) - 2 * base) < 1e-12
     # identical vectors: nothing to balance
     assert oracle.herding_objective(np.ones((2, 4, 3)), np.tile(np.arange(4), (2, 1))) == 0.0
+
+
+# --------------------------------------------------------------------------------------
+# RandomizedBalance (Algorithm 2's subroutine with the bound w of Algorithm 5).
+# --------------------------------------------------------------------------------------
+def _rand_state(seed, d=40):
+    """An oracle whose running sum is r = z0 - z1 of a first (greedy) pair, plus a second pair."""
+    rng = np.random.default_rng(seed)
+    z = rng.standard_normal((1, 4, d)).astype(np.float32)
+    o = PairBalanceOracle(1, 4, d)
+    o.begin_epoch()
+    s0 = o.balance_one(0, z[0, 0], z[0, 1])
+    r = s0 * (z[0, 0].astype(np.float64) - z[0, 1])
+    c = z[0, 2].astype(np.float64) - z[0, 3]
+    return o, z, r, c
+
+
+def test_randomized_probability_formula_and_update():
+    for seed in range(6):
+        o, z, r, c = _rand_state(seed)
+        t = float(r @ c)
+        w = 3.0 * abs(t) + 1.0
+        p = 0.5 - t / (2 * w)                       # Algorithm 5 / Algorithm 2 with w made explicit
+        assert 0 < p < 1 and (p > 0.5) == (t < 0)   # leaning towards the greedy sign
+        for u, want in ((max(p - 1e-3, 0.0), +1), (min(p + 1e-3, 1 - 1e-12), -1)):
+            o2, z2, _, _ = _rand_state(seed)
+            s = o2.balance_one_randomized(0, z2[0, 2], z2[0, 3], u, w)
+            assert s == want
+            np.testing.assert_allclose(o2.r(), r + want * c, atol=1e-12)
+            assert o2.out_of_bound == 0
+
+
+def test_randomized_limits():
+    o, z, r, c = _rand_state(11)
+    t = float(r @ c)
+    # a huge bound makes it a fair coin
+    for u, want in ((0.49999, +1), (0.50001, -1)):
+        o2, z2, _, _ = _rand_state(11)
+        assert o2.balance_one_randomized(0, z2[0, 2], z2[0, 3], u, 1e18) == want
+    # |<r,c>| beyond the bound: the draw no longer matters, the greedy sign comes out, counted
+    for u in (0.0, 0.3, 0.999999):
+        o2, z2, _, _ = _rand_state(11)
+        s = o2.balance_one_randomized(0, z2[0, 2], z2[0, 3], u, abs(t) * 0.5)
+        assert s == (+1 if t < 0 else -1) and o2.out_of_bound == 1
+    with pytest.raises(RuntimeError):
+        o.balance_one_randomized(0, z[0, 2], z[0, 3], 0.5, 0.0)
+
+
+def test_randomized_expected_sign_is_minus_t_over_w():
+    o, z, r, c = _rand_state(3)
+    t = float(r @ c)
+    w = 2.0 * abs(t)
+    us = (np.arange(4000) + 0.5) / 4000            # an even grid of draws
+    total = 0
+    for u in us:
+        o2, z2, _, _ = _rand_state(3)
+        total += o2.balance_one_randomized(0, z2[0, 2], z2[0, 3], float(u), w)
+    assert abs(total / len(us) - (-t / w)) < 2e-3  # E[s] = 2p - 1 = -<r,c>/w
+
+
+def test_randomized_replay_band():
+    o, z, r, c = _rand_state(5)
+    t = float(r @ c); w = 4 * abs(t) + 1; p = 0.5 - t / (2 * w)
+    rn, cn = np.linalg.norm(r), np.linalg.norm(c)
+    tau = 1e-3
+    band = tau * rn * cn / (2 * w)
+    o2, z2, _, _ = _rand_state(5)
+    s = o2.balance_one_randomized(0, z2[0, 2], z2[0, 3], p + 0.5 * band, w, replay=+1, tau=tau)
+    assert s == +1 and o2.near_ties == 1 and o2.mismatches == 0      # inside the band: adopted
+    o3, z3, _, _ = _rand_state(5)
+    s = o3.balance_one_randomized(0, z3[0, 2], z3[0, 3], p + 2.0 * band, w, replay=+1, tau=tau)
+    assert s == -1 and o3.mismatches == 1                              # outside: own sign kept
