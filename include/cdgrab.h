@@ -108,6 +108,23 @@ int cdgrab_begin_epoch(cdgrab_t *h, void *stream);
 int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream);
 
 /*
+ * cdgrab_step with the randomized balance rule the paper's theory is stated for
+ * (RandomizedBalance, the subroutine of Algorithm 2, with the bound w of Algorithm 5 made
+ * explicit; Algorithm 2 prints w = 1): for worker i, p_i = 1/2 - <r,c_i>/(2w) and s_i = +1 with
+ * probability p_i.  The draws are the caller's: s_i = +1 iff u_dev[i] < p_i.
+ *   u_dev: DEVICE float [m], uniforms in [0,1), must stay valid until the step's work completes
+ *   w:     bound, w > 0 (else CDGRAB_ERR_INVALID)
+ * Where |<r,c_i>| > w Algorithm 5 would stop; here p_i leaves [0,1], the decision becomes the
+ * greedy one, and the position is counted (cdgrab_out_of_bound).  Algorithm 5's other stopping
+ * condition, ||r||_inf > w, is not evaluated.  Everything else is as in cdgrab_step.
+ */
+int cdgrab_step_randomized(cdgrab_t *h, const void *grads_dev, const float *u_dev, double w, void *stream);
+
+/* Synchronise the device and return how many positions of the current/last epoch had
+ * |<r,c>| > w under the randomized rule (negative CDGRAB_ERR_* on error). */
+long long cdgrab_out_of_bound(cdgrab_t *h);
+
+/*
  * cdgrab_step that also returns what the paper's parameter server sends back to the workers
  * (Algorithm 4, "compute avg. gradient ... send to all the workers"): the average of each of
  * the two gather buffers, mean_out_dev[q][x] = (1/m) sum_i grads_dev[q][i][x] for q = 0, 1.

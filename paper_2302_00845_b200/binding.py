@@ -28,6 +28,8 @@ SIGNATURES = {
     "cdgrab_set_perms": (C.c_int, [C.c_void_p, C.c_void_p]),
     "cdgrab_begin_epoch": (C.c_int, [C.c_void_p, C.c_void_p]),
     "cdgrab_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_step_randomized": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p]),
+    "cdgrab_out_of_bound": (C.c_longlong, [C.c_void_p]),
     "cdgrab_step_mean": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_end_epoch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_get_signs": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -135,6 +137,15 @@ class CdGrab:
     def step(self, grads, stream=None):
         """grads: CUDA tensor [2][m][d] of the handle's dtype."""
         _check(lib().cdgrab_step(self._h, _ptr(grads), _stream_ptr(stream)), "cdgrab_step")
+
+    def step_randomized(self, grads, u, w: float, stream=None):
+        """step() under the randomized rule: u CUDA float32 [m] uniforms, w > 0 the bound."""
+        _check(lib().cdgrab_step_randomized(self._h, _ptr(grads), _ptr(u), float(w), _stream_ptr(stream)),
+               "cdgrab_step_randomized")
+
+    @property
+    def out_of_bound(self) -> int:
+        return int(lib().cdgrab_out_of_bound(self._h))
 
     def step_mean(self, grads, mean_out, stream=None):
         """step() that also writes the average of each gather buffer into mean_out (CUDA float32 [2][d])."""

@@ -27,6 +27,7 @@ void free_all(cdgrab_ctx *h) {
   cudaFree(h->margins); cudaFree(h->rnorm2); cudaFree(h->status); cudaFree(h->gram);
   cudaFree(h->partials);
   cudaFree(h->ticket);
+  cudaFree(h->oob);
   if (h->prof_ev) {
     for (int i = 0; i < 2 * h->prof_cap; ++i) if (h->prof_ev[i]) cudaEventDestroy(h->prof_ev[i]);
     free(h->prof_ev);
@@ -125,6 +126,8 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
   ok = ok && cudaMalloc(&h->rnorm2, sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&h->status, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMalloc(&h->gram, sizeof(double) * ((size_t)m * m + m)) == cudaSuccess;
+  ok = ok && cudaMalloc(&h->oob, sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cudaMemset(h->oob, 0, sizeof(unsigned long long)) == cudaSuccess;
   ok = ok && cudaMalloc(&h->ticket, sizeof(unsigned)) == cudaSuccess;
   ok = ok && cudaMemset(h->ticket, 0, sizeof(unsigned)) == cudaSuccess;
   if (ok && path == CDGRAB_PATH_FMA) {
@@ -227,6 +230,7 @@ int cdgrab_begin_epoch(cdgrab_t *h, void *stream) {
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e = cudaMemsetAsync(h->r, 0, sizeof(float) * (size_t)h->d, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->rnorm2, 0, sizeof(double), st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->oob, 0, sizeof(unsigned long long), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->signs, 0, (size_t)h->m * (h->n / 2), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->margins, 0, sizeof(float) * (size_t)h->m * (h->n / 2), st);
   if (e == cudaSuccess && h->r_split)
@@ -256,6 +260,22 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   h->k++;
   return CDGRAB_OK;
+}
+
+int cdgrab_step_randomized(cdgrab_t *h, const void *grads_dev, const float *u_dev, double w, void *stream) {
+  if (!valid(h) || !u_dev || !(w > 0.0)) return CDGRAB_ERR_INVALID;
+  h->rule_randomized = 1; h->rule_u = u_dev; h->rule_w = w;
+  const int rc = cdgrab_step(h, grads_dev, stream);
+  h->rule_randomized = 0; h->rule_u = nullptr; h->rule_w = 0.0;
+  return rc;
+}
+
+long long cdgrab_out_of_bound(cdgrab_t *h) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  unsigned long long v = 0;
+  if (cudaMemcpy(&v, h->oob, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  return (long long)v;
 }
 
 int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, void *stream) {

@@ -39,6 +39,10 @@ struct cdgrab_ctx {
   int *status;           // [1] device status word
   double *gram;          // [m*m + m] G (row-major) then b
   double *partials;      // pass-1 partial sums
+  int rule_randomized;   // balance rule of the step being enqueued (0: greedy)
+  const float *rule_u;   // [m] uniforms for the randomized rule
+  double rule_w;
+  unsigned long long *oob;  // [1] positions with |<r,c>| > w seen by the randomized rule this epoch
   float *mean_out;       // [2][d] destination of the averaged gather buffers for the step being enqueued, or NULL
   size_t partials_bytes;
   int gram_chunks;       // grid.x of the FMA Gram kernels

@@ -10,6 +10,7 @@
 //                      permutation slots of Algorithm 7, update of r): the step's inputs
 //                      come from HBM once and are re-read from cache for the update
 #include "common.cuh"
+#include "scan.cuh"
 
 template <int M>
 struct Tri {
@@ -175,7 +176,7 @@ __global__ void __launch_bounds__(FusedCfg<M>::THREADS)
 fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, int k,
                   const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
                   int8_t *__restrict__ signs, float *__restrict__ margins,
-                  double *__restrict__ rnorm2, int *__restrict__ status) {
+                  double *__restrict__ rnorm2, int *__restrict__ status, const CdgRule rule) {
   extern __shared__ double dsh[];
   constexpr int WARPS = FusedCfg<M>::THREADS / 32;
   double *red = dsh;                                  // [WARPS][NPAD]
@@ -198,12 +199,13 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
     for (int i = 0; i < M; ++i) t[i] = tot[Tri<M>::NPAIR + i];
     double rn2 = *rnorm2;
     bool bad = false;
+    int oob = 0;
     const int half = n >> 1;
 #pragma unroll
     for (int i = 0; i < M; ++i) {
       if (i < m) {
         const double ti = t[i], gii = tot[Tri<M>::idx(i, i)];
-        const int s = (ti < 0.0) ? 1 : -1;   // +1 iff ||r+c|| < ||r-c||; a tie gives -1
+        const int s = cdg_decide(rule, i, ti, oob);   // greedy: +1 iff ||r+c|| < ||r-c||, a tie gives -1
         bad |= !(isfinite(ti) && isfinite(gii));
         const double sd = (double)s;
 #pragma unroll
@@ -223,6 +225,7 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
     }
     *rnorm2 = rn2;
     if (bad) atomicOr(status, CDG_ST_NONFINITE);
+    if (oob) atomicAdd(rule.oob, (unsigned long long)oob);
   }
   __syncthreads();
 
@@ -274,7 +277,7 @@ static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, cudaStream_t
     CdgProfScope ps(h, CDGRAB_K_FUSED, st);
     fused_step_kernel<T, M><<<1, FusedCfg<M>::THREADS, smem, st>>>(
         (const T *)grads, h->r, h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs,
-        h->margins, h->rnorm2, h->status);
+        h->margins, h->rnorm2, h->status, cdg_rule_of(h));
   }
   return cudaGetLastError();
 }
@@ -420,6 +423,7 @@ struct FtTail {
   int8_t *signs;
   float *margins;
   double *rnorm2;
+  CdgRule rule;
 };
 
 template <typename T, int M>
@@ -580,7 +584,8 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   scan_load_pairs(S, tail.perm_cur, m, tail.n, tail.k);
   if (threadIdx.x == 0) *tail.ticket = 0u;                    // ready for the next launch
   __syncthreads();
-  scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status);
+  scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
+                        tail.rule);
 }
 
 bool cdg_fma_tma_supported(int m, long long d, int dtype) {
@@ -659,6 +664,7 @@ static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, cudaStream_t st) {
   tail.ticket = h->ticket;
   tail.perm_cur = h->perm_cur; tail.perm_next = h->perm_next;
   tail.signs = h->signs; tail.margins = h->margins; tail.rnorm2 = h->rnorm2;
+  tail.rule = cdg_rule_of(h);
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     gram_fma_tma_kernel<T, M><<<h->gram_chunks, kFtThreads, h->fma_tma_smem, st>>>(

@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(256)
 scan_kernel(const double *__restrict__ gram, int m, int n, int k,
             const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
             int8_t *__restrict__ signs, float *__restrict__ margins,
-            double *__restrict__ rnorm2, int *__restrict__ status, int use_smem) {
+            double *__restrict__ rnorm2, int *__restrict__ status, int use_smem, const CdgRule rule) {
   extern __shared__ double sh[];
   const ScanSmem S = scan_smem(sh, m);
   const double *G = gram;
@@ -135,7 +135,7 @@ scan_kernel(const double *__restrict__ gram, int m, int n, int k,
   }
   scan_load_pairs(S, perm_cur, m, n, k);
   __syncthreads();
-  scan_decide_and_write(S, G, m, n, k, perm_next, signs, margins, rnorm2, status);
+  scan_decide_and_write(S, G, m, n, k, perm_next, signs, margins, rnorm2, status, rule);
 }
 
 // ------------------------------------------------------------------------------------
@@ -383,7 +383,7 @@ cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
   {
     CdgProfScope ps(h, CDGRAB_K_SCAN, st);
     scan_kernel<<<1, 256, smem, st>>>(h->gram, m, h->n, h->k, h->perm_cur, h->perm_next, h->signs,
-                                     h->margins, h->rnorm2, h->status, use_smem);
+                                     h->margins, h->rnorm2, h->status, use_smem, cdg_rule_of(h));
   }
   return cudaGetLastError();
 }

@@ -7,6 +7,33 @@
 
 #include "common.cuh"
 
+// Which balance rule decides the signs.  Greedy (Algorithm 6): +1 iff <r,c> < 0.
+// Randomized (Algorithm 2's subroutine with the bound w of Algorithm 5): p = 1/2 - <r,c>/(2w),
+// +1 iff u_i < p with u_i the caller's uniform draw for worker i; positions with |<r,c>| > w
+// (where Algorithm 5 would stop) are counted in *oob.
+struct CdgRule {
+  int randomized;
+  const float *u;             // [m] uniforms in [0,1), device
+  double w;
+  unsigned long long *oob;    // device counter
+};
+
+__device__ __forceinline__ int cdg_decide(const CdgRule &rule, int i, double ti, int &oob_local) {
+  if (!rule.randomized) return (ti < 0.0) ? 1 : -1;   // a tie gives -1
+  const double p = 0.5 - ti / (2.0 * rule.w);
+  if (fabs(ti) > rule.w) ++oob_local;
+  return ((double)rule.u[i] < p) ? 1 : -1;
+}
+
+inline CdgRule cdg_rule_of(const cdgrab_ctx *h) {
+  CdgRule r;
+  r.randomized = h->rule_randomized;
+  r.u = h->rule_u;
+  r.w = h->rule_w;
+  r.oob = h->oob;
+  return r;
+}
+
 struct ScanSmem {
   double *t;     // [m]  starts as b; entry i is <r_{i-1}, c_i> once worker i is decided
   double *rn;    // [m]  ||r||^2 seen by worker i
@@ -42,17 +69,18 @@ __device__ __forceinline__ void scan_load_pairs(const ScanSmem &S, const int32_t
 __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const double *G, int m, int n, int k,
                                                       int32_t *__restrict__ perm_next, int8_t *__restrict__ signs,
                                                       float *__restrict__ margins, double *__restrict__ rnorm2,
-                                                      int *__restrict__ status) {
+                                                      int *__restrict__ status, const CdgRule rule) {
   const int tid = threadIdx.x;
   if (tid < 32) {
     const int lane = tid;
     double rn2 = *rnorm2;
     bool bad = false;
+    int oob = 0;
     for (int i = 0; i < m; ++i) {
       const double ti = S.t[i];
       const double gii = G[(size_t)i * m + i];
-      // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0; a tie gives -1
-      const int s = (ti < 0.0) ? 1 : -1;
+      // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0 (or the randomized rule)
+      const int s = cdg_decide(rule, i, ti, oob);
       bad |= !(isfinite(ti) && isfinite(gii));
       const double sd = (double)s;
       // every later t_j gains s_i G_ij, summed in the order i = 0, 1, ...
@@ -65,6 +93,7 @@ __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const d
     if (lane == 0) {
       *rnorm2 = rn2;
       if (bad) atomicOr(status, CDG_ST_NONFINITE);
+      if (oob) atomicAdd(rule.oob, (unsigned long long)oob);
     }
   }
   __syncthreads();
