@@ -57,7 +57,8 @@ enum {
   CDGRAB_PATH_AUTO = 0,
   CDGRAB_PATH_FUSED = 1, /* one launch per step, whole step on chip (small d)            */
   CDGRAB_PATH_FMA = 2,   /* two passes, Gram matrix on the fp32 FMA pipe                 */
-  CDGRAB_PATH_UMMA = 3   /* two passes, Gram matrix on tcgen05 tensor cores (bf16)       */
+  CDGRAB_PATH_UMMA = 3,  /* two passes, Gram matrix on tcgen05 tensor cores (bf16)       */
+  CDGRAB_PATH_INDEPENDENT = 4 /* ID-GraB mode: one running sum per worker (see below)     */
 };
 
 /*
@@ -70,6 +71,20 @@ enum {
  * On success *out receives the handle.
  */
 int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out);
+
+/*
+ * Same interface for ID-GraB (PairBal), the uncoordinated baseline of the paper's experiments
+ * (Section 5): every worker i keeps its own running sum r_i and balances its own differences
+ * against it, s_i = +1 iff <r_i, c_i> < 0, r_i <- r_i + s_i c_i; the workers do not see each
+ * other.  Equals m separate handles with m = 1.  The handle holds m*d floats of running sums.
+ * cdgrab_get_r returns worker 0's sum, cdgrab_get_r_worker any worker's; margins are
+ * |<r_i,c_i>| / (||r_i|| ||c_i||) computed directly.  cdgrab_step_randomized and
+ * cdgrab_step_mean are CDGRAB_ERR_INVALID on such a handle.
+ */
+int cdgrab_create_independent(int m, int n, long long d, int dtype, cdgrab_t **out);
+
+/* Running sum of one worker of an independent-mode handle: out is HOST or DEVICE float [d]. */
+int cdgrab_get_r_worker(cdgrab_t *h, int worker, float *out, void *stream);
 
 /* Free the handle and everything it owns.  Synchronises the device.  NULL is allowed. */
 int cdgrab_destroy(cdgrab_t *h);

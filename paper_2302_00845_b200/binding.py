@@ -19,11 +19,13 @@ ERR_INVALID, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_NONFINITE, ERR_TIMEOUT, ERR_DEV
 ERR_TOO_LARGE = -8
 PATH_AUTO, PATH_FUSED, PATH_FMA, PATH_UMMA = 0, 1, 2, 3
 KERNEL_KINDS = ("gram", "combine", "scan", "update", "fused", "logreg")
-PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma"}
+PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma", 4: "independent"}
 
 # name -> (restype, argtypes); the single list of what include/cdgrab.h declares
 SIGNATURES = {
     "cdgrab_create": (C.c_int, [C.c_int, C.c_int, C.c_longlong, C.c_int, C.POINTER(C.c_void_p)]),
+    "cdgrab_create_independent": (C.c_int, [C.c_int, C.c_int, C.c_longlong, C.c_int, C.POINTER(C.c_void_p)]),
+    "cdgrab_get_r_worker": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]),
     "cdgrab_destroy": (C.c_int, [C.c_void_p]),
     "cdgrab_set_perms": (C.c_int, [C.c_void_p, C.c_void_p]),
     "cdgrab_begin_epoch": (C.c_int, [C.c_void_p, C.c_void_p]),
@@ -102,10 +104,13 @@ def _ptr(t):
 class CdGrab:
     """Order-server state for m workers x n items in R^d (see ``include/cdgrab.h``)."""
 
-    def __init__(self, m: int, n: int, d: int, dtype: str | int = "f32"):
+    def __init__(self, m: int, n: int, d: int, dtype: str | int = "f32", independent: bool = False):
         code = {"f32": F32, "bf16": BF16}.get(dtype, dtype)
         h = C.c_void_p()
-        _check(lib().cdgrab_create(m, n, d, code, C.byref(h)), "cdgrab_create")
+        if independent:   # ID-GraB (PairBal): one running sum per worker
+            _check(lib().cdgrab_create_independent(m, n, d, code, C.byref(h)), "cdgrab_create_independent")
+        else:
+            _check(lib().cdgrab_create(m, n, d, code, C.byref(h)), "cdgrab_create")
         self._h = h
         self.m, self.n, self.d, self.dtype = m, n, d, code
 
@@ -180,6 +185,13 @@ class CdGrab:
     def r(self):
         import torch
         return self._fetch("cdgrab_get_r", (self.d,), torch.float32)
+
+    def r_worker(self, i: int):
+        import torch
+        out = torch.empty(self.d, dtype=torch.float32, device="cuda")
+        _check(lib().cdgrab_get_r_worker(self._h, i, _ptr(out), _stream_ptr()), "cdgrab_get_r_worker")
+        torch.cuda.current_stream().synchronize()
+        return out
 
     def margins(self):
         import torch

@@ -75,7 +75,17 @@ const char *cdgrab_strerror(int code) {
   }
 }
 
+static int create_impl(int m, int n, long long d, int dtype, int independent, cdgrab_t **out);
+
 int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
+  return create_impl(m, n, d, dtype, 0, out);
+}
+
+int cdgrab_create_independent(int m, int n, long long d, int dtype, cdgrab_t **out) {
+  return create_impl(m, n, d, dtype, 1, out);
+}
+
+static int create_impl(int m, int n, long long d, int dtype, int independent, cdgrab_t **out) {
   if (!out) return CDGRAB_ERR_INVALID;
   *out = nullptr;
   if (m < 1 || m > 1024 || n < 2 || (n & 1) || d < 1) return CDGRAB_ERR_INVALID;
@@ -96,6 +106,7 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
   h->magic = CDG_MAGIC;
   h->m = m; h->n = n; h->d = d; h->dtype = dtype;
   h->device = dev; h->num_sms = prop.multiProcessorCount;
+  h->independent = independent;
 
   // ---- choose the path ------------------------------------------------------------
   const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);
@@ -113,12 +124,14 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
       return CDGRAB_ERR_INVALID;
     }
   }
+  if (independent) path = CDGRAB_PATH_INDEPENDENT;
   h->path = path;
 
   // ---- allocations ----------------------------------------------------------------
   const size_t np = (size_t)m * (size_t)(n / 2);
   bool ok = true;
-  ok = ok && cudaMalloc(&h->r, sizeof(float) * (size_t)d) == cudaSuccess;
+  const size_t r_elems = (size_t)d * (independent ? (size_t)m : 1);
+  ok = ok && cudaMalloc(&h->r, sizeof(float) * r_elems) == cudaSuccess;
   ok = ok && cudaMalloc(&h->perm_cur, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
   ok = ok && cudaMalloc(&h->perm_next, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
   ok = ok && cudaMalloc(&h->signs, np) == cudaSuccess;
@@ -130,6 +143,11 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
   ok = ok && cudaMemset(h->oob, 0, sizeof(unsigned long long)) == cudaSuccess;
   ok = ok && cudaMalloc(&h->ticket, sizeof(unsigned)) == cudaSuccess;
   ok = ok && cudaMemset(h->ticket, 0, sizeof(unsigned)) == cudaSuccess;
+  if (ok && independent) {
+    h->gram_chunks = cdg_indep_chunks(h);
+    h->partials_bytes = sizeof(double) * 3 * (size_t)m * (size_t)h->gram_chunks;
+    ok = ok && cudaMalloc(&h->partials, h->partials_bytes) == cudaSuccess;
+  }
   if (ok && path == CDGRAB_PATH_FMA) {
     if (fma_columns_ok(h)) {
       // thread-per-column kernel: one partial vector (<= 152 doubles) per block
@@ -178,7 +196,7 @@ int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
   cudaMemset(h->margins, 0, sizeof(float) * np);
   cudaMemset(h->rnorm2, 0, sizeof(double));
   cudaMemset(h->status, 0, sizeof(int));
-  cudaMemset(h->r, 0, sizeof(float) * (size_t)d);
+  cudaMemset(h->r, 0, sizeof(float) * r_elems);
   if (cudaDeviceSynchronize() != cudaSuccess) {
     cudaGetLastError();
     free_all(h);
@@ -228,7 +246,7 @@ int cdgrab_begin_epoch(cdgrab_t *h, void *stream) {
   if (!valid(h)) return CDGRAB_ERR_INVALID;
   if (h->epoch_open) return CDGRAB_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
-  cudaError_t e = cudaMemsetAsync(h->r, 0, sizeof(float) * (size_t)h->d, st);
+  cudaError_t e = cudaMemsetAsync(h->r, 0, sizeof(float) * (size_t)h->d * (h->independent ? (size_t)h->m : 1), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->rnorm2, 0, sizeof(double), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->oob, 0, sizeof(unsigned long long), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->signs, 0, (size_t)h->m * (h->n / 2), st);
@@ -247,7 +265,10 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
-  if (h->path == CDGRAB_PATH_FUSED) {
+  if (h->independent) {
+    if (h->rule_randomized || h->mean_out) return CDGRAB_ERR_INVALID;  // greedy rule only in this mode
+    e = cdg_launch_indep(h, grads_dev, st);
+  } else if (h->path == CDGRAB_PATH_FUSED) {
     e = cdg_launch_fused(h, grads_dev, st);
   } else {
     if (h->path == CDGRAB_PATH_UMMA) e = cdg_launch_gram_umma(h, grads_dev, st);
@@ -318,6 +339,10 @@ int cdgrab_get_signs(cdgrab_t *h, int8_t *out, void *stream) {
 int cdgrab_get_r(cdgrab_t *h, float *out, void *stream) {
   if (!valid(h)) return CDGRAB_ERR_INVALID;
   return copy_out(out, h->r, sizeof(float) * (size_t)h->d, stream);
+}
+int cdgrab_get_r_worker(cdgrab_t *h, int worker, float *out, void *stream) {
+  if (!valid(h) || !h->independent || worker < 0 || worker >= h->m) return CDGRAB_ERR_INVALID;
+  return copy_out(out, h->r + (size_t)worker * (size_t)h->d, sizeof(float) * (size_t)h->d, stream);
 }
 int cdgrab_get_margins(cdgrab_t *h, float *out, void *stream) {
   if (!valid(h)) return CDGRAB_ERR_INVALID;

@@ -39,6 +39,7 @@ struct cdgrab_ctx {
   int *status;           // [1] device status word
   double *gram;          // [m*m + m] G (row-major) then b
   double *partials;      // pass-1 partial sums
+  int independent;       // 1: ID-GraB mode, r is [m][d] (one running sum per worker)
   int rule_randomized;   // balance rule of the step being enqueued (0: greedy)
   const float *rule_u;   // [m] uniforms for the randomized rule
   double rule_w;
@@ -123,6 +124,10 @@ void *cdg_tensor_map_encoder();
 bool cdg_fma_tma_supported(int m, long long d, int dtype);
 int cdg_fma_tma_setup(cdgrab_ctx *h);
 cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+
+// ID-GraB (independent workers)
+int cdg_indep_chunks(const cdgrab_ctx *h);
+cudaError_t cdg_launch_indep(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 
 // tcgen05 path
 bool cdg_umma_supported(int m, long long d, int dtype);
