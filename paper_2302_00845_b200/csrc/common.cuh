@@ -74,6 +74,7 @@ struct cdgrab_ctx {
   int umma_box_rows;       // rows of the gradient TMA box (2m rounded up to 16)
   int umma_ncols;          // MMA N = box_rows + 16
   int umma_subs_per_stage;
+  int umma_drain;          // pipeline iterations per TMEM accumulation chunk
   int umma_stages;
   size_t umma_smem;
   CUtensorMap tm_r;        // 3-D tensor map over r_split

@@ -21,7 +21,8 @@
 // zeros (written once) pads N to a multiple of 16.  The same bytes serve as operand A (16
 // row groups from the block base) and operand B (the first N = box_rows + 16 rows).  A ragged
 // last block (d not a multiple of 64) is loaded with 2-D boxes of 8 rows into the same layout.
-// Roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2..5 read the accumulator back (tcgen05.ld) and write the CTA's partial H.
+// Roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2..5 drain the
+// accumulator (tcgen05.ld) chunk by chunk into fp32 registers and write the CTA's partial H.
 // Every wait is bounded: on expiry the CTA raises the time-out bit of the status word,
 // drains the copies it has in flight, frees its TMEM and returns.
 #include <cudaTypedefs.h>
@@ -36,6 +37,7 @@ constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr int kSubCols = 64;             // bf16 columns per TMA box = one 128-byte swizzle row
 constexpr int kRBoxRows = 16;
+constexpr int kMaxCols = 144;            // MMA N at m = 64: 128 gradient rows + 16
 constexpr long long kWaitCycles = kCdgWaitCycles;
 
 struct UmmaParams {
@@ -46,6 +48,7 @@ struct UmmaParams {
   int stages;
   long long nblk_full; // d / 64: blocks loaded by the 3-D maps
   int tail;            // 1 when d % 64 != 0: one more, ragged block
+  int drain;           // pipeline iterations accumulated in TMEM before the sum is drained
 };
 
 // K-major, 128-byte swizzle: rows 128 B apart, 8-row groups `sbo` bytes apart
@@ -76,7 +79,8 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
-  __shared__ __align__(8) uint64_t bar_accum;
+  __shared__ __align__(8) uint64_t bar_acc_full[2];    // accumulator buffer b holds a finished chunk
+  __shared__ __align__(8) uint64_t bar_acc_empty[2];   // ... has been read back and may be overwritten
   __shared__ uint32_t tmem_base_sh;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -97,7 +101,10 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
-    mbar_init(smem_u32(&bar_accum), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bar_acc_full[b]), 1);
+      mbar_init(smem_u32(&bar_acc_empty[b]), 4);     // one arrival per read-back warp
+    }
     mbar_init_fence();
   }
   // row groups that are never loaded (gradient groups wholly past row 2m, and the padding
@@ -114,7 +121,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // visible to the MMA's smem reads
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&tmem_base_sh)), "r"(256u) : "memory");
+                 ::"r"(smem_u32(&tmem_base_sh)), "r"(512u) : "memory");   // two accumulators of 256 columns
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -161,9 +168,20 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = ncols
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.ncols >> 3) << 17) |
                              ((128u >> 4) << 24);
+      // The fp32 accumulation inside the tensor core truncates; over hundreds of thousands of
+      // columns that becomes a visible bias on sums of same-sign products.  So the sum is kept
+      // in TMEM only for `drain` iterations (about 1024 columns), then handed to the read-back
+      // warps, which add the chunks in fp32 registers with round-to-nearest, while the MMAs
+      // continue into the other accumulator buffer.
       bool ok = true;
       for (int it = 0; it < n_iter && ok; ++it) {
         const int s = it % p.stages;
+        const int c = it / p.drain, buf = c & 1;
+        const bool chunk_start = (it % p.drain) == 0;
+        if (chunk_start && c >= 2) {
+          ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), ((c >> 1) - 1) & 1, deadline);
+          if (!ok) break;
+        }
         ok = mbar_wait(smem_u32(&bar_full[s]), (it / p.stages) & 1, deadline);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -172,34 +190,41 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
           const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
           cnt = (int)min((long long)p.subs, blk_hi - first);   // blocks past blk_hi belong to the next CTA
         }
+        const uint32_t acc = tmem_acc + (uint32_t)buf * 256u;
         for (int q = 0; q < cnt; ++q) {
           const uint64_t desc = umma_desc(tiles + s * stage_bytes + q * 1024u, group_bytes);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4) {
             // 16 bf16 = 32 bytes further along K inside the swizzle row
             const uint64_t dk = desc + (uint64_t)(k4 * 2);
-            umma_bf16(tmem_acc, dk, dk, idesc, (it | q | k4) != 0);
+            umma_bf16(acc, dk, dk, idesc, !(chunk_start && q == 0 && k4 == 0));
           }
         }
         umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
+        if ((it % p.drain) == p.drain - 1 || it == n_iter - 1)
+          umma_commit(smem_u32(&bar_acc_full[buf]));   // chunk complete
       }
-      if (ok) umma_commit(smem_u32(&bar_accum));  // accumulator complete
-      else atomicOr(status, CDG_ST_TIMEOUT);
+      if (!ok) atomicOr(status, CDG_ST_TIMEOUT);
     }
   } else {
-    // ---------------- accumulator read-back: TMEM -> partial H ----------------
-    const bool ok = (n_iter == 0) ? true : mbar_wait(smem_u32(&bar_accum), 0, deadline);
-    if (!ok) {
-      if (lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
-    } else {
+    // ---------------- accumulator read-back: TMEM chunks -> fp32 registers -> partial H ----------------
+    const int lg = warp & 3;                 // TMEM lane group this warp may read
+    const int row = lg * 32 + lane;
+    const int nchunks = (n_iter + p.drain - 1) / p.drain;
+    float accr[kMaxCols];
+#pragma unroll
+    for (int j = 0; j < kMaxCols; ++j) accr[j] = 0.f;
+    bool ok = true;
+    for (int c = 0; c < nchunks && ok; ++c) {
+      const int buf = c & 1;
+      ok = mbar_wait(smem_u32(&bar_acc_full[buf]), (c >> 1) & 1, deadline);
+      if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int lg = warp & 3;                 // TMEM lane group this warp may read
-      const int row = lg * 32 + lane;
-      float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.ncols;
-      for (int c0 = 0; c0 < p.ncols; c0 += 16) {
-        uint32_t v[16];
-        if (n_iter > 0) {
-          const uint32_t taddr = tmem_acc + ((uint32_t)(lg * 32) << 16) + (uint32_t)c0;
+#pragma unroll
+      for (int piece = 0; piece < kMaxCols / 16; ++piece) {
+        if (piece * 16 < p.ncols) {
+          uint32_t v[16];
+          const uint32_t taddr = tmem_acc + (uint32_t)buf * 256u + ((uint32_t)(lg * 32) << 16) + (uint32_t)(piece * 16);
           asm volatile(
               "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
               "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -208,16 +233,26 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
                 "=r"(v[14]), "=r"(v[15])
               : "r"(taddr) : "memory");
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0u;
+          for (int j = 0; j < 16; ++j) accr[piece * 16 + j] += __uint_as_float(v[j]);
         }
-        if (row < p.rows_used) {
+      }
+      // the buffer may be overwritten once all four warps have read it
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+    }
+    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+    if (row < p.rows_used) {
+      float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.ncols;
+#pragma unroll
+      for (int piece = 0; piece < kMaxCols / 16; ++piece) {
+        if (piece * 16 < p.ncols) {
 #pragma unroll
           for (int j = 0; j < 16; j += 4)
-            *reinterpret_cast<float4 *>(dst + c0 + j) =
-                make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                            __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+            *reinterpret_cast<float4 *>(dst + piece * 16 + j) =
+                make_float4(accr[piece * 16 + j], accr[piece * 16 + j + 1], accr[piece * 16 + j + 2],
+                            accr[piece * 16 + j + 3]);
         }
       }
     }
@@ -227,7 +262,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(256u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(512u) : "memory");
   }
 }
 
@@ -336,6 +371,12 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     if (v >= 1 && v <= 8) subs = v;
   }
   h->umma_subs_per_stage = subs;
+  // TMEM chunk length in pipeline iterations (about 4096 columns); CDGRAB_UMMA_DRAIN overrides
+  h->umma_drain = 4096 / (subs * kSubCols) > 0 ? 4096 / (subs * kSubCols) : 1;
+  if (const char *e = getenv("CDGRAB_UMMA_DRAIN")) {
+    const int v = atoi(e);
+    if (v >= 1 && v <= (1 << 20)) h->umma_drain = v;
+  }
   const size_t group_bytes = (size_t)subs * 1024;
   const size_t stage_bytes = group_bytes * (h->umma_ncols / 8);
   const int ngroups = h->umma_ncols / 8;
@@ -392,6 +433,7 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
   p.stages = h->umma_stages;
   p.nblk_full = nblk_full;
   p.tail = (h->d % kSubCols) ? 1 : 0;
+  p.drain = h->umma_drain;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     gram_umma_kernel<<<h->umma_ctas, kThreads, h->umma_smem, st>>>(h->tm_g, h->tm_r, h->tm_g2, h->tm_r2, p,

@@ -41,8 +41,14 @@ def run_full(name, steps):
         err = rel_l2(gpu.r().cpu().numpy().astype(np.float64), cpu.r())
         assert err <= R_TOL[wl.dtype], err
         assert gpu.status() == binding.OK
+        # accuracy of the GPU's <r,c>: its relative margins against the oracle's fp64 trace
+        t, rn, cn = cpu.trace()
+        want = np.where(rn * cn > 0, np.abs(t) / np.maximum(rn * cn, 1e-300), 0.0)[:, :steps]
+        got = gpu.margins().cpu().numpy()[:, :steps].astype(np.float64)
+        margin_err = float(np.abs(got - want).max())
+        assert margin_err <= 0.05 * TAU[wl.dtype], margin_err   # far inside the tie band
         print(f"{name} full size, {steps} steps: path={gpu.path} near_ties={cpu.near_ties} "
-              f"raw_agree={raw / (m * steps):.4f} r_rel_err={err:.2e}")
+              f"raw_agree={raw / (m * steps):.4f} r_rel_err={err:.2e} max_margin_err={margin_err:.2e}")
         return gpu.path
     finally:
         gpu.destroy(); cpu.close()
