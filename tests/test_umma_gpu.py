@@ -62,3 +62,23 @@ def test_umma_matches_fma_path_signs(monkeypatch):
     assert torch.equal(out["umma"][0], out["fma"][0])
     assert torch.equal(out["umma"][1], out["fma"][1])   # same signs -> same fp32 update order
     np.testing.assert_allclose(out["umma"][2].numpy(), out["fma"][2].numpy(), rtol=1e-3, atol=1e-6)
+
+
+@pytest.mark.parametrize("mean,scale", [(0.3, 0.1), (1.0, 0.1)])
+def test_umma_long_rows_with_common_mean(mean, scale, monkeypatch):
+    """Rows of 16 M columns (about 108 K columns per CTA, many accumulator chunks) whose shared
+    mean is 3x / 10x the per-example noise: the four-term cancellation G = H - H - H + H has to
+    survive the tensor core's accumulation error."""
+    monkeypatch.setenv("CDGRAB_FORCE_PATH", "umma")
+    m, n, d = 8, 4, 16_000_000
+    pr = Pair(m, n, d, "bf16")
+    try:
+        assert pr.gpu.path == "umma"
+        pr.begin()
+        for k in range(n // 2):
+            pr.step(grads(m, d, 40 + k, mean, scale))
+        rep = pr.end()
+        print(f"umma long rows mean={mean} scale={scale}:", rep)
+        assert rep.raw_agreement == 1.0
+    finally:
+        pr.close()
