@@ -184,6 +184,20 @@ int cdgrab_get_next_perms(cdgrab_t *h, int32_t *out, void *stream);
  * creation (CDGRAB_ERR_NONFINITE, CDGRAB_ERR_TIMEOUT, CDGRAB_ERR_CUDA) or CDGRAB_OK. */
 int cdgrab_status(cdgrab_t *h);
 
+/* Synchronise the device and clear the device status word (after the caller has dealt with a
+ * reported condition). */
+int cdgrab_clear_status(cdgrab_t *h);
+
+/*
+ * Self-test of the bounded device-side wait used by the TMA-fed kernels: a one-thread kernel
+ * waits on a barrier that nothing completes, gives up after `cycles` SM clock cycles
+ * (1 .. 2e9), raises the time-out bit of the status word and returns; nothing is in flight, so
+ * the context stays usable.  Synchronous.  *waited_cycles (HOST, may be NULL) receives how long
+ * the kernel actually waited.  Afterwards cdgrab_status() reports CDGRAB_ERR_TIMEOUT until
+ * cdgrab_clear_status() is called.
+ */
+int cdgrab_selftest_wait_timeout(cdgrab_t *h, long long cycles, long long *waited_cycles);
+
 /* Code path the handle uses (CDGRAB_PATH_*).  The environment variable
  * CDGRAB_FORCE_PATH = fused | fma | umma, read at create time, overrides the automatic
  * choice when the forced path supports the shape; otherwise create fails with

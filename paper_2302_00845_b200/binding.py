@@ -40,6 +40,8 @@ SIGNATURES = {
     "cdgrab_get_perms": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_get_next_perms": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_status": (C.c_int, [C.c_void_p]),
+    "cdgrab_clear_status": (C.c_int, [C.c_void_p]),
+    "cdgrab_selftest_wait_timeout": (C.c_int, [C.c_void_p, C.c_longlong, C.POINTER(C.c_longlong)]),
     "cdgrab_path": (C.c_int, [C.c_void_p]),
     "cdgrab_launch_count": (C.c_longlong, [C.c_void_p]),
     "cdgrab_strerror": (C.c_char_p, [C.c_int]),

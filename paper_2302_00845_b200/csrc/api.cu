@@ -406,6 +406,31 @@ int cdgrab_profile_read(cdgrab_t *h, int kind, double *total_ms, long long *laun
   return CDGRAB_OK;
 }
 
+int cdgrab_selftest_wait_timeout(cdgrab_t *h, long long cycles, long long *waited_cycles) {
+  if (!valid(h) || cycles < 1 || cycles > 2000000000ll) return CDGRAB_ERR_INVALID;
+  long long *dev = nullptr;
+  if (cudaMalloc(&dev, sizeof(long long)) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_NOMEM; }
+  int rc = CDGRAB_OK;
+  long long waited = 0;
+  if (cdg_launch_wait_selftest(h, cycles, dev, nullptr) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(&waited, dev, sizeof(long long), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    rc = CDGRAB_ERR_CUDA;
+  }
+  cudaFree(dev);
+  if (waited_cycles) *waited_cycles = waited;
+  return rc;
+}
+
+int cdgrab_clear_status(cdgrab_t *h) {
+  if (!valid(h)) return CDGRAB_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemset(h->status, 0, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  return CDGRAB_OK;
+}
+
 int cdgrab_path(const cdgrab_t *h) { return valid(h) ? h->path : CDGRAB_ERR_INVALID; }
 
 long long cdgrab_launch_count(const cdgrab_t *h) { return valid(h) ? h->launches : -1; }

@@ -130,6 +130,8 @@ cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream
 int cdg_indep_chunks(const cdgrab_ctx *h);
 cudaError_t cdg_launch_indep(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 
+cudaError_t cdg_launch_wait_selftest(cdgrab_ctx *h, long long cycles, long long *waited_dev, cudaStream_t st);
+
 // tcgen05 path
 bool cdg_umma_supported(int m, long long d, int dtype);
 int cdg_umma_setup(cdgrab_ctx *h);   // allocations + tensor maps; CDGRAB_* code

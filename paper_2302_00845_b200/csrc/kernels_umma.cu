@@ -351,6 +351,27 @@ bool encode_map_3d(CUtensorMap *map, const void *base, long long nblk, int rows,
 
 }  // namespace
 
+// Self-test of the bounded wait every TMA-fed kernel here relies on: one thread waits on a
+// barrier that nothing ever completes, gives up after `cycles`, raises the time-out bit and
+// returns.  No copy, no TMEM, nothing in flight.
+__global__ void wait_timeout_selftest_kernel(long long cycles, int *status, long long *waited) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    mbar_init_fence();
+    const long long t0 = clock64();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, t0 + cycles);
+    *waited = clock64() - t0;
+    if (!ok) atomicOr(status, CDG_ST_TIMEOUT);
+  }
+}
+
+cudaError_t cdg_launch_wait_selftest(cdgrab_ctx *h, long long cycles, long long *waited_dev, cudaStream_t st) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(cycles, h->status, waited_dev);
+  h->launches++;
+  return cudaGetLastError();
+}
+
 void *cdg_tensor_map_encoder() { return (void *)encode_fn(); }
 
 bool cdg_umma_supported(int m, long long d, int dtype) {
