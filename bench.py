@@ -38,11 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by kernel kind and workload; valid only while the kernel source hash matches.
-NCU_TRAFFIC: dict = {
-    # captured at d = 8,000,000 (profiles/*_gpt2_d8m.md), scaled by d to a full-size launch
-    ("gram", "gpt2"): {"bytes": 2.105445e9 * 15.5, "source": "8fbf93204aa13d41"},
-    ("update", "gpt2"): {"bytes": 2.156762e9 * 15.5, "source": "8fbf93204aa13d41"},
-}
+NCU_TRAFFIC: dict = {}   # filled below, after source_hash is defined
 
 
 def parse_args():
@@ -157,12 +153,22 @@ def aggregate_replicas(ms_local: float, examples_local: int, world: int, device:
     return examples_local * world / (ms * 1e-3), ms
 
 
-def source_hash() -> str:
+def source_hash(files=None) -> str:
+    """Hash of the kernel sources a traffic figure was captured with (all of csrc by default)."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2302_00845_b200", "csrc")
-    for f in sorted(os.listdir(csrc)):
+    for f in sorted(files or os.listdir(csrc)):
         h.update(open(os.path.join(csrc, f), "rb").read())
     return h.hexdigest()[:16]
+
+
+# captured with ncu --set full (profiles/*.md); gpt2 figures were taken at d = 8,000,000 and are
+# scaled by d to a full-size launch (traffic grows in proportion to d)
+NCU_TRAFFIC.update({
+    ("gram", "gpt2"): {"bytes": 2.105556e9 * 15.5, "files": ["kernels_umma.cu", "ptx.cuh"], "source": "6420258e27a6fc43"},
+    ("update", "gpt2"): {"bytes": 2.155589e9 * 15.5, "files": ["kernels_generic.cu"], "source": "729b498181954917"},
+    ("gram", "mid"): {"bytes": 144.179e6, "files": ["kernels_fma.cu", "ptx.cuh", "scan.cuh"], "source": "8c910e75f8a3a487"},
+})
 
 
 # ------------------------------------------------------------------------------------------
@@ -347,7 +353,7 @@ def run_native(args):
         ab = algorithmic_bytes(dom, wl)
         achieved = ab / (avg_ms * 1e-3) / 1e9
         tr = NCU_TRAFFIC.get((dom, wl.name))
-        traffic = tr["bytes"] if tr and tr.get("source") == source_hash() else None
+        traffic = tr["bytes"] if tr and tr.get("source") == source_hash(tr.get("files")) else None
         roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
                 "avg_launch_ms": avg_ms, "algorithmic_bytes_per_launch": ab,

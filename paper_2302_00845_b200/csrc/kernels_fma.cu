@@ -563,8 +563,10 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     // slice p adds blocks p, p+3, ... in that order; the slices are then added in order
     const int e = threadIdx.x % NP, p = threadIdx.x / NP;
     double v = 0.0;
-    if (e < Tri<M>::NACC)
+    if (e < Tri<M>::NACC) {
+#pragma unroll 8
       for (int b = p; b < (int)gridDim.x; b += 3) v += __ldcg(partials + (size_t)b * Tri<M>::NACC + e);
+    }
     slices[p * NP + e] = v;
   }
   __syncthreads();
