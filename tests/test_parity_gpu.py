@@ -317,3 +317,28 @@ def test_handles_side_by_side_do_not_disturb_each_other(m, d, dtype):
     finally:
         for h in hs:
             h.destroy()
+
+
+@pytest.mark.parametrize("m,d,dtype", [(4, 2048, "f32"), (16, 200_000, "f32"), (32, 30_016, "bf16")])
+def test_work_follows_the_callers_stream(m, d, dtype):
+    """An epoch issued on a side stream (inputs produced on that stream too) gives the same result
+    as on the default stream: nothing in the library falls back to another stream."""
+    n = 6
+    def run(stream):
+        with torch.cuda.stream(stream):
+            with binding.CdGrab(m, n, d, dtype) as h:
+                h.begin_epoch(stream)
+                for k in range(n // 2):
+                    g = random_grads(m, d, dtype, 4200 + k, mean=0.1)
+                    g = g * 1.0            # produced by a kernel on this stream just before the step
+                    h.step(g, stream)
+                out = torch.empty(m, n, dtype=torch.int32, device="cuda")
+                h.end_epoch(out, stream)
+                stream.synchronize()
+                res = (h.signs().cpu(), h.r().cpu(), out.cpu())
+                assert h.status() == binding.OK
+                return res
+    a = run(torch.cuda.default_stream())
+    b = run(torch.cuda.Stream())
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
