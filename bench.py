@@ -294,8 +294,10 @@ def run_native(args):
             h.begin_epoch()
         buf = bufs[state["step"] % nbuf]
         if prob is not None:
-            h.logreg_grads(prob.X, prob.y, prob.w, buf)
-        h.step(buf)
+            # gradients and balancing in one launch, straight from the feature rows
+            h.step_logreg(prob.X, prob.y, prob.w)
+        else:
+            h.step(buf)
         state["step"] += 1
 
     def barrier():
@@ -367,6 +369,8 @@ def run_native(args):
 
     # ---- end to end through the host-buffer call ----------------------------------------------
     e2e = None
+    if prob is not None:
+        h.logreg_grads(prob.X, prob.y, prob.w, bufs[0])   # the gradient bytes for the host-side legs
     if not args.no_e2e and world == 1:
         e2e = run_e2e(h, wl, bufs[0], state, one_step)
 

@@ -243,6 +243,17 @@ int cdgrab_logreg_grads(cdgrab_t *h, const float *X, const float *y, const float
                         float *grads_out, void *stream);
 
 /*
+ * Logistic regression without a gradient buffer: cdgrab_logreg_grads followed by cdgrab_step in
+ * one launch, the pair differences formed straight from the feature rows,
+ *   c_i = (sigma(<w,x_p>) - y_p) x_p - (sigma(<w,x_q>) - y_q) x_q,  p, q = perm_cur[i][2k], [2k+1]
+ * (each product rounded to fp32 as a stored gradient would be).  Same arguments as
+ * cdgrab_logreg_grads minus the output; X and w 16-byte aligned.  Only for fp32 handles small
+ * enough for the single-launch path (cdgrab_path == CDGRAB_PATH_FUSED), else CDGRAB_ERR_INVALID.
+ * Counts as one balancing step.  Asynchronous on `stream`.
+ */
+int cdgrab_step_logreg(cdgrab_t *h, const float *X, const float *y, const float *w, void *stream);
+
+/*
  * Same step with the gradients in HOST memory (pinned memory makes the copy
  * asynchronous): grads_host [2][m][d] is copied into staging_dev (DEVICE, at least
  * 2*m*d elements, 16-byte aligned, caller-owned) on `stream`, then cdgrab_step runs on it.

@@ -48,6 +48,7 @@ SIGNATURES = {
     "cdgrab_profile_enable": (C.c_int, [C.c_void_p, C.c_int]),
     "cdgrab_profile_read": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]),
     "cdgrab_logreg_grads": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_step_logreg": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_step_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_herding_workspace_bytes": (C.c_longlong, [C.c_int, C.c_int, C.c_longlong]),
     "cdgrab_herding_objective": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_longlong, C.c_void_p,
@@ -158,6 +159,11 @@ class CdGrab:
         """step() that also writes the average of each gather buffer into mean_out (CUDA float32 [2][d])."""
         _check(lib().cdgrab_step_mean(self._h, _ptr(grads), _ptr(mean_out), _stream_ptr(stream)),
                "cdgrab_step_mean")
+
+    def step_logreg(self, X, y, w, stream=None):
+        """One balancing step straight from the feature rows (no gradient buffer)."""
+        _check(lib().cdgrab_step_logreg(self._h, _ptr(X), _ptr(y), _ptr(w), _stream_ptr(stream)),
+               "cdgrab_step_logreg")
 
     def step_host(self, grads_host, staging, stream=None):
         """grads_host: pinned host tensor [2][m][d]; staging: CUDA tensor of the same size."""

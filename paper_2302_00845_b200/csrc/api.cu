@@ -283,6 +283,16 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   return CDGRAB_OK;
 }
 
+int cdgrab_step_logreg(cdgrab_t *h, const float *X, const float *y, const float *w, void *stream) {
+  if (!valid(h) || !X || !y || !w) return CDGRAB_ERR_INVALID;
+  if (h->dtype != CDGRAB_F32 || h->path != CDGRAB_PATH_FUSED) return CDGRAB_ERR_INVALID;
+  if ((((uintptr_t)X | (uintptr_t)w) & 15) != 0) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
+  if (cdg_launch_fused_logreg(h, X, y, w, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->k++;
+  return CDGRAB_OK;
+}
+
 int cdgrab_step_randomized(cdgrab_t *h, const void *grads_dev, const float *u_dev, double w, void *stream) {
   if (!valid(h) || !u_dev || !(w > 0.0)) return CDGRAB_ERR_INVALID;
   h->rule_randomized = 1; h->rule_u = u_dev; h->rule_w = w;

@@ -114,6 +114,7 @@ cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st)
 cudaError_t cdg_launch_mean(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_gram_fma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_fused_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w, cudaStream_t st);
 cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,
                               float *out, cudaStream_t st);
 bool cdg_fused_supported(int m, long long d, int dtype);

@@ -164,6 +164,49 @@ fma_combine_kernel(const double *__restrict__ partials, int blocks, int m, doubl
   }
 }
 
+// One thread: Algorithm 6 for i = 0..m-1 on t_i = b_i + sum_{k<i} s_k G_ki from the block totals
+// (triangle entries, then b), signs / margins / permutation slots (Algorithm 7) written out, the
+// signs also left in ssh as +-1.0f for the update that follows.
+template <int M>
+__device__ __forceinline__ void fused_decide(const double *tot, int m, int n, int k,
+                                             const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
+                                             int8_t *__restrict__ signs, float *__restrict__ margins,
+                                             double *__restrict__ rnorm2, int *__restrict__ status,
+                                             const CdgRule &rule, float *ssh) {
+  double t[M];
+#pragma unroll
+  for (int i = 0; i < M; ++i) t[i] = tot[Tri<M>::NPAIR + i];
+  double rn2 = *rnorm2;
+  bool bad = false;
+  int oob = 0;
+  const int half = n >> 1;
+#pragma unroll
+  for (int i = 0; i < M; ++i) {
+    if (i < m) {
+      const double ti = t[i], gii = tot[Tri<M>::idx(i, i)];
+      const int s = cdg_decide(rule, i, ti, oob);   // greedy: +1 iff ||r+c|| < ||r-c||, a tie gives -1
+      bad |= !(isfinite(ti) && isfinite(gii));
+      const double sd = (double)s;
+#pragma unroll
+      for (int j = i + 1; j < M; ++j) t[j] += sd * tot[Tri<M>::idx(i, j)];
+      const size_t pos = (size_t)i * half + k;
+      signs[pos] = (int8_t)s;
+      const double den = rn2 * gii;
+      margins[pos] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
+      const int32_t first = perm_cur[(size_t)i * n + 2 * k];
+      const int32_t second = perm_cur[(size_t)i * n + 2 * k + 1];
+      perm_next[(size_t)i * n + k] = (s == 1) ? first : second;           // front slot
+      perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;  // back slot
+      rn2 += 2.0 * sd * ti + gii;
+      if (rn2 < 0.0) rn2 = 0.0;
+      ssh[i] = (float)s;
+    }
+  }
+  *rnorm2 = rn2;
+  if (bad) atomicOr(status, CDG_ST_NONFINITE);
+  if (oob) atomicAdd(rule.oob, (unsigned long long)oob);
+}
+
 // ------------------------------------------------------------------------------------
 // Whole step in one CTA.  The thread count shrinks with M so the accumulators stay in
 // registers: 1024 threads for M = 4, 512 for M = 8, 256 for M = 16.
@@ -192,41 +235,8 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
   if (threadIdx.x < Tri<M>::NACC) tot[threadIdx.x] = v;
   __syncthreads();
 
-  if (threadIdx.x == 0) {
-    // Algorithm 6 for i = 0..m-1 on t_i = b_i + sum_{k<i} s_k G_ki
-    double t[M];
-#pragma unroll
-    for (int i = 0; i < M; ++i) t[i] = tot[Tri<M>::NPAIR + i];
-    double rn2 = *rnorm2;
-    bool bad = false;
-    int oob = 0;
-    const int half = n >> 1;
-#pragma unroll
-    for (int i = 0; i < M; ++i) {
-      if (i < m) {
-        const double ti = t[i], gii = tot[Tri<M>::idx(i, i)];
-        const int s = cdg_decide(rule, i, ti, oob);   // greedy: +1 iff ||r+c|| < ||r-c||, a tie gives -1
-        bad |= !(isfinite(ti) && isfinite(gii));
-        const double sd = (double)s;
-#pragma unroll
-        for (int j = i + 1; j < M; ++j) t[j] += sd * tot[Tri<M>::idx(i, j)];
-        const size_t pos = (size_t)i * half + k;
-        signs[pos] = (int8_t)s;
-        const double den = rn2 * gii;
-        margins[pos] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
-        const int32_t first = perm_cur[(size_t)i * n + 2 * k];
-        const int32_t second = perm_cur[(size_t)i * n + 2 * k + 1];
-        perm_next[(size_t)i * n + k] = (s == 1) ? first : second;           // front slot
-        perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;  // back slot
-        rn2 += 2.0 * sd * ti + gii;
-        if (rn2 < 0.0) rn2 = 0.0;
-        ssh[i] = (float)s;
-      }
-    }
-    *rnorm2 = rn2;
-    if (bad) atomicOr(status, CDG_ST_NONFINITE);
-    if (oob) atomicAdd(rule.oob, (unsigned long long)oob);
-  }
+  if (threadIdx.x == 0)
+    fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh);
   __syncthreads();
 
   // r <- r + sum_i s_i c_i (i ascending), inputs re-read through the cache
@@ -250,6 +260,166 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
     *reinterpret_cast<float4 *>(r + x) =
         make_float4((float)a4[0], (float)a4[1], (float)a4[2], (float)a4[3]);
   }
+}
+
+// ------------------------------------------------------------------------------------
+// Logistic regression without a gradient buffer: the whole step from the feature rows.
+// For worker i the pair's items are p = perm_cur[i][2k], q = perm_cur[i][2k+1]; with
+// a = sigma(<w,x_p>) - y_p and b = sigma(<w,x_q>) - y_q the difference is c_i = a x_p - b x_q
+// (each product rounded to fp32 like a stored gradient would be).  One CTA: coefficients,
+// Gram, decisions, update.
+// ------------------------------------------------------------------------------------
+template <int M>
+__device__ __forceinline__ void logreg_diffs(const float *__restrict__ X, const size_t *rowoff, const float *coef,
+                                             int m, size_t x, float (&c)[M][4]) {
+#pragma unroll
+  for (int i = 0; i < M; ++i) {
+    if (i < m) {
+      float xp[4], xq[4];
+      ld4<float>(X + rowoff[i] + x, xp);
+      ld4<float>(X + rowoff[m + i] + x, xq);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) c[i][j] = __fsub_rn(__fmul_rn(coef[i], xp[j]), __fmul_rn(coef[m + i], xq[j]));
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) c[i][j] = 0.f;
+    }
+  }
+}
+
+template <int M>
+__global__ void __launch_bounds__(FusedCfg<M>::THREADS)
+fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ y, const float *__restrict__ w,
+                         float *r, int m, int n, long long d, int k, const int32_t *__restrict__ perm_cur,
+                         int32_t *__restrict__ perm_next, int8_t *__restrict__ signs, float *__restrict__ margins,
+                         double *__restrict__ rnorm2, int *__restrict__ status, const CdgRule rule) {
+  extern __shared__ double dsh[];
+  constexpr int WARPS = FusedCfg<M>::THREADS / 32;
+  double *red = dsh;                                  // [WARPS][NPAD]; first used as [WARPS][2M] for the dots
+  double *tot = red + WARPS * Tri<M>::NPAD;           // [NPAD]
+  float *ssh = reinterpret_cast<float *>(tot + Tri<M>::NPAD);  // [M]
+  float *coef = ssh + M;                              // [2M]: a_0..a_{m-1}, b_0..b_{m-1}
+  float *yv = coef + 2 * M;                           // [2M]
+  size_t *rowoff = reinterpret_cast<size_t *>(yv + 2 * M);      // [2M] element offsets of the rows in X
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long nvec = d / 4;
+
+  if (threadIdx.x < 2 * m) {
+    const int q = threadIdx.x / m, i = threadIdx.x % m;
+    const int item = perm_cur[(size_t)i * n + 2 * k + q];
+    rowoff[threadIdx.x] = ((size_t)i * n + item) * (size_t)d;
+    yv[threadIdx.x] = y[(size_t)i * n + item];
+  }
+  __syncthreads();
+
+  // <w, x> for the 2m rows
+  {
+    float z[2 * M];
+#pragma unroll
+    for (int e = 0; e < 2 * M; ++e) z[e] = 0.f;
+    for (long long v = threadIdx.x; v < nvec; v += blockDim.x) {
+      const size_t x = (size_t)v * 4;
+      float wv[4];
+      ld4<float>(w + x, wv);
+#pragma unroll
+      for (int e = 0; e < 2 * M; ++e) {
+        if (e < 2 * m) {
+          float xv[4];
+          ld4<float>(X + rowoff[e] + x, xv);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) z[e] = fmaf(wv[j], xv[j], z[e]);
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 2 * M; ++e) {
+      double v = (double)z[e];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+      if (lane == 0) red[warp * 2 * M + e] = v;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < 2 * m) {
+    double zz = 0.0;
+    for (int wi = 0; wi < WARPS; ++wi) zz += red[wi * 2 * M + threadIdx.x];
+    const float zf = (float)zz;
+    // sigma(z) - y without cancellation for y in {0,1}: sigma(z) - 1 = -sigma(-z)
+    coef[threadIdx.x] = (yv[threadIdx.x] > 0.5f) ? -1.f / (1.f + expf(zf)) : 1.f / (1.f + expf(-zf));
+  }
+  __syncthreads();
+
+  float acc[Tri<M>::NPAD];
+#pragma unroll
+  for (int e = 0; e < Tri<M>::NPAD; ++e) acc[e] = 0.f;
+  for (long long v = threadIdx.x; v < nvec; v += blockDim.x) {
+    const size_t x = (size_t)v * 4;
+    float c[M][4], rv[4];
+    logreg_diffs<M>(X, rowoff, coef, m, x, c);
+    ld4_r(r + x, rv);
+#pragma unroll
+    for (int a = 0; a < M; ++a) {
+#pragma unroll
+      for (int b = a; b < M; ++b) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[Tri<M>::idx(a, b)] = fmaf(c[a][j], c[b][j], acc[Tri<M>::idx(a, b)]);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[Tri<M>::NPAIR + a] = fmaf(rv[j], c[a][j], acc[Tri<M>::NPAIR + a]);
+    }
+  }
+  const double v = block_reduce_acc<M, WARPS>(acc, red);
+  if (threadIdx.x < Tri<M>::NACC) tot[threadIdx.x] = v;
+  __syncthreads();
+  if (threadIdx.x == 0)
+    fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh);
+  __syncthreads();
+
+  for (long long vv = threadIdx.x; vv < nvec; vv += blockDim.x) {
+    const size_t x = (size_t)vv * 4;
+    float c[M][4], rv[4];
+    logreg_diffs<M>(X, rowoff, coef, m, x, c);
+    ld4_r(r + x, rv);
+    double a4[4] = {(double)rv[0], (double)rv[1], (double)rv[2], (double)rv[3]};
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+      if (i < m) {
+        const float s = ssh[i];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) a4[j] += (double)(s * c[i][j]);
+      }
+    }
+    *reinterpret_cast<float4 *>(r + x) = make_float4((float)a4[0], (float)a4[1], (float)a4[2], (float)a4[3]);
+  }
+}
+
+template <int M>
+static cudaError_t launch_fused_logreg_t(cdgrab_ctx *h, const float *X, const float *y, const float *w,
+                                         cudaStream_t st) {
+  constexpr int WARPS = FusedCfg<M>::THREADS / 32;
+  const size_t smem = (WARPS * Tri<M>::NPAD + Tri<M>::NPAD) * sizeof(double) + (M + 4 * M) * sizeof(float) +
+                      2 * M * sizeof(size_t) + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(fused_logreg_step_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  {
+    CdgProfScope ps(h, CDGRAB_K_FUSED, st);
+    fused_logreg_step_kernel<M><<<1, FusedCfg<M>::THREADS, smem, st>>>(
+        X, y, w, h->r, h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs, h->margins, h->rnorm2,
+        h->status, cdg_rule_of(h));
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t cdg_launch_fused_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w, cudaStream_t st) {
+  const int M = h->m <= 4 ? 4 : (h->m <= 8 ? 8 : 16);
+  if (M == 4) return launch_fused_logreg_t<4>(h, X, y, w, st);
+  if (M == 8) return launch_fused_logreg_t<8>(h, X, y, w, st);
+  return launch_fused_logreg_t<16>(h, X, y, w, st);
 }
 
 // ------------------------------------------------------------------------------------
