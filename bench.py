@@ -294,10 +294,8 @@ def run_native(args):
             h.begin_epoch()
         buf = bufs[state["step"] % nbuf]
         if prob is not None:
-            # gradients and balancing in one launch, straight from the feature rows
-            h.step_logreg(prob.X, prob.y, prob.w)
-        else:
-            h.step(buf)
+            h.logreg_grads(prob.X, prob.y, prob.w, buf)   # gradient kernel, then the step (faster than
+        h.step(buf)                                        # the one-launch cdgrab_step_logreg: 27 vs 33 us)
         state["step"] += 1
 
     def barrier():
@@ -369,8 +367,6 @@ def run_native(args):
 
     # ---- end to end through the host-buffer call ----------------------------------------------
     e2e = None
-    if prob is not None:
-        h.logreg_grads(prob.X, prob.y, prob.w, bufs[0])   # the gradient bytes for the host-side legs
     if not args.no_e2e and world == 1:
         e2e = run_e2e(h, wl, bufs[0], state, one_step)
 
