@@ -198,6 +198,17 @@ int cdgrab_clear_status(cdgrab_t *h);
  */
 int cdgrab_selftest_wait_timeout(cdgrab_t *h, long long cycles, long long *waited_cycles);
 
+/*
+ * Checkpoint / resume.  cdgrab_save_state copies everything a handle needs to continue (epoch
+ * position, running sum(s), both permutation tables, signs, margins) into host_buf (HOST, at
+ * least cdgrab_state_bytes(h) bytes); cdgrab_load_state puts it into a handle created with the
+ * same m, n, d, dtype and mode (else CDGRAB_ERR_INVALID), in or between epochs.  Both are
+ * synchronous.  A run continued from a loaded state gives bit-identical results.
+ */
+long long cdgrab_state_bytes(const cdgrab_t *h);
+int cdgrab_save_state(cdgrab_t *h, void *host_buf, long long bytes);
+int cdgrab_load_state(cdgrab_t *h, const void *host_buf, long long bytes);
+
 /* Code path the handle uses (CDGRAB_PATH_*).  The environment variable
  * CDGRAB_FORCE_PATH = fused | fma | umma, read at create time, overrides the automatic
  * choice when the forced path supports the shape; otherwise create fails with

@@ -42,6 +42,9 @@ SIGNATURES = {
     "cdgrab_status": (C.c_int, [C.c_void_p]),
     "cdgrab_clear_status": (C.c_int, [C.c_void_p]),
     "cdgrab_selftest_wait_timeout": (C.c_int, [C.c_void_p, C.c_longlong, C.POINTER(C.c_longlong)]),
+    "cdgrab_state_bytes": (C.c_longlong, [C.c_void_p]),
+    "cdgrab_save_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_longlong]),
+    "cdgrab_load_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_longlong]),
     "cdgrab_path": (C.c_int, [C.c_void_p]),
     "cdgrab_launch_count": (C.c_longlong, [C.c_void_p]),
     "cdgrab_strerror": (C.c_char_p, [C.c_int]),
@@ -212,6 +215,17 @@ class CdGrab:
     def next_perms(self):
         import torch
         return self._fetch("cdgrab_get_next_perms", (self.m, self.n), torch.int32)
+
+    def save_state(self):
+        """Host copy (numpy uint8 array) of everything needed to continue in another handle."""
+        import numpy as np
+        nbytes = int(lib().cdgrab_state_bytes(self._h))
+        buf = np.empty(nbytes, dtype=np.uint8)
+        _check(lib().cdgrab_save_state(self._h, buf.ctypes.data, nbytes), "cdgrab_save_state")
+        return buf
+
+    def load_state(self, buf):
+        _check(lib().cdgrab_load_state(self._h, buf.ctypes.data, int(buf.nbytes)), "cdgrab_load_state")
 
     def status(self) -> int:
         return lib().cdgrab_status(self._h)

@@ -441,6 +441,77 @@ int cdgrab_clear_status(cdgrab_t *h) {
   return CDGRAB_OK;
 }
 
+// ---- checkpoint / resume -----------------------------------------------------------------
+namespace {
+struct StateHeader {
+  uint32_t magic;
+  int m, n, dtype, independent, k, epoch_open;
+  long long d;
+  double rnorm2;
+  unsigned long long oob;
+};
+struct StateSizes { size_t r, perm, signs, margins, total; };
+StateSizes state_sizes(const cdgrab_ctx *h) {
+  StateSizes z;
+  z.r = sizeof(float) * (size_t)h->d * (h->independent ? (size_t)h->m : 1);
+  z.perm = sizeof(int32_t) * (size_t)h->m * h->n;
+  z.signs = (size_t)h->m * (h->n / 2);
+  z.margins = sizeof(float) * (size_t)h->m * (h->n / 2);
+  z.total = sizeof(StateHeader) + z.r + 2 * z.perm + z.signs + z.margins;
+  return z;
+}
+}  // namespace
+
+long long cdgrab_state_bytes(const cdgrab_t *h) { return valid(h) ? (long long)state_sizes(h).total : CDGRAB_ERR_INVALID; }
+
+int cdgrab_save_state(cdgrab_t *h, void *host_buf, long long bytes) {
+  if (!valid(h) || !host_buf) return CDGRAB_ERR_INVALID;
+  const StateSizes z = state_sizes(h);
+  if (bytes < (long long)z.total) return CDGRAB_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  StateHeader hd;
+  memset(&hd, 0, sizeof(hd));
+  hd.magic = CDG_MAGIC; hd.m = h->m; hd.n = h->n; hd.dtype = h->dtype; hd.independent = h->independent;
+  hd.k = h->k; hd.epoch_open = h->epoch_open; hd.d = h->d;
+  char *p = (char *)host_buf + sizeof(StateHeader);
+  bool ok = cudaMemcpy(&hd.rnorm2, h->rnorm2, sizeof(double), cudaMemcpyDeviceToHost) == cudaSuccess;
+  ok = ok && cudaMemcpy(&hd.oob, h->oob, sizeof(hd.oob), cudaMemcpyDeviceToHost) == cudaSuccess;
+  ok = ok && cudaMemcpy(p, h->r, z.r, cudaMemcpyDeviceToHost) == cudaSuccess; p += z.r;
+  ok = ok && cudaMemcpy(p, h->perm_cur, z.perm, cudaMemcpyDeviceToHost) == cudaSuccess; p += z.perm;
+  ok = ok && cudaMemcpy(p, h->perm_next, z.perm, cudaMemcpyDeviceToHost) == cudaSuccess; p += z.perm;
+  ok = ok && cudaMemcpy(p, h->signs, z.signs, cudaMemcpyDeviceToHost) == cudaSuccess; p += z.signs;
+  ok = ok && cudaMemcpy(p, h->margins, z.margins, cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  memcpy(host_buf, &hd, sizeof(hd));
+  return CDGRAB_OK;
+}
+
+int cdgrab_load_state(cdgrab_t *h, const void *host_buf, long long bytes) {
+  if (!valid(h) || !host_buf) return CDGRAB_ERR_INVALID;
+  const StateSizes z = state_sizes(h);
+  if (bytes < (long long)z.total) return CDGRAB_ERR_INVALID;
+  StateHeader hd;
+  memcpy(&hd, host_buf, sizeof(hd));
+  if (hd.magic != CDG_MAGIC || hd.m != h->m || hd.n != h->n || hd.d != h->d || hd.dtype != h->dtype ||
+      hd.independent != h->independent || hd.k < 0 || hd.k > h->n / 2)
+    return CDGRAB_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  const char *p = (const char *)host_buf + sizeof(StateHeader);
+  bool ok = cudaMemcpy(h->rnorm2, &hd.rnorm2, sizeof(double), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(h->oob, &hd.oob, sizeof(hd.oob), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(h->r, p, z.r, cudaMemcpyHostToDevice) == cudaSuccess; p += z.r;
+  ok = ok && cudaMemcpy(h->perm_cur, p, z.perm, cudaMemcpyHostToDevice) == cudaSuccess; p += z.perm;
+  ok = ok && cudaMemcpy(h->perm_next, p, z.perm, cudaMemcpyHostToDevice) == cudaSuccess; p += z.perm;
+  ok = ok && cudaMemcpy(h->signs, p, z.signs, cudaMemcpyHostToDevice) == cudaSuccess; p += z.signs;
+  ok = ok && cudaMemcpy(h->margins, p, z.margins, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cdg_launch_split_r(h, nullptr) == cudaSuccess;
+  ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->k = hd.k;
+  h->epoch_open = hd.epoch_open;
+  return CDGRAB_OK;
+}
+
 int cdgrab_path(const cdgrab_t *h) { return valid(h) ? h->path : CDGRAB_ERR_INVALID; }
 
 long long cdgrab_launch_count(const cdgrab_t *h) { return valid(h) ? h->launches : -1; }

@@ -455,6 +455,27 @@ cudaError_t cdg_launch_mean(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// r -> its exact three-way bf16 split (after a state load on the tensor-core path)
+__global__ void split_r_kernel(const float *__restrict__ r, long long d, long long d_pad,
+                               __nv_bfloat16 *__restrict__ r_split) {
+  const long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (x >= d) return;
+  const float v = r[x];
+  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(hi);
+  const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+  r_split[x] = hi;
+  r_split[(size_t)d_pad + x] = mid;
+  r_split[2 * (size_t)d_pad + x] = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+}
+
+cudaError_t cdg_launch_split_r(cdgrab_ctx *h, cudaStream_t st) {
+  if (!h->r_split) return cudaSuccess;
+  split_r_kernel<<<(unsigned)((h->d + 255) / 256), 256, 0, st>>>(h->r, h->d, h->d_pad, h->r_split);
+  h->launches++;
+  return cudaGetLastError();
+}
+
 cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,
                               float *out, cudaStream_t st) {
   dim3 grid(h->m, 2);
