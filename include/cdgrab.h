@@ -86,6 +86,26 @@ int cdgrab_create_independent(int m, int n, long long d, int dtype, cdgrab_t **o
 /* Running sum of one worker of an independent-mode handle: out is HOST or DEVICE float [d]. */
 int cdgrab_get_r_worker(cdgrab_t *h, int worker, float *out, void *stream);
 
+/*
+ * Column-sharded order server (the direction the paper's conclusion calls an order server; the
+ * method reduces over d, so it shards over d with one small exchange per step).  Each shard -- a
+ * GPU, or a slice on one GPU -- owns d_local consecutive columns of every gradient row and of r.
+ * Per step:
+ *   cdgrab_step_begin  (every shard)  pass 1 over the shard's columns; its partial G = C^T C and
+ *                      b = C^T r land in gram_out_dev: DEVICE double [m*m + m], caller-owned
+ *   the caller sums those m*m + m doubles over all shards (e.g. one NCCL all-reduce) so that
+ *   every shard holds the same totals
+ *   cdgrab_step_finish (every shard)  the m decisions of Algorithm 6 on the totals -- identical on
+ *                      every shard -- then the update of the shard's slice of r
+ * grads_dev is the shard's slice [2][m][d_local] (contiguous), the same buffer in both calls.
+ * All other calls (begin/end_epoch, get_*, set_perms) work as usual on each shard; signs and
+ * permutations come out identical everywhere.  cdgrab_step itself, the randomized rule and the
+ * fused average are not available on a shard handle.
+ */
+int cdgrab_create_shard(int m, int n, long long d_local, int dtype, cdgrab_t **out);
+int cdgrab_step_begin(cdgrab_t *h, const void *grads_dev, double *gram_out_dev, void *stream);
+int cdgrab_step_finish(cdgrab_t *h, const void *grads_dev, const double *gram_in_dev, void *stream);
+
 /* Free the handle and everything it owns.  Synchronises the device.  NULL is allowed. */
 int cdgrab_destroy(cdgrab_t *h);
 

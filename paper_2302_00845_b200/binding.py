@@ -26,6 +26,9 @@ SIGNATURES = {
     "cdgrab_create": (C.c_int, [C.c_int, C.c_int, C.c_longlong, C.c_int, C.POINTER(C.c_void_p)]),
     "cdgrab_create_independent": (C.c_int, [C.c_int, C.c_int, C.c_longlong, C.c_int, C.POINTER(C.c_void_p)]),
     "cdgrab_get_r_worker": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]),
+    "cdgrab_create_shard": (C.c_int, [C.c_int, C.c_int, C.c_longlong, C.c_int, C.POINTER(C.c_void_p)]),
+    "cdgrab_step_begin": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "cdgrab_step_finish": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_destroy": (C.c_int, [C.c_void_p]),
     "cdgrab_set_perms": (C.c_int, [C.c_void_p, C.c_void_p]),
     "cdgrab_begin_epoch": (C.c_int, [C.c_void_p, C.c_void_p]),
@@ -110,10 +113,13 @@ def _ptr(t):
 class CdGrab:
     """Order-server state for m workers x n items in R^d (see ``include/cdgrab.h``)."""
 
-    def __init__(self, m: int, n: int, d: int, dtype: str | int = "f32", independent: bool = False):
+    def __init__(self, m: int, n: int, d: int, dtype: str | int = "f32", independent: bool = False,
+                 shard: bool = False):
         code = {"f32": F32, "bf16": BF16}.get(dtype, dtype)
         h = C.c_void_p()
-        if independent:   # ID-GraB (PairBal): one running sum per worker
+        if shard:         # one column shard of a coordinated order: d is the shard's width
+            _check(lib().cdgrab_create_shard(m, n, d, code, C.byref(h)), "cdgrab_create_shard")
+        elif independent:   # ID-GraB (PairBal): one running sum per worker
             _check(lib().cdgrab_create_independent(m, n, d, code, C.byref(h)), "cdgrab_create_independent")
         else:
             _check(lib().cdgrab_create(m, n, d, code, C.byref(h)), "cdgrab_create")
@@ -157,6 +163,16 @@ class CdGrab:
     @property
     def out_of_bound(self) -> int:
         return int(lib().cdgrab_out_of_bound(self._h))
+
+    def step_begin(self, grads, gram_out, stream=None):
+        """Shard handle: pass 1; gram_out is a CUDA float64 tensor [m*m + m] for the partial (G, b)."""
+        _check(lib().cdgrab_step_begin(self._h, _ptr(grads), _ptr(gram_out), _stream_ptr(stream)),
+               "cdgrab_step_begin")
+
+    def step_finish(self, grads, gram_in, stream=None):
+        """Shard handle: decisions on the summed (G, b) and the update of this shard's slice of r."""
+        _check(lib().cdgrab_step_finish(self._h, _ptr(grads), _ptr(gram_in), _stream_ptr(stream)),
+               "cdgrab_step_finish")
 
     def step_mean(self, grads, mean_out, stream=None):
         """step() that also writes the average of each gather buffer into mean_out (CUDA float32 [2][d])."""
@@ -275,3 +291,33 @@ def herding_objective(z, perms, stream=None) -> float:
     _check(lib().cdgrab_herding_objective(_ptr(z), _ptr(perms), m, n, d, _ptr(ws), nbytes, _ptr(out),
                                           _stream_ptr(stream)), "cdgrab_herding_objective")
     return float(out.item())
+
+
+class ShardedCdGrab:
+    """One rank of a column-sharded order server over ``torch.distributed``: this rank owns
+    d_local columns; every step all-reduces m*m + m doubles (NCCL on GPUs)."""
+
+    def __init__(self, m: int, n: int, d_local: int, dtype="f32", group=None, handle=None,
+                 device="cuda"):
+        """``handle``: an object with step_begin / step_finish / begin_epoch / end_epoch / destroy
+        to drive instead of a new shard handle (host-side tests of the exchange)."""
+        import torch
+        self.h = handle if handle is not None else CdGrab(m, n, d_local, dtype, shard=True)
+        self.group = group
+        self.gram = torch.empty(m * m + m, dtype=torch.float64, device=device)
+
+    def begin_epoch(self):
+        self.h.begin_epoch()
+
+    def step(self, grads_local):
+        import torch.distributed as dist
+        self.h.step_begin(grads_local, self.gram)
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(self.group) > 1:
+            dist.all_reduce(self.gram, op=dist.ReduceOp.SUM, group=self.group)
+        self.h.step_finish(grads_local, self.gram)
+
+    def end_epoch(self, perms_out=None):
+        self.h.end_epoch(perms_out)
+
+    def destroy(self):
+        self.h.destroy()

@@ -75,7 +75,7 @@ const char *cdgrab_strerror(int code) {
   }
 }
 
-static int create_impl(int m, int n, long long d, int dtype, int independent, cdgrab_t **out);
+static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t **out);
 
 int cdgrab_create(int m, int n, long long d, int dtype, cdgrab_t **out) {
   return create_impl(m, n, d, dtype, 0, out);
@@ -85,7 +85,15 @@ int cdgrab_create_independent(int m, int n, long long d, int dtype, cdgrab_t **o
   return create_impl(m, n, d, dtype, 1, out);
 }
 
-static int create_impl(int m, int n, long long d, int dtype, int independent, cdgrab_t **out) {
+int cdgrab_create_shard(int m, int n, long long d_local, int dtype, cdgrab_t **out) {
+  return create_impl(m, n, d_local, dtype, 2, out);
+}
+
+// mode 0: coordinated order on one device; 1: independent workers; 2: one column shard of a
+// coordinated order (split steps, never the single-launch paths)
+static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t **out) {
+  const int independent = (mode == 1);
+  const int shard = (mode == 2);
   if (!out) return CDGRAB_ERR_INVALID;
   *out = nullptr;
   if (m < 1 || m > 1024 || n < 2 || (n & 1) || d < 1) return CDGRAB_ERR_INVALID;
@@ -107,6 +115,7 @@ static int create_impl(int m, int n, long long d, int dtype, int independent, cd
   h->m = m; h->n = n; h->d = d; h->dtype = dtype;
   h->device = dev; h->num_sms = prop.multiProcessorCount;
   h->independent = independent;
+  h->shard = shard;
 
   // ---- choose the path ------------------------------------------------------------
   const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);
@@ -114,12 +123,12 @@ static int create_impl(int m, int n, long long d, int dtype, int independent, cd
   const bool umma_ok = cdg_umma_supported(m, d, dtype);
   int path;
   if (forced == CDGRAB_PATH_AUTO) {
-    if (fused_ok && step_bytes <= (size_t)768 * 1024) path = CDGRAB_PATH_FUSED;
+    if (fused_ok && step_bytes <= (size_t)768 * 1024 && !shard) path = CDGRAB_PATH_FUSED;
     else if (umma_ok && !fma_columns_ok(h)) path = CDGRAB_PATH_UMMA;
     else path = CDGRAB_PATH_FMA;
   } else {
     path = forced;
-    if ((path == CDGRAB_PATH_FUSED && !fused_ok) || (path == CDGRAB_PATH_UMMA && !umma_ok)) {
+    if ((path == CDGRAB_PATH_FUSED && (!fused_ok || shard)) || (path == CDGRAB_PATH_UMMA && !umma_ok)) {
       delete h;
       return CDGRAB_ERR_INVALID;
     }
@@ -186,6 +195,7 @@ static int create_impl(int m, int n, long long d, int dtype, int independent, cd
     if (!(e && e[0] == '0')) {
       const int rc = cdg_fma_tma_setup(h);
       if (rc != CDGRAB_OK) { free_all(h); delete h; return rc; }
+      if (shard) h->fma_tma_fused = 0;   // the decisions wait for the sum over all shards
     }
   }
 
@@ -259,9 +269,44 @@ int cdgrab_begin_epoch(cdgrab_t *h, void *stream) {
   return CDGRAB_OK;
 }
 
+static cudaError_t launch_pass1(cdgrab_ctx *h, const void *grads_dev, cudaStream_t st) {
+  if (h->path == CDGRAB_PATH_UMMA) return cdg_launch_gram_umma(h, grads_dev, st);
+  if (h->fma_tma) return cdg_launch_gram_fma_tma(h, grads_dev, st);
+  if (fma_columns_ok(h)) return cdg_launch_gram_fma(h, grads_dev, st);
+  return cdg_launch_gram_generic(h, grads_dev, st);
+}
+
+int cdgrab_step_begin(cdgrab_t *h, const void *grads_dev, double *gram_out_dev, void *stream) {
+  if (!valid(h) || !grads_dev || !gram_out_dev || !h->shard) return CDGRAB_ERR_INVALID;
+  if ((((uintptr_t)grads_dev & 15) | ((uintptr_t)gram_out_dev & 7)) != 0) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || h->k >= h->n / 2 || h->shard_pending) return CDGRAB_ERR_STATE;
+  double *own = h->gram;
+  h->gram = gram_out_dev;                       // pass 1 leaves this shard's partial (G, b) there
+  const cudaError_t e = launch_pass1(h, grads_dev, (cudaStream_t)stream);
+  h->gram = own;
+  if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->shard_pending = 1;
+  return CDGRAB_OK;
+}
+
+int cdgrab_step_finish(cdgrab_t *h, const void *grads_dev, const double *gram_in_dev, void *stream) {
+  if (!valid(h) || !grads_dev || !gram_in_dev || !h->shard) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || !h->shard_pending) return CDGRAB_ERR_STATE;
+  double *own = h->gram;
+  h->gram = const_cast<double *>(gram_in_dev);  // the sum over all shards
+  cudaError_t e = cdg_launch_scan(h, (cudaStream_t)stream);
+  h->gram = own;
+  if (e == cudaSuccess) e = cdg_launch_update(h, grads_dev, (cudaStream_t)stream);
+  if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->shard_pending = 0;
+  h->k++;
+  return CDGRAB_OK;
+}
+
 int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   if (!valid(h) || !grads_dev) return CDGRAB_ERR_INVALID;
   if (((uintptr_t)grads_dev & 15) != 0) return CDGRAB_ERR_INVALID;
+  if (h->shard) return CDGRAB_ERR_INVALID;   // a shard steps through cdgrab_step_begin / _finish
   if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
@@ -271,10 +316,7 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   } else if (h->path == CDGRAB_PATH_FUSED) {
     e = cdg_launch_fused(h, grads_dev, st);
   } else {
-    if (h->path == CDGRAB_PATH_UMMA) e = cdg_launch_gram_umma(h, grads_dev, st);
-    else if (h->fma_tma) e = cdg_launch_gram_fma_tma(h, grads_dev, st);
-    else if (fma_columns_ok(h)) e = cdg_launch_gram_fma(h, grads_dev, st);
-    else e = cdg_launch_gram_generic(h, grads_dev, st);
+    e = launch_pass1(h, grads_dev, st);
     if (e == cudaSuccess && !(h->fma_tma && h->fma_tma_fused)) e = cdg_launch_scan(h, st);
     if (e == cudaSuccess) e = cdg_launch_update(h, grads_dev, st);
   }
@@ -335,7 +377,7 @@ int cdgrab_step_host(cdgrab_t *h, const void *grads_host, void *staging_dev, voi
 
 int cdgrab_end_epoch(cdgrab_t *h, int32_t *perms_out, void *stream) {
   if (!valid(h)) return CDGRAB_ERR_INVALID;
-  if (!h->epoch_open || h->k != h->n / 2) return CDGRAB_ERR_STATE;
+  if (!h->epoch_open || h->k != h->n / 2 || h->shard_pending) return CDGRAB_ERR_STATE;
   int32_t *t = h->perm_cur; h->perm_cur = h->perm_next; h->perm_next = t;
   h->epoch_open = 0;
   if (perms_out) return copy_out(perms_out, h->perm_cur, sizeof(int32_t) * (size_t)h->m * h->n, stream);

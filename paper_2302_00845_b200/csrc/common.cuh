@@ -39,6 +39,8 @@ struct cdgrab_ctx {
   int *status;           // [1] device status word
   double *gram;          // [m*m + m] G (row-major) then b
   double *partials;      // pass-1 partial sums
+  int shard;             // 1: this handle holds one column shard (split steps)
+  int shard_pending;     // step_begin issued, step_finish outstanding
   int independent;       // 1: ID-GraB mode, r is [m][d] (one running sum per worker)
   int rule_randomized;   // balance rule of the step being enqueued (0: greedy)
   const float *rule_u;   // [m] uniforms for the randomized rule

@@ -82,3 +82,49 @@ def test_algorithmic_bytes_model():
     assert bench.algorithmic_bytes("gram", wl) == inp + 4 * 124_000_000
     assert bench.algorithmic_bytes("update", wl) == inp + 8 * 124_000_000
     assert inp == 31_744_000_000
+
+
+class _FakeShard:
+    """Stands in for a shard handle: its partial sums are a known function of the rank."""
+
+    def __init__(self, rank):
+        self.rank, self.seen = rank, []
+
+    def begin_epoch(self):
+        pass
+
+    def step_begin(self, grads, gram):
+        gram.copy_(torch.arange(gram.numel(), dtype=torch.float64) * (self.rank + 1))
+
+    def step_finish(self, grads, gram):
+        self.seen.append(gram.clone())
+
+
+def _shard_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2302_00845_b200 import binding
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    m = 3
+    fake = _FakeShard(rank)
+    sh = binding.ShardedCdGrab(m, 4, 16, "f32", handle=fake, device="cpu")
+    sh.begin_epoch()
+    sh.step(None)
+    sh.step(None)
+    out[rank] = [t.tolist() for t in fake.seen]
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_wrapper_all_reduces_the_partial_sums_world_size_2_gloo():
+    ctx = mp.get_context("spawn")
+    out = ctx.Manager().dict()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_shard_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    want = [3.0 * i for i in range(3 * 3 + 3)]          # rank 0 gives i, rank 1 gives 2 i
+    assert out[0] == [want, want] and out[1] == out[0]  # both ranks finish on the same bits
