@@ -583,6 +583,25 @@ __device__ __forceinline__ void ft_consume(const T *gt, const float *rt, int m, 
   }
 }
 
+// Local entry (group, l) -> entry of the full triangle (row-major pairs a <= b, then b); -1: padding.
+template <int M>
+struct SplitMap {
+  short v[2][Split<M>::NLPAD];
+  constexpr SplitMap() : v{} {
+    for (int g = 0; g < 2; ++g)
+      for (int l = 0; l < Split<M>::NLPAD; ++l) v[g][l] = -1;
+    int cnt[2] = {0, 0}, e = 0;
+    for (int a = 0; a < M; ++a)
+      for (int b = a; b < M; ++b) {
+        const int g = Split<M>::owner(a, b);
+        v[g][cnt[g]++] = (short)e++;
+      }
+    for (int a = 0; a < M; ++a) v[1][Split<M>::count(1) + a] = (short)(Tri<M>::NPAIR + a);
+  }
+};
+template <int M>
+__constant__ SplitMap<M> kSplitMap = SplitMap<M>();
+
 // When enabled, the last CTA to finish also runs the scalar part of the step.
 struct FtTail {
   int enabled;
@@ -605,7 +624,6 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   __shared__ __align__(8) uint64_t bar_full[kFtMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kFtMaxStages];
   __shared__ double red[16 * Split<M>::NLPAD];      // [warp][local entry]
-  __shared__ short lmap[2][Split<M>::NLPAD];        // local entry -> entry of the full triangle (-1: padding)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = warp >> 3;                       // 0, 1: compute groups; 2: producer
@@ -629,24 +647,6 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     }
     mbar_init_fence();
   }
-  if (threadIdx.x < 2 * Split<M>::NLPAD) (&lmap[0][0])[threadIdx.x] = -1;
-  __syncthreads();
-  if (threadIdx.x < Tri<M>::NACC) {
-    // entry e of the triangle -> (group, local index): count the same-group entries before it
-    const int e = threadIdx.x;
-    if (e < Tri<M>::NPAIR) {
-      int a = 0, rem = e;
-      while (rem >= M - a) { rem -= M - a; ++a; }
-      const int b = a + rem, g = Split<M>::owner(a, b);
-      int l = 0;
-      for (int x = 0; x < M; ++x)
-        for (int y = x; y < M; ++y)
-          if ((x < a || (x == a && y < b)) && Split<M>::owner(x, y) == g) ++l;
-      lmap[g][l] = (short)e;
-    } else {
-      lmap[1][Split<M>::count(1) + (e - Tri<M>::NPAIR)] = (short)e;
-    }
-  }
   __syncthreads();
   const long long deadline = clock64() + kCdgWaitCycles;
 
@@ -654,7 +654,15 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
 #pragma unroll
   for (int e = 0; e < Split<M>::NLPAD; ++e) acc[e] = 0.f;
 
+  // what the scalar tail will need, fetched now by idle lanes of the producer warp
+  int32_t pf_first = 0, pf_second = 0;
+  double pf_rn2 = 0.0;
   if (group == 2) {
+    if (tail.enabled && lane >= 1 && lane <= m) {
+      pf_first = tail.perm_cur[(size_t)(lane - 1) * tail.n + 2 * tail.k];
+      pf_second = tail.perm_cur[(size_t)(lane - 1) * tail.n + 2 * tail.k + 1];
+    }
+    if (tail.enabled && lane == 17) pf_rn2 = *tail.rnorm2;
     if (lane == 0) {
       int issued = 0;
       bool ok = true;
@@ -702,7 +710,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   // thread (g, l): add the 8 warps of group g in warp order, store under the triangle's entry
   if (threadIdx.x < 2 * Split<M>::NLPAD) {
     const int g = threadIdx.x / Split<M>::NLPAD, l = threadIdx.x % Split<M>::NLPAD;
-    const int e = lmap[g][l];
+    const int e = kSplitMap<M>.v[g][l];
     if (e >= 0) {
       double v = 0.0;
 #pragma unroll
@@ -728,16 +736,31 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   double *sh = reinterpret_cast<double *>(base_ptr);
   const ScanSmem S = scan_smem(sh, m);
   double *slices = S.g + (size_t)m * m;                       // [3][NPAD] block-list slices
+  double *rn2_sh = slices + 3 * Tri<M>::NPAD;
   constexpr int NP = Tri<M>::NPAD;
   if (threadIdx.x < 3 * NP) {
     // slice p adds blocks p, p+3, ... in that order; the slices are then added in order
     const int e = threadIdx.x % NP, p = threadIdx.x / NP;
     double v = 0.0;
     if (e < Tri<M>::NACC) {
-#pragma unroll 8
-      for (int b = p; b < (int)gridDim.x; b += 3) v += __ldcg(partials + (size_t)b * Tri<M>::NACC + e);
+#pragma unroll 1
+      for (int b0 = p; b0 < (int)gridDim.x; b0 += 3 * 26) {
+        double x[26];            // all loads of a batch in flight before the first add
+#pragma unroll
+        for (int q = 0; q < 26; ++q) {
+          const int b = b0 + 3 * q;
+          x[q] = (b < (int)gridDim.x) ? __ldcg(partials + (size_t)b * Tri<M>::NACC + e) : 0.0;
+        }
+#pragma unroll
+        for (int q = 0; q < 26; ++q)
+          if (b0 + 3 * q < (int)gridDim.x) v += x[q];
+      }
     }
     slices[p * NP + e] = v;
+  }
+  if (group == 2) {
+    if (lane >= 1 && lane <= m) { S.p[2 * (lane - 1)] = pf_first; S.p[2 * (lane - 1) + 1] = pf_second; }
+    if (lane == 17) *rn2_sh = pf_rn2;
   }
   __syncthreads();
   if (threadIdx.x < Tri<M>::NACC) {
@@ -753,11 +776,10 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       if (a < m) S.t[a] = v;
     }
   }
-  scan_load_pairs(S, tail.perm_cur, m, tail.n, tail.k);
   if (threadIdx.x == 0) *tail.ticket = 0u;                    // ready for the next launch
   __syncthreads();
   scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
-                        tail.rule);
+                        tail.rule, *rn2_sh);
 }
 
 bool cdg_fma_tma_supported(int m, long long d, int dtype) {

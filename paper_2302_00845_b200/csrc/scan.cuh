@@ -66,29 +66,60 @@ __device__ __forceinline__ void scan_load_pairs(const ScanSmem &S, const int32_t
 
 // S.t = b, S.p = pairs and G (shared or global, row-major [m][m]) must be ready and visible
 // to the block (barrier before the call).  Warp 0 decides, the block writes out.
+// rn2_in: ||r||^2 before the step when the caller fetched it ahead of time, else negative
+// (the routine then reads *rnorm2 itself).
 __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const double *G, int m, int n, int k,
                                                       int32_t *__restrict__ perm_next, int8_t *__restrict__ signs,
                                                       float *__restrict__ margins, double *__restrict__ rnorm2,
-                                                      int *__restrict__ status, const CdgRule rule) {
+                                                      int *__restrict__ status, const CdgRule rule,
+                                                      double rn2_in = -1.0) {
   const int tid = threadIdx.x;
   if (tid < 32) {
     const int lane = tid;
-    double rn2 = *rnorm2;
+    double rn2 = (rn2_in >= 0.0) ? rn2_in : *rnorm2;
     bool bad = false;
     int oob = 0;
-    for (int i = 0; i < m; ++i) {
-      const double ti = S.t[i];
-      const double gii = G[(size_t)i * m + i];
-      // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0 (or the randomized rule)
-      const int s = cdg_decide(rule, i, ti, oob);
-      bad |= !(isfinite(ti) && isfinite(gii));
-      const double sd = (double)s;
-      // every later t_j gains s_i G_ij, summed in the order i = 0, 1, ...
-      for (int j = i + 1 + lane; j < m; j += 32) S.t[j] += sd * G[(size_t)i * m + j];
-      if (lane == 0) { S.s[i] = s; S.rn[i] = rn2; }
-      rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
-      if (rn2 < 0.0) rn2 = 0.0;
-      __syncwarp();
+    if (m <= 64) {
+      // The chain stays in registers: lane j holds t_j and t_{j+32}; row i of G is fetched one
+      // decision ahead, so a decision costs two shuffles and one multiply-add.
+      const bool h0 = lane < m, h1 = lane + 32 < m;
+      double t0 = h0 ? S.t[lane] : 0.0, t1 = h1 ? S.t[lane + 32] : 0.0;
+      double g0 = h0 ? G[lane] : 0.0, g1 = h1 ? G[lane + 32] : 0.0;
+      for (int i = 0; i < m; ++i) {
+        double n0 = 0.0, n1 = 0.0;
+        if (i + 1 < m) {
+          if (h0) n0 = G[(size_t)(i + 1) * m + lane];
+          if (h1) n1 = G[(size_t)(i + 1) * m + lane + 32];
+        }
+        const double ti = __shfl_sync(0xffffffffu, (i < 32) ? t0 : t1, i & 31);
+        const double gii = __shfl_sync(0xffffffffu, (i < 32) ? g0 : g1, i & 31);
+        // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0 (or the randomized rule)
+        const int s = cdg_decide(rule, i, ti, oob);
+        bad |= !(isfinite(ti) && isfinite(gii));
+        const double sd = (double)s;
+        // every later t_j gains s_i G_ij, summed in the order i = 0, 1, ...
+        if (lane > i) t0 += sd * g0;
+        if (lane + 32 > i) t1 += sd * g1;
+        if (lane == 0) { S.s[i] = s; S.rn[i] = rn2; }
+        rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
+        if (rn2 < 0.0) rn2 = 0.0;
+        g0 = n0; g1 = n1;
+      }
+      if (h0) S.t[lane] = t0;
+      if (h1) S.t[lane + 32] = t1;
+    } else {
+      for (int i = 0; i < m; ++i) {
+        const double ti = S.t[i];
+        const double gii = G[(size_t)i * m + i];
+        const int s = cdg_decide(rule, i, ti, oob);
+        bad |= !(isfinite(ti) && isfinite(gii));
+        const double sd = (double)s;
+        for (int j = i + 1 + lane; j < m; j += 32) S.t[j] += sd * G[(size_t)i * m + j];
+        if (lane == 0) { S.s[i] = s; S.rn[i] = rn2; }
+        rn2 += 2.0 * sd * ti + gii;
+        if (rn2 < 0.0) rn2 = 0.0;
+        __syncwarp();
+      }
     }
     if (lane == 0) {
       *rnorm2 = rn2;
