@@ -317,7 +317,8 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
     e = cdg_launch_fused(h, grads_dev, st);
   } else {
     e = launch_pass1(h, grads_dev, st);
-    if (e == cudaSuccess && !(h->fma_tma && h->fma_tma_fused)) e = cdg_launch_scan(h, st);
+    const bool decided = (h->path == CDGRAB_PATH_UMMA) ? h->umma_fused : (h->fma_tma && h->fma_tma_fused);
+    if (e == cudaSuccess && !decided) e = cdg_launch_scan(h, st);
     if (e == cudaSuccess) e = cdg_launch_update(h, grads_dev, st);
   }
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }

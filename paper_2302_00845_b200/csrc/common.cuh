@@ -74,7 +74,7 @@ struct cdgrab_ctx {
   float *umma_partials;    // [ctas][128][ncols]
   int umma_ctas;
   int umma_box_rows;       // rows of the gradient TMA box (2m rounded up to 16)
-  int umma_ncols;          // MMA N = box_rows + 16
+  int umma_ncols;          // columns of a partial H row = box_rows + 16
   int umma_subs_per_stage;
   int umma_drain;          // pipeline iterations per TMEM accumulation chunk
   int umma_stages;
@@ -84,6 +84,10 @@ struct cdgrab_ctx {
   const void *tm_g_base;   // gradient buffer the cached maps were encoded for
   CUtensorMap tm_g;        // 3-D map over the gradient rows
   CUtensorMap tm_g2;       // 2-D map over the gradient rows (ragged last block)
+  CUtensorMap tm_g4;       // 4-D map over the full 8-row groups of the gradient rows
+  int umma_g4;             // row groups one 4-D copy brings in (0: per-group copies only)
+  int umma_paired;         // 2m <= 64: one MMA covers two 64-column blocks
+  int umma_fused;          // the combine launch also takes the decisions (last block)
 };
 
 template <typename T>

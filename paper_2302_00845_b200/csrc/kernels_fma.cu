@@ -603,17 +603,7 @@ template <int M>
 __constant__ SplitMap<M> kSplitMap = SplitMap<M>();
 
 // When enabled, the last CTA to finish also runs the scalar part of the step.
-struct FtTail {
-  int enabled;
-  int n, k;
-  unsigned *ticket;          // zero between launches
-  const int32_t *perm_cur;
-  int32_t *perm_next;
-  int8_t *signs;
-  float *margins;
-  double *rnorm2;
-  CdgRule rule;
-};
+using FtTail = CdgTail;
 
 template <typename T, int M>
 __global__ void __launch_bounds__(kFtThreads, 1)
@@ -852,13 +842,7 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
 
 template <typename T, int M>
 static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, cudaStream_t st) {
-  FtTail tail;
-  tail.enabled = h->fma_tma_fused;
-  tail.n = h->n; tail.k = h->k;
-  tail.ticket = h->ticket;
-  tail.perm_cur = h->perm_cur; tail.perm_next = h->perm_next;
-  tail.signs = h->signs; tail.margins = h->margins; tail.rnorm2 = h->rnorm2;
-  tail.rule = cdg_rule_of(h);
+  const FtTail tail = cdg_tail_of(h, h->fma_tma_fused);
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     gram_fma_tma_kernel<T, M><<<h->gram_chunks, kFtThreads, h->fma_tma_smem, st>>>(

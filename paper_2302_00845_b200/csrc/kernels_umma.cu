@@ -30,6 +30,7 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "scan.cuh"
 
 namespace {
 
@@ -41,14 +42,16 @@ constexpr int kMaxCols = 144;            // MMA N at m = 64: 128 gradient rows +
 constexpr long long kWaitCycles = kCdgWaitCycles;
 
 struct UmmaParams {
-  int box_rows;        // gradient rows held per block (2m rounded up to 16)
-  int ncols;           // MMA N = box_rows + 16
+  int box_rows;        // gradient rows held per block (2m rounded up to 16; 64 when paired)
+  int ncols;           // columns of a partial H row = box_rows + 16 (MMA N, or half of it when paired)
   int rows_used;       // 2m
   int subs;            // 64-column blocks per stage
   int stages;
   long long nblk_full; // d / 64: blocks loaded by the 3-D maps
   int tail;            // 1 when d % 64 != 0: one more, ragged block
   int drain;           // pipeline iterations accumulated in TMEM before the sum is drained
+  int g4;              // full 8-row groups fetched by one 4-D copy (0: per-group copies only)
+  int paired;          // 2m <= 64: blocks j and j + subs/2 of a stage share one MMA (see the kernel)
 };
 
 // K-major, 128-byte swizzle: rows 128 B apart, 8-row groups `sbo` bytes apart
@@ -75,7 +78,7 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __global__ void __launch_bounds__(kThreads, 1)
 gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constant__ CUtensorMap tm_r3,
                  const __grid_constant__ CUtensorMap tm_g2, const __grid_constant__ CUtensorMap tm_r2,
-                 const UmmaParams p, float *__restrict__ partials, int *__restrict__ status) {
+                 const __grid_constant__ CUtensorMap tm_g4, const UmmaParams p, float *__restrict__ partials, int *__restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
@@ -85,14 +88,32 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-B alignment
-  const uint32_t group_bytes = (uint32_t)p.subs * 1024u;         // one row group of a stage
-  const int ngroups = p.ncols >> 3;
+  // Paired mode (2m <= 64).  With at most 64 gradient rows, half of a 128-row MMA would idle
+  // and the issue rate of the small MMAs, not HBM, would bound the kernel.  So one MMA takes two
+  // 64-column blocks at once: a stage is laid out as 20 row groups
+  //   [0..7] rows of block j | [8..15] rows of block j + subs/2 | [16] r of j | [17] 0 | [18] r of j' | [19] 0
+  // A = groups 0..15 (M = 128), B = all 20 (N = 160).  D rows 0..63 x columns 0..63 and 128..143
+  // hold block j's products, rows 64..127 x columns 64..127 and 144..159 block j''s; the other
+  // entries are cross terms nobody reads.
+  const int paired = p.paired;
+  const int hb = p.subs >> 1;                                    // blocks per half stage (paired)
+  const uint32_t group_bytes = (uint32_t)(paired ? hb : p.subs) * 1024u;   // one row group of a stage
+  const int ngroups = paired ? 20 : (p.ncols >> 3);
   const int ggroups = p.box_rows >> 3;                           // gradient row groups
   const uint32_t stage_bytes = group_bytes * ngroups;
 
-  // this CTA's K range in full blocks; the last CTA also owns the ragged block, taken first
-  const long long blk_lo = p.nblk_full * (long long)blockIdx.x / gridDim.x;
-  const long long blk_hi = p.nblk_full * (long long)(blockIdx.x + 1) / gridDim.x;
+  // this CTA's K range in full blocks; the last CTA also owns the ragged block, taken first.
+  // Paired: whole stages per CTA, so that both halves of a stage belong to the same CTA (blocks
+  // past the end of the rows are read as zeros).
+  long long blk_lo, blk_hi;
+  if (paired) {
+    const long long units = (p.nblk_full + p.subs - 1) / p.subs;
+    blk_lo = units * (long long)blockIdx.x / gridDim.x * p.subs;
+    blk_hi = units * (long long)(blockIdx.x + 1) / gridDim.x * p.subs;
+  } else {
+    blk_lo = p.nblk_full * (long long)blockIdx.x / gridDim.x;
+    blk_hi = p.nblk_full * (long long)(blockIdx.x + 1) / gridDim.x;
+  }
   const int has_tail = (p.tail && blockIdx.x == gridDim.x - 1) ? 1 : 0;
   const int n_iter = has_tail + (int)((blk_hi - blk_lo + p.subs - 1) / p.subs);
 
@@ -111,8 +132,9 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   // group after the r rows) are zeroed once
   const int lgroups = (p.rows_used + 7) >> 3;                    // gradient row groups that get loaded
   for (int s = 0; s < p.stages; ++s) {
-    for (int g = lgroups; g < ngroups; ++g) {
-      if (g == ggroups) continue;                                // the r rows
+    for (int g = 0; g < ngroups; ++g) {
+      const bool loaded = paired ? (g < 16 ? (g & 7) < lgroups : !(g & 1)) : (g < lgroups || g == ggroups);
+      if (loaded) continue;
       uint8_t *z = smem_raw + (tiles - smem_u32(smem_raw)) + (size_t)s * stage_bytes + (size_t)g * group_bytes;
       for (uint32_t o = threadIdx.x * 16; o < group_bytes; o += kThreads * 16)
         *reinterpret_cast<uint4 *>(z + o) = make_uint4(0, 0, 0, 0);
@@ -141,17 +163,37 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
         if (!ok) break;
         const uint32_t full = smem_u32(&bar_full[s]);
         const uint32_t base = tiles + s * stage_bytes;
+        const uint32_t rbase = base + (paired ? 16 : ggroups) * group_bytes;   // the r rows (first half)
         if (has_tail && it == 0) {
           // ragged block: 8-row 2-D boxes into block slot 0 of every loaded row group
           const int col = (int)(p.nblk_full * kSubCols);   // 128-byte aligned
-          mbar_expect_tx(full, (uint32_t)(lgroups + 1) * 1024u);
+          mbar_expect_tx(full, (uint32_t)(lgroups + 1) * (1024u + (paired ? group_bytes : 0u)));
           for (int g = 0; g < lgroups; ++g) tma_load_2d(base + g * group_bytes, &tm_g2, col, g * 8, full);
-          tma_load_2d(base + ggroups * group_bytes, &tm_r2, col, 0, full);
+          tma_load_2d(rbase, &tm_r2, col, 0, full);
+          if (paired) {
+            // the other half of the pair: blocks past the end, which the copies fill with zeros
+            const int past = (int)p.nblk_full;
+            const uint32_t hbase = base + 8 * group_bytes;
+            if (p.g4 > 0) tma_load_4d(hbase, &tm_g4, 0, 0, past, 0, full);
+            for (int g = p.g4; g < lgroups; ++g) tma_load_3d(hbase + g * group_bytes, &tm_g3, 0, g * 8, past, full);
+            tma_load_3d(rbase + 2 * group_bytes, &tm_r3, 0, 0, past, full);
+          }
+        } else if (paired) {
+          const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
+          mbar_expect_tx(full, 2u * (uint32_t)(lgroups + 1) * group_bytes);
+          for (int hf = 0; hf < 2; ++hf) {
+            const int blk = (int)(first + (long long)hf * hb);
+            const uint32_t hbase = base + hf * 8 * group_bytes;
+            if (p.g4 > 0) tma_load_4d(hbase, &tm_g4, 0, 0, blk, 0, full);
+            for (int g = p.g4; g < lgroups; ++g) tma_load_3d(hbase + g * group_bytes, &tm_g3, 0, g * 8, blk, full);
+            tma_load_3d(rbase + hf * 2 * group_bytes, &tm_r3, 0, 0, blk, full);
+          }
         } else {
           const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
           mbar_expect_tx(full, (uint32_t)(lgroups + 1) * group_bytes);
-          for (int g = 0; g < lgroups; ++g) tma_load_3d(base + g * group_bytes, &tm_g3, 0, g * 8, (int)first, full);
-          tma_load_3d(base + ggroups * group_bytes, &tm_r3, 0, 0, (int)first, full);
+          if (p.g4 > 0) tma_load_4d(base, &tm_g4, 0, 0, (int)first, 0, full);
+          for (int g = p.g4; g < lgroups; ++g) tma_load_3d(base + g * group_bytes, &tm_g3, 0, g * 8, (int)first, full);
+          tma_load_3d(rbase, &tm_r3, 0, 0, (int)first, full);
         }
         issued = it + 1;
       }
@@ -166,8 +208,8 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = ncols
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.ncols >> 3) << 17) |
-                             ((128u >> 4) << 24);
+      const uint32_t mma_n = paired ? 160u : (uint32_t)p.ncols;
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((mma_n >> 3) << 17) | ((128u >> 4) << 24);
       // The fp32 accumulation inside the tensor core truncates; over hundreds of thousands of
       // columns that becomes a visible bias on sums of same-sign products.  So the sum is kept
       // in TMEM only for `drain` iterations (about 1024 columns), then handed to the read-back
@@ -188,7 +230,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
         int cnt = 1;
         if (!(has_tail && it == 0)) {
           const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
-          cnt = (int)min((long long)p.subs, blk_hi - first);   // blocks past blk_hi belong to the next CTA
+          cnt = paired ? hb : (int)min((long long)p.subs, blk_hi - first);   // blocks past blk_hi belong to the next CTA
         }
         const uint32_t acc = tmem_acc + (uint32_t)buf * 256u;
         for (int q = 0; q < cnt; ++q) {
@@ -224,7 +266,9 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       for (int piece = 0; piece < kMaxCols / 16; ++piece) {
         if (piece * 16 < p.ncols) {
           uint32_t v[16];
-          const uint32_t taddr = tmem_acc + (uint32_t)buf * 256u + ((uint32_t)(lg * 32) << 16) + (uint32_t)(piece * 16);
+          // paired: rows 0..63 own D columns 0..63 and 128..143, rows 64..127 own 64..127 and 144..159
+          const int src = paired ? (piece < 4 ? piece + 4 * (lg >> 1) : 8 + (lg >> 1)) : piece;
+          const uint32_t taddr = tmem_acc + (uint32_t)buf * 256u + ((uint32_t)(lg * 32) << 16) + (uint32_t)(src * 16);
           asm volatile(
               "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
               "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -243,7 +287,21 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
     }
     if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
-    if (row < p.rows_used) {
+    if (paired) {
+      // rows 64..127 hold the same entries of H for the other block of each pair: add them to
+      // rows 0..63 through the (now idle) stage ring; only the four read-back warps take part
+      float *xch = reinterpret_cast<float *>(smem_raw + (tiles - smem_u32(smem_raw)));
+      if (lg >= 2) {
+#pragma unroll
+        for (int j = 0; j < 80; ++j) xch[(row & 63) * 81 + j] = accr[j];
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (lg < 2) {
+#pragma unroll
+        for (int j = 0; j < 80; ++j) accr[j] += xch[row * 81 + j];
+      }
+    }
+    if (row < p.rows_used && !(paired && lg >= 2)) {
       float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.ncols;
 #pragma unroll
       for (int piece = 0; piece < kMaxCols / 16; ++piece) {
@@ -271,8 +329,10 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
 // w, w+8, w+16, ... in that order, the eight warp sums are then added in warp order.
 __global__ void __launch_bounds__(256)
 umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows, int m,
-                    double *__restrict__ gram) {
+                    double *__restrict__ gram, int *__restrict__ status, const CdgTail tail) {
   __shared__ double part[8][32];
+  __shared__ double scan_sh[4 * 64 + 64 * 64];     // m <= 64 on this path
+  __shared__ int is_last;
   const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
   const int total = m * m + m;
   const int e = blockIdx.x * 32 + lane;
@@ -304,6 +364,23 @@ umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int
     for (int w = 0; w < 8; ++w) v += part[w][lane];
     gram[e] = v;
   }
+  if (!tail.enabled) return;
+
+  // ---- the block that takes the last ticket has all of (G, b) before it: it decides ----
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(tail.ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const ScanSmem S = scan_smem(scan_sh, m);
+  for (int j = threadIdx.x; j < m; j += blockDim.x) S.t[j] = __ldcg(gram + (size_t)m * m + j);
+  for (int q = threadIdx.x; q < m * m; q += blockDim.x) S.g[q] = __ldcg(gram + q);
+  scan_load_pairs(S, tail.perm_cur, m, tail.n, tail.k);
+  if (threadIdx.x == 0) *tail.ticket = 0u;                    // ready for the next launch
+  __syncthreads();
+  scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
+                        tail.rule);
 }
 
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
@@ -349,6 +426,20 @@ bool encode_map_3d(CUtensorMap *map, const void *base, long long nblk, int rows,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 4-D view {64 columns, 8 rows of a group, nblk blocks, groups} of the same memory; one box
+// {64, 8, blocks, groups} lands as [group][block][8 rows][128 B], the layout the per-group boxes build
+bool encode_map_4d(CUtensorMap *map, const void *base, long long nblk, int groups, long long pitch_elems, int blocks) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)kSubCols, 8, (cuuint64_t)nblk, (cuuint64_t)groups};
+  cuuint64_t strides[3] = {(cuuint64_t)pitch_elems * 2, (cuuint64_t)kSubCols * 2, (cuuint64_t)pitch_elems * 16};
+  cuuint32_t box[4] = {(cuuint32_t)kSubCols, 8, (cuuint32_t)blocks, (cuuint32_t)groups};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 // Self-test of the bounded wait every TMA-fed kernel here relies on: one thread waits on a
@@ -380,17 +471,23 @@ bool cdg_umma_supported(int m, long long d, int dtype) {
 }
 
 int cdg_umma_setup(cdgrab_ctx *h) {
-  const int box_rows = ((2 * h->m + 15) / 16) * 16;
+  h->umma_paired = (2 * h->m <= 64) ? 1 : 0;      // CDGRAB_UMMA_PAIRED=0: one block per MMA
+  if (const char *e = getenv("CDGRAB_UMMA_PAIRED")) {
+    if (atoi(e) == 0) h->umma_paired = 0;
+  }
+  const int box_rows = h->umma_paired ? 64 : ((2 * h->m + 15) / 16) * 16;
   h->umma_box_rows = box_rows;
   h->umma_ncols = box_rows + kRBoxRows;
   // 64-column blocks per stage: stages of roughly 70-80 KB measured best (4 blocks at m = 64,
   // 6-8 at m = 32); CDGRAB_UMMA_SUBS overrides
   int subs = 76 / (h->umma_ncols / 8);
   subs = subs < 2 ? 2 : (subs > 8 ? 8 : subs);
+  if (h->umma_paired) subs = 6;                  // three stages of 60 KB
   if (const char *e = getenv("CDGRAB_UMMA_SUBS")) {
     const int v = atoi(e);
-    if (v >= 1 && v <= 8) subs = v;
+    if (v >= 1 && v <= (h->umma_paired ? 10 : 8)) subs = v;
   }
+  if (h->umma_paired && (subs & 1)) ++subs;      // two halves per stage
   h->umma_subs_per_stage = subs;
   // TMEM chunk length in pipeline iterations (about 4096 columns); CDGRAB_UMMA_DRAIN overrides
   h->umma_drain = 4096 / (subs * kSubCols) > 0 ? 4096 / (subs * kSubCols) : 1;
@@ -398,9 +495,9 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     const int v = atoi(e);
     if (v >= 1 && v <= (1 << 20)) h->umma_drain = v;
   }
-  const size_t group_bytes = (size_t)subs * 1024;
-  const size_t stage_bytes = group_bytes * (h->umma_ncols / 8);
-  const int ngroups = h->umma_ncols / 8;
+  const size_t group_bytes = (size_t)(h->umma_paired ? subs / 2 : subs) * 1024;
+  const int ngroups = h->umma_paired ? 20 : h->umma_ncols / 8;
+  const size_t stage_bytes = group_bytes * ngroups;
   const size_t slack = (ngroups < 16) ? (16 - ngroups) * group_bytes : 0;  // operand A spans 16 row groups
   const size_t budget = 226 * 1024 - 1024 - slack;
   int stages = (int)(budget / stage_bytes);
@@ -411,6 +508,10 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   const long long nblk_full = h->d / kSubCols;
   const long long total_sub = (h->d + kSubCols - 1) / kSubCols;
   h->umma_ctas = (int)((nblk_full < h->num_sms) ? (nblk_full > 0 ? nblk_full : 1) : h->num_sms);
+  if (h->umma_paired) {
+    const long long units = (nblk_full + subs - 1) / subs;
+    h->umma_ctas = (int)(units < h->num_sms ? (units > 0 ? units : 1) : h->num_sms);
+  }
   h->d_pad = total_sub * kSubCols;
   if (cudaMalloc(&h->r_split, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
       cudaMalloc(&h->umma_partials, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess) {
@@ -420,7 +521,8 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   if (cudaMemset(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
       cudaMemset(h->umma_partials, 0, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess)
     return CDGRAB_ERR_CUDA;
-  if (!encode_map_3d(&h->tm_r, h->r_split, nblk_full, 3, h->d_pad, subs)) return CDGRAB_ERR_CUDA;
+  if (!encode_map_3d(&h->tm_r, h->r_split, nblk_full, 3, h->d_pad, h->umma_paired ? subs / 2 : subs))
+    return CDGRAB_ERR_CUDA;
   if (!encode_map_2d(&h->tm_r2, h->r_split, h->d, 3, h->d_pad)) return CDGRAB_ERR_CUDA;
   if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->umma_smem) !=
       cudaSuccess) {
@@ -428,6 +530,10 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     return CDGRAB_ERR_CUDA;
   }
   h->tm_g_base = nullptr;
+  h->umma_fused = h->shard ? 0 : 1;      // a shard's decisions wait for the sum over shards
+  if (const char *e = getenv("CDGRAB_UMMA_FUSE_TAIL")) {
+    if (atoi(e) == 0) h->umma_fused = 0;
+  }
   return CDGRAB_OK;
 }
 
@@ -441,9 +547,18 @@ void cdg_umma_teardown(cdgrab_ctx *h) {
 cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
   const long long nblk_full = h->d / kSubCols;
   if (grads != h->tm_g_base) {
-    if (!encode_map_3d(&h->tm_g, grads, nblk_full, 2 * h->m, h->d, h->umma_subs_per_stage) ||
+    const int box_blocks = h->umma_paired ? h->umma_subs_per_stage / 2 : h->umma_subs_per_stage;
+    if (!encode_map_3d(&h->tm_g, grads, nblk_full, 2 * h->m, h->d, box_blocks) ||
         !encode_map_2d(&h->tm_g2, grads, h->d, 2 * h->m, h->d))
       return cudaErrorInvalidValue;
+    // one copy for all full row groups of a (half) stage; CDGRAB_UMMA_G4=0: per-group copies only
+    h->umma_g4 = (2 * h->m) / 8;
+    if (const char *e = getenv("CDGRAB_UMMA_G4")) {
+      if (atoi(e) == 0) h->umma_g4 = 0;
+    }
+    if ((long long)h->d * 16 >= (1ll << 40)) h->umma_g4 = 0;     // the group stride must fit the map
+    if (h->umma_g4 > 0 && !encode_map_4d(&h->tm_g4, grads, nblk_full, h->umma_g4, h->d, box_blocks)) h->umma_g4 = 0;
+    if (h->umma_g4 == 0) h->tm_g4 = h->tm_g;
     h->tm_g_base = grads;
   }
   UmmaParams p;
@@ -455,16 +570,19 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
   p.nblk_full = nblk_full;
   p.tail = (h->d % kSubCols) ? 1 : 0;
   p.drain = h->umma_drain;
+  p.g4 = h->umma_g4;
+  p.paired = h->umma_paired;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
-    gram_umma_kernel<<<h->umma_ctas, kThreads, h->umma_smem, st>>>(h->tm_g, h->tm_r, h->tm_g2, h->tm_r2, p,
+    gram_umma_kernel<<<h->umma_ctas, kThreads, h->umma_smem, st>>>(h->tm_g, h->tm_r, h->tm_g2, h->tm_r2, h->tm_g4, p,
                                                                    h->umma_partials, h->status);
   }
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
     const int total = h->m * h->m + h->m;
     umma_combine_kernel<<<(total + 31) / 32, 256, 0, st>>>(h->umma_partials, h->umma_ctas, h->umma_ncols,
-                                                             h->umma_box_rows, h->m, h->gram);
+                                                             h->umma_box_rows, h->m, h->gram, h->status,
+                                                             cdg_tail_of(h, h->umma_fused));
   }
   return cudaGetLastError();
 }

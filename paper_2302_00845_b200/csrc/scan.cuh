@@ -34,6 +34,31 @@ inline CdgRule cdg_rule_of(const cdgrab_ctx *h) {
   return r;
 }
 
+// What a pass-1 kernel needs to finish the step itself: the block that takes the last ticket
+// runs the scalar part (no block ever waits for another).
+struct CdgTail {
+  int enabled;
+  int n, k;
+  unsigned *ticket;          // zero between launches
+  const int32_t *perm_cur;
+  int32_t *perm_next;
+  int8_t *signs;
+  float *margins;
+  double *rnorm2;
+  CdgRule rule;
+};
+
+inline CdgTail cdg_tail_of(const cdgrab_ctx *h, int enabled) {
+  CdgTail t;
+  t.enabled = enabled;
+  t.n = h->n; t.k = h->k;
+  t.ticket = h->ticket;
+  t.perm_cur = h->perm_cur; t.perm_next = h->perm_next;
+  t.signs = h->signs; t.margins = h->margins; t.rnorm2 = h->rnorm2;
+  t.rule = cdg_rule_of(h);
+  return t;
+}
+
 struct ScanSmem {
   double *t;     // [m]  starts as b; entry i is <r_{i-1}, c_i> once worker i is decided
   double *rn;    // [m]  ||r||^2 seen by worker i

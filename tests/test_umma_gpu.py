@@ -32,6 +32,10 @@ def run(m, n, d, seed, mean=0.0, scale=1.0):
     (32, 4, 64 * 148 * 3 + 8),   # every SM busy, ragged last K block
     (17, 6, 100_000),      # 2m not a multiple of 16
     (64, 4, 1_000_000),    # many pipeline turns per CTA
+    (32, 6, 1_000_000 + 24),   # two blocks per MMA, whole stages per CTA, ragged last block
+    (20, 4, 300_000),      # two blocks per MMA with unused row groups in both halves
+    (18, 4, 64 * 8 * 40),  # fewer stages than SMs; 2m = 36: a ragged row group beside the 4-D copy
+    (33, 4, 200_000),      # first m past the two-block mode
 ])
 def test_umma_shapes(m, n, d, monkeypatch):
     monkeypatch.setenv("CDGRAB_FORCE_PATH", "umma")
