@@ -116,6 +116,8 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
   h->device = dev; h->num_sms = prop.multiProcessorCount;
   h->independent = independent;
   h->shard = shard;
+  h->pdl = 1;                      // CDGRAB_PDL=0: plain stream order between the launches of a step
+  if (const char *e = getenv("CDGRAB_PDL")) h->pdl = atoi(e) ? 1 : 0;
 
   // ---- choose the path ------------------------------------------------------------
   const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);

@@ -55,6 +55,7 @@ struct cdgrab_ctx {
   int fma_tma_stages;
   int fma_tma_boxrows;     // rows per bulk-tensor copy
   int fma_tma_contig;      // 1: each CTA owns a contiguous range of tiles
+  int pdl;                 // 1: dependent launches start early and wait on the device for their predecessor
   int fma_tma_fused;       // 1: the last CTA of pass 1 also combines and decides (no scan launch)
   unsigned *ticket;        // [1] arrival counter of that hand-over, zero between launches
   size_t fma_tma_smem;
@@ -112,6 +113,29 @@ struct CdgProfScope {
   }
   ~CdgProfScope() { if (slot >= 0) cudaEventRecord(h->prof_ev[2 * slot + 1], st); }
 };
+
+// Programmatic dependent launch.  A kernel launched through cdg_launch_dep may be scheduled while
+// its predecessor in the stream is still running; it must call cdg_grid_dep_wait() before it
+// touches anything the predecessor writes (the wait returns once that grid has completed and
+// its writes are visible; without the launch attribute it returns at once).  A predecessor may
+// call cdg_grid_dep_trigger() to let the successor's blocks take SMs as its own blocks leave.
+#ifdef __CUDACC__
+__device__ __forceinline__ void cdg_grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void cdg_grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t cdg_launch_dep(const cdgrab_ctx *h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                  cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = h->pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
 
 // ---- launchers (each returns a cudaError_t; every kernel launch sits in a CdgProfScope) ----------
 cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream_t st);

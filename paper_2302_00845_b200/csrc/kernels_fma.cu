@@ -225,6 +225,7 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
   double *red = dsh;                                  // [WARPS][NPAD]
   double *tot = red + WARPS * Tri<M>::NPAD;           // [NPAD]
   float *ssh = reinterpret_cast<float *>(tot + Tri<M>::NPAD);  // [M]
+  cdg_grid_dep_wait();            // r comes from the step before, the rows from the caller's last launch
 
   float acc[Tri<M>::NPAD];
 #pragma unroll
@@ -445,9 +446,9 @@ static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, cudaStream_t
   }
   {
     CdgProfScope ps(h, CDGRAB_K_FUSED, st);
-    fused_step_kernel<T, M><<<1, FusedCfg<M>::THREADS, smem, st>>>(
-        (const T *)grads, h->r, h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs,
-        h->margins, h->rnorm2, h->status, cdg_rule_of(h));
+    cdg_launch_dep(h, fused_step_kernel<T, M>, dim3(1), dim3(FusedCfg<M>::THREADS), smem, st, (const T *)grads, h->r,
+                   h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs, h->margins, h->rnorm2, h->status,
+                   cdg_rule_of(h));
   }
   return cudaGetLastError();
 }
@@ -638,6 +639,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     mbar_init_fence();
   }
   __syncthreads();
+  cdg_grid_dep_wait();      // r is written by the launch before this one
   const long long deadline = clock64() + kCdgWaitCycles;
 
   float acc[Split<M>::NLPAD];
@@ -845,9 +847,9 @@ static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, cudaStream_t st) {
   const FtTail tail = cdg_tail_of(h, h->fma_tma_fused);
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
-    gram_fma_tma_kernel<T, M><<<h->gram_chunks, kFtThreads, h->fma_tma_smem, st>>>(
-        h->tm_fg, h->tm_fr, h->m, h->d, h->fma_tma_stages, h->fma_tma_boxrows, h->fma_tma_contig, h->partials,
-        h->status, tail);
+    cdg_launch_dep(h, gram_fma_tma_kernel<T, M>, dim3(h->gram_chunks), dim3(kFtThreads), h->fma_tma_smem, st,
+                   h->tm_fg, h->tm_fr, h->m, h->d, h->fma_tma_stages, h->fma_tma_boxrows, h->fma_tma_contig,
+                   h->partials, h->status, tail);
   }
   if (!h->fma_tma_fused) {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);

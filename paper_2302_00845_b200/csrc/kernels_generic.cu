@@ -128,6 +128,7 @@ scan_kernel(const double *__restrict__ gram, int m, int n, int k,
             int8_t *__restrict__ signs, float *__restrict__ margins,
             double *__restrict__ rnorm2, int *__restrict__ status, int use_smem, const CdgRule rule) {
   extern __shared__ double sh[];
+  cdg_grid_dep_wait();            // (G, b) come from the launch before this one
   const ScanSmem S = scan_smem(sh, m);
   const double *G = gram;
   for (int j = threadIdx.x; j < m; j += blockDim.x) S.t[j] = gram[(size_t)m * m + j];
@@ -212,6 +213,7 @@ update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__re
               int sign_stride, int m, long long d, __nv_bfloat16 *__restrict__ r_split,
               long long d_pad, float *__restrict__ mean_out) {
   extern __shared__ float ssh[];  // [m] signs as +-1.0f
+  cdg_grid_dep_wait();            // the signs come from the launch before this one
   for (int i = threadIdx.x; i < m; i += blockDim.x) ssh[i] = (float)signs[(size_t)i * sign_stride];
   __syncthreads();
   const long long nvec = d / VEC;
@@ -384,8 +386,8 @@ cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
   }
   {
     CdgProfScope ps(h, CDGRAB_K_SCAN, st);
-    scan_kernel<<<1, 256, smem, st>>>(h->gram, m, h->n, h->k, h->perm_cur, h->perm_next, h->signs,
-                                     h->margins, h->rnorm2, h->status, use_smem, cdg_rule_of(h));
+    cdg_launch_dep(h, scan_kernel, dim3(1), dim3(256), smem, st, h->gram, m, h->n, h->k, h->perm_cur, h->perm_next,
+                   h->signs, h->margins, h->rnorm2, h->status, use_smem, cdg_rule_of(h));
   }
   return cudaGetLastError();
 }
@@ -402,17 +404,17 @@ static void launch_update_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
   CdgProfScope ps(h, CDGRAB_K_UPDATE, st);
   if (h->mean_out) {
     if (h->r_split)
-      update_kernel<T, AccT, VEC, true, true><<<(unsigned)blocks, 256, smem, st>>>(
-          (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad, h->mean_out);
+      cdg_launch_dep(h, update_kernel<T, AccT, VEC, true, true>, dim3((unsigned)blocks), dim3(256), smem, st,
+                     (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad, h->mean_out);
     else
-      update_kernel<T, AccT, VEC, false, true><<<(unsigned)blocks, 256, smem, st>>>(
-          (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0, h->mean_out);
+      cdg_launch_dep(h, update_kernel<T, AccT, VEC, false, true>, dim3((unsigned)blocks), dim3(256), smem, st,
+                     (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0, h->mean_out);
   } else if (h->r_split) {
-    update_kernel<T, AccT, VEC, true, false><<<(unsigned)blocks, 256, smem, st>>>(
-        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad, nullptr);
+    cdg_launch_dep(h, update_kernel<T, AccT, VEC, true, false>, dim3((unsigned)blocks), dim3(256), smem, st,
+                   (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, h->r_split, h->d_pad, nullptr);
   } else {
-    update_kernel<T, AccT, VEC, false, false><<<(unsigned)blocks, 256, smem, st>>>(
-        (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0, nullptr);
+    cdg_launch_dep(h, update_kernel<T, AccT, VEC, false, false>, dim3((unsigned)blocks), dim3(256), smem, st,
+                   (const T *)grads, h->r, sg, h->n / 2, h->m, h->d, nullptr, 0, nullptr);
   }
 }
 

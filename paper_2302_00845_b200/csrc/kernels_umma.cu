@@ -150,6 +150,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_base_sh;
+  cdg_grid_dep_wait();            // r (as its bf16 split) is written by the launch before this one
   const long long deadline = clock64() + kWaitCycles;
 
   if (warp == 0) {
@@ -334,6 +335,7 @@ umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int
   __shared__ double scan_sh[4 * 64 + 64 * 64];     // m <= 64 on this path
   __shared__ int is_last;
   const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+  cdg_grid_dep_wait();            // the partial H come from the launch before this one
   const int total = m * m + m;
   const int e = blockIdx.x * 32 + lane;
   const size_t cs = (size_t)128 * ncols;   // one CTA's partial H
@@ -574,15 +576,14 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
   p.paired = h->umma_paired;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
-    gram_umma_kernel<<<h->umma_ctas, kThreads, h->umma_smem, st>>>(h->tm_g, h->tm_r, h->tm_g2, h->tm_r2, h->tm_g4, p,
-                                                                   h->umma_partials, h->status);
+    cdg_launch_dep(h, gram_umma_kernel, dim3(h->umma_ctas), dim3(kThreads), h->umma_smem, st, h->tm_g, h->tm_r,
+                   h->tm_g2, h->tm_r2, h->tm_g4, p, h->umma_partials, h->status);
   }
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
     const int total = h->m * h->m + h->m;
-    umma_combine_kernel<<<(total + 31) / 32, 256, 0, st>>>(h->umma_partials, h->umma_ctas, h->umma_ncols,
-                                                             h->umma_box_rows, h->m, h->gram, h->status,
-                                                             cdg_tail_of(h, h->umma_fused));
+    cdg_launch_dep(h, umma_combine_kernel, dim3((total + 31) / 32), dim3(256), 0, st, h->umma_partials, h->umma_ctas,
+                   h->umma_ncols, h->umma_box_rows, h->m, h->gram, h->status, cdg_tail_of(h, h->umma_fused));
   }
   return cudaGetLastError();
 }
