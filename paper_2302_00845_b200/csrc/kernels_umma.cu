@@ -71,6 +71,12 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
       ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accum) : "memory");
 }
+// true in exactly one lane of a converged warp (the same lane every time)
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -207,48 +213,53 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = ncols
-      const uint32_t mma_n = paired ? 160u : (uint32_t)p.ncols;
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((mma_n >> 3) << 17) | ((128u >> 4) << 24);
-      // The fp32 accumulation inside the tensor core truncates; over hundreds of thousands of
-      // columns that becomes a visible bias on sums of same-sign products.  So the sum is kept
-      // in TMEM only for `drain` iterations (about 1024 columns), then handed to the read-back
-      // warps, which add the chunks in fp32 registers with round-to-nearest, while the MMAs
-      // continue into the other accumulator buffer.
-      bool ok = true;
-      for (int it = 0; it < n_iter && ok; ++it) {
-        const int s = it % p.stages;
-        const int c = it / p.drain, buf = c & 1;
-        const bool chunk_start = (it % p.drain) == 0;
-        if (chunk_start && c >= 2) {
-          ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), ((c >> 1) - 1) & 1, deadline);
-          if (!ok) break;
-        }
-        ok = mbar_wait(smem_u32(&bar_full[s]), (it / p.stages) & 1, deadline);
-        if (!ok) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        int cnt = 1;
-        if (!(has_tail && it == 0)) {
-          const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
-          cnt = paired ? hb : (int)min((long long)p.subs, blk_hi - first);   // blocks past blk_hi belong to the next CTA
-        }
-        const uint32_t acc = tmem_acc + (uint32_t)buf * 256u;
-        for (int q = 0; q < cnt; ++q) {
-          const uint64_t desc = umma_desc(tiles + s * stage_bytes + q * 1024u, group_bytes);
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4) {
-            // 16 bf16 = 32 bytes further along K inside the swizzle row
-            const uint64_t dk = desc + (uint64_t)(k4 * 2);
-            umma_bf16(acc, dk, dk, idesc, !(chunk_start && q == 0 && k4 == 0));
-          }
-        }
-        umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
-        if ((it % p.drain) == p.drain - 1 || it == n_iter - 1)
-          umma_commit(smem_u32(&bar_acc_full[buf]));   // chunk complete
+    // The whole warp runs the loop converged and one elected lane issues: operands of
+    // tcgen05.mma computed under a lane test would have to be moved into uniform registers one
+    // by one (84 cycles per MMA were measured that way), operands of converged code start there.
+    // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = ncols
+    const uint32_t mma_n = paired ? 160u : (uint32_t)p.ncols;
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((mma_n >> 3) << 17) | ((128u >> 4) << 24);
+    // The fp32 accumulation inside the tensor core truncates; over hundreds of thousands of
+    // columns that becomes a visible bias on sums of same-sign products.  So the sum is kept
+    // in TMEM only for `drain` iterations (about 4096 columns), then handed to the read-back
+    // warps, which add the chunks in fp32 registers with round-to-nearest, while the MMAs
+    // continue into the other accumulator buffer.
+    bool ok = true;
+    int s = 0, c = 0, in_chunk = 0;          // stage, chunk number, position inside the chunk
+    uint32_t full_parity = 0;
+    for (int it = 0; it < n_iter; ++it) {
+      const int buf = c & 1;
+      const bool chunk_start = in_chunk == 0;
+      if (chunk_start && c >= 2) ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), ((c >> 1) - 1) & 1, deadline);
+      if (ok) ok = mbar_wait(smem_u32(&bar_full[s]), full_parity, deadline);
+      ok = __all_sync(0xffffffffu, ok);      // the lanes leave together
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      int cnt = 1;
+      if (!(has_tail && it == 0)) {
+        const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
+        cnt = paired ? hb : (int)min((long long)p.subs, blk_hi - first);   // blocks past blk_hi belong to the next CTA
       }
-      if (!ok) atomicOr(status, CDG_ST_TIMEOUT);
+      const uint32_t acc = tmem_acc + (uint32_t)buf * 256u;
+      const uint32_t sbase = tiles + (uint32_t)s * stage_bytes;
+      const bool chunk_end = (in_chunk == p.drain - 1) || (it == n_iter - 1);
+      for (int q = 0; q < cnt; ++q) {
+        const uint64_t desc = umma_desc(sbase + q * 1024u, group_bytes);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) {
+          // 16 bf16 = 32 bytes further along K inside the swizzle row
+          const uint64_t dk = desc + (uint64_t)(k4 * 2);
+          if (elect_one()) umma_bf16(acc, dk, dk, idesc, !(chunk_start && q == 0 && k4 == 0));
+        }
+      }
+      if (elect_one()) {
+        umma_commit(smem_u32(&bar_empty[s]));  // stage reusable once these MMAs have read it
+        if (chunk_end) umma_commit(smem_u32(&bar_acc_full[buf]));   // chunk complete
+      }
+      if (++in_chunk == p.drain) { in_chunk = 0; ++c; }
+      if (++s == p.stages) { s = 0; full_parity ^= 1u; }
     }
+    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
   } else {
     // ---------------- accumulator read-back: TMEM chunks -> fp32 registers -> partial H ----------------
     const int lg = warp & 3;                 // TMEM lane group this warp may read
