@@ -658,9 +658,10 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     if (lane == 0) {
       int issued = 0;
       bool ok = true;
+      int s = 0;
+      uint32_t turn = 0;                       // how often the ring has wrapped
       for (int it = 0; it < n_iter; ++it) {
-        const int s = it % stages;
-        if (it >= stages) ok = mbar_wait(smem_u32(&bar_empty[s]), ((it / stages) - 1) & 1, deadline);
+        if (turn > 0) ok = mbar_wait(smem_u32(&bar_empty[s]), (turn - 1) & 1, deadline);
         if (!ok) break;
         const long long tile = t_lo + (long long)it * t_step;
         const int col = (int)(tile * kFtCols);            // 256 elements: 16-byte aligned for both types
@@ -670,6 +671,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
         for (int q = 0; q < nbox; ++q) tma_load_2d(dst + q * box_bytes, &tm_g, col, q * box_rows, full);
         tma_load_2d(dst + g_bytes, &tm_r, col, 0, full);
         issued = it + 1;
+        if (++s == stages) { s = 0; ++turn; }
       }
       if (!ok) {
         atomicOr(status, CDG_ST_TIMEOUT);
@@ -680,9 +682,10 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   } else {
     const int col = threadIdx.x & (kFtCols - 1);
     bool ok = true;
+    int s = 0;
+    uint32_t parity = 0;
     for (int it = 0; it < n_iter && ok; ++it) {
-      const int s = it % stages;
-      ok = mbar_wait(smem_u32(&bar_full[s]), (it / stages) & 1, deadline);
+      ok = mbar_wait(smem_u32(&bar_full[s]), parity, deadline);
       if (!ok) break;
       const T *gt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes);
       const float *rt = reinterpret_cast<const float *>(base_ptr + (size_t)s * stage_bytes + g_bytes);
@@ -690,6 +693,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       else ft_consume<T, M, 1>(gt, rt, m, col, acc);
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));   // this warp is done with the stage
+      if (++s == stages) { s = 0; parity ^= 1u; }
     }
     if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
     // warp totals of the local entries, as doubles
