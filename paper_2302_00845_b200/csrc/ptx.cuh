@@ -1,5 +1,5 @@
 // Inline-PTX helpers shared by the TMA-fed kernels: mbarriers with bounded waits and tiled
-// bulk-tensor loads (no cluster multicast anywhere).
+// bulk-tensor loads (every copy lands in the issuing CTA's own shared memory).
 #pragma once
 
 #include <cuda.h>
