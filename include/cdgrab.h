@@ -170,6 +170,19 @@ long long cdgrab_out_of_bound(cdgrab_t *h);
 int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, void *stream);
 
 /*
+ * `count` consecutive steps of Algorithm 7's outer loop in one call, for gradients that are
+ * staged ahead (a whole epoch of a small problem): grads_dev is DEVICE memory laid out
+ * [count][2][m][d] in the handle's dtype, 16-byte aligned, step j at offset j*2*m*d elements.
+ * The result is bit-identical to `count` calls of cdgrab_step on the slices (greedy rule of
+ * Algorithm 6).  On the single-launch path (small steps) the steps run inside one kernel launch
+ * and the running sum never leaves the SM's caches between them; on the other paths the call
+ * loops over cdgrab_step.  CDGRAB_ERR_STATE if fewer than `count` steps remain in the epoch
+ * (nothing is done then); CDGRAB_ERR_INVALID on a shard handle or count < 1.  Asynchronous on
+ * `stream` like cdgrab_step.
+ */
+int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream);
+
+/*
  * Close the epoch after exactly n/2 steps (else CDGRAB_ERR_STATE): the next permutations
  * become the current ones (Algorithm 4, last lines of the epoch loop) and, if perms_out is
  * not NULL, are copied there.  perms_out: HOST or DEVICE pointer, int32 [m][n];

@@ -51,6 +51,7 @@ SIGNATURES = {
     "cdgrab_path": (C.c_int, [C.c_void_p]),
     "cdgrab_launch_count": (C.c_longlong, [C.c_void_p]),
     "cdgrab_strerror": (C.c_char_p, [C.c_int]),
+    "cdgrab_step_many": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "cdgrab_profile_enable": (C.c_int, [C.c_void_p, C.c_int]),
     "cdgrab_profile_read": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]),
     "cdgrab_logreg_grads": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -178,6 +179,11 @@ class CdGrab:
         """step() that also writes the average of each gather buffer into mean_out (CUDA float32 [2][d])."""
         _check(lib().cdgrab_step_mean(self._h, _ptr(grads), _ptr(mean_out), _stream_ptr(stream)),
                "cdgrab_step_mean")
+
+    def step_many(self, grads, stream=None):
+        """grads: contiguous CUDA tensor [count][2][m][d]; the count steps in one call."""
+        _check(lib().cdgrab_step_many(self._h, _ptr(grads), int(grads.shape[0]), _stream_ptr(stream)),
+               "cdgrab_step_many")
 
     def step_logreg(self, X, y, w, stream=None):
         """One balancing step straight from the feature rows (no gradient buffer)."""

@@ -316,7 +316,7 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
     if (h->rule_randomized || h->mean_out) return CDGRAB_ERR_INVALID;  // greedy rule only in this mode
     e = cdg_launch_indep(h, grads_dev, st);
   } else if (h->path == CDGRAB_PATH_FUSED) {
-    e = cdg_launch_fused(h, grads_dev, st);
+    e = cdg_launch_fused(h, grads_dev, 1, st);
   } else {
     e = launch_pass1(h, grads_dev, st);
     const bool decided = (h->path == CDGRAB_PATH_UMMA) ? h->umma_fused : (h->fma_tma && h->fma_tma_fused);
@@ -325,6 +325,27 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   }
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   h->k++;
+  return CDGRAB_OK;
+}
+
+int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream) {
+  if (!valid(h) || !grads_dev || count < 1) return CDGRAB_ERR_INVALID;
+  if (((uintptr_t)grads_dev & 15) != 0 || h->shard) return CDGRAB_ERR_INVALID;
+  if (!h->epoch_open || h->k + count > h->n / 2) return CDGRAB_ERR_STATE;
+  const size_t step_bytes = 2 * (size_t)h->m * (size_t)h->d * (h->dtype == CDGRAB_F32 ? 4 : 2);
+  if (h->path == CDGRAB_PATH_FUSED && !h->independent && !h->rule_randomized && !h->mean_out) {
+    if (step_bytes % 16 != 0) return CDGRAB_ERR_INVALID;
+    if (cdg_launch_fused(h, grads_dev, count, (cudaStream_t)stream) != cudaSuccess) {
+      cudaGetLastError();
+      return CDGRAB_ERR_CUDA;
+    }
+    h->k += count;
+    return CDGRAB_OK;
+  }
+  for (int i = 0; i < count; ++i) {
+    const int rc = cdgrab_step(h, (const char *)grads_dev + (size_t)i * step_bytes, stream);
+    if (rc != CDGRAB_OK) return rc;
+  }
   return CDGRAB_OK;
 }
 

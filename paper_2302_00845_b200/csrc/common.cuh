@@ -143,7 +143,7 @@ cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st);
 cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_mean(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_split_r(cdgrab_ctx *h, cudaStream_t st);
-cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, int count, cudaStream_t st);   // count steps, one launch
 cudaError_t cdg_launch_gram_fma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_fused_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w, cudaStream_t st);
 cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,

@@ -216,7 +216,7 @@ struct FusedCfg { static constexpr int THREADS = (M <= 4) ? 1024 : (M <= 8 ? 512
 
 template <typename T, int M>
 __global__ void __launch_bounds__(FusedCfg<M>::THREADS)
-fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, int k,
+fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, int k, int count,
                   const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
                   int8_t *__restrict__ signs, float *__restrict__ margins,
                   double *__restrict__ rnorm2, int *__restrict__ status, const CdgRule rule) {
@@ -227,10 +227,12 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
   float *ssh = reinterpret_cast<float *>(tot + Tri<M>::NPAD);  // [M]
   cdg_grid_dep_wait();            // r comes from the step before, the rows from the caller's last launch
 
+  // `count` consecutive steps ([count][2][m][d] rows): r stays in this SM's cache between them
+  const long long nvec = d / 4;
+  for (int kk = 0; kk < count; ++kk, ++k, g += 2 * (size_t)m * (size_t)d) {
   float acc[Tri<M>::NPAD];
 #pragma unroll
   for (int e = 0; e < Tri<M>::NPAD; ++e) acc[e] = 0.f;
-  const long long nvec = d / 4;
   gram_accumulate<T, M>(g, r, m, d, threadIdx.x, blockDim.x, nvec, acc);
   const double v = block_reduce_acc<M, WARPS>(acc, red);
   if (threadIdx.x < Tri<M>::NACC) tot[threadIdx.x] = v;
@@ -260,6 +262,8 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
     }
     *reinterpret_cast<float4 *>(r + x) =
         make_float4((float)a4[0], (float)a4[1], (float)a4[2], (float)a4[3]);
+  }
+  __syncthreads();   // the new r and the shared arrays are settled before the next step reads them
   }
 }
 
@@ -434,7 +438,7 @@ bool cdg_fused_supported(int m, long long d, int dtype) {
 }
 
 template <typename T, int M>
-static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, int count, cudaStream_t st) {
   const size_t smem = ((FusedCfg<M>::THREADS / 32) * Tri<M>::NPAD + Tri<M>::NPAD) * sizeof(double) +
                       M * sizeof(float);
   static bool attr_set = false;
@@ -447,22 +451,22 @@ static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, cudaStream_t
   {
     CdgProfScope ps(h, CDGRAB_K_FUSED, st);
     cdg_launch_dep(h, fused_step_kernel<T, M>, dim3(1), dim3(FusedCfg<M>::THREADS), smem, st, (const T *)grads, h->r,
-                   h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs, h->margins, h->rnorm2, h->status,
-                   cdg_rule_of(h));
+                   h->m, h->n, h->d, h->k, count, h->perm_cur, h->perm_next, h->signs, h->margins, h->rnorm2,
+                   h->status, cdg_rule_of(h));
   }
   return cudaGetLastError();
 }
 
-cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+cudaError_t cdg_launch_fused(cdgrab_ctx *h, const void *grads, int count, cudaStream_t st) {
   const int M = pick_M(h->m);
   if (h->dtype == CDGRAB_F32) {
-    if (M == 4) return launch_fused_t<float, 4>(h, grads, st);
-    if (M == 8) return launch_fused_t<float, 8>(h, grads, st);
-    return launch_fused_t<float, 16>(h, grads, st);
+    if (M == 4) return launch_fused_t<float, 4>(h, grads, count, st);
+    if (M == 8) return launch_fused_t<float, 8>(h, grads, count, st);
+    return launch_fused_t<float, 16>(h, grads, count, st);
   }
-  if (M == 4) return launch_fused_t<__nv_bfloat16, 4>(h, grads, st);
-  if (M == 8) return launch_fused_t<__nv_bfloat16, 8>(h, grads, st);
-  return launch_fused_t<__nv_bfloat16, 16>(h, grads, st);
+  if (M == 4) return launch_fused_t<__nv_bfloat16, 4>(h, grads, count, st);
+  if (M == 8) return launch_fused_t<__nv_bfloat16, 8>(h, grads, count, st);
+  return launch_fused_t<__nv_bfloat16, 16>(h, grads, count, st);
 }
 
 template <typename T, int M>
