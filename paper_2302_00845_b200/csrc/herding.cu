@@ -16,8 +16,10 @@ struct HerdPlan {
   int seglen;      // positions per segment (the last one may be shorter)
 };
 
-HerdPlan herd_plan(int n, long long d) {
-  long long nseg = (n + 31) / 32;
+HerdPlan herd_plan(int m, int n, long long d) {
+  // about 160 gathered rows per thread: segments of 32 positions at m = 5, of one position at m >= 160
+  const int want_len = m >= 160 ? 1 : 160 / m;
+  long long nseg = (n + want_len - 1) / want_len;
   const long long cap = (8ll << 20) / d;          // at most 8 Mi (segment, coordinate) cells
   if (nseg > cap) nseg = cap;
   if (nseg < 1) nseg = 1;
@@ -61,6 +63,33 @@ __global__ void herd_prefix(double *__restrict__ segsum, int nseg, long long d, 
   zbar[x] = run * inv_count;
 }
 
+// Many segments (long sequences of short vectors): one block per coordinate.  Thread t adds a
+// run of consecutive segments, thread 0 turns the 256 run totals into exclusive offsets in run
+// order, then every thread writes the exclusive prefix of its run.  Fixed order throughout.
+__global__ void __launch_bounds__(256)
+herd_prefix_block(double *__restrict__ segsum, int nseg, long long d, double inv_count, double *__restrict__ zbar) {
+  __shared__ double runs[256];
+  const long long x = blockIdx.x;
+  const int len = (nseg + 255) / 256;
+  const int s0 = min(nseg, (int)threadIdx.x * len), s1 = min(nseg, s0 + len);
+  double tot = 0.0;
+  for (int s = s0; s < s1; ++s) tot += segsum[(size_t)s * d + x];
+  runs[threadIdx.x] = tot;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double run = 0.0;
+    for (int t = 0; t < 256; ++t) { const double v = runs[t]; runs[t] = run; run += v; }
+    zbar[x] = run * inv_count;
+  }
+  __syncthreads();
+  double run = runs[threadIdx.x];
+  for (int s = s0; s < s1; ++s) {
+    const double v = segsum[(size_t)s * d + x];
+    segsum[(size_t)s * d + x] = run;
+    run += v;
+  }
+}
+
 // thread (segment, coordinate): walk the segment from its starting prefix, track max |prefix|
 __global__ void herd_segment_max(const float *__restrict__ z, const int32_t *__restrict__ perms, int m, int n,
                                  long long d, int nseg, int seglen, const double *__restrict__ segsum,
@@ -100,7 +129,7 @@ __global__ void herd_segment_max(const float *__restrict__ z, const int32_t *__r
 
 extern "C" long long cdgrab_herding_workspace_bytes(int m, int n, long long d) {
   if (m < 1 || n < 1 || d < 1) return -1;
-  const HerdPlan p = herd_plan(n, d);
+  const HerdPlan p = herd_plan(m, n, d);
   return (long long)sizeof(double) * ((long long)p.nseg * d + d);
 }
 
@@ -110,7 +139,7 @@ extern "C" int cdgrab_herding_objective(const float *z_dev, const int32_t *perms
   if (!z_dev || !perms_dev || !workspace_dev || !out_dev || m < 1 || n < 1 || d < 1) return CDGRAB_ERR_INVALID;
   if (workspace_bytes < cdgrab_herding_workspace_bytes(m, n, d)) return CDGRAB_ERR_INVALID;
   if (((uintptr_t)workspace_dev & 7) != 0 || ((uintptr_t)out_dev & 7) != 0) return CDGRAB_ERR_INVALID;
-  const HerdPlan p = herd_plan(n, d);
+  const HerdPlan p = herd_plan(m, n, d);
   cudaStream_t st = (cudaStream_t)stream;
   double *segsum = (double *)workspace_dev;
   double *zbar = segsum + (size_t)p.nseg * d;
@@ -118,7 +147,10 @@ extern "C" int cdgrab_herding_objective(const float *z_dev, const int32_t *perms
   const unsigned gb = (unsigned)((cells + 255) / 256);
   if (cudaMemsetAsync(out_dev, 0, sizeof(double), st) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   herd_segment_sums<<<gb, 256, 0, st>>>(z_dev, perms_dev, m, n, d, p.nseg, p.seglen, segsum);
-  herd_prefix<<<(unsigned)((d + 127) / 128), 128, 0, st>>>(segsum, p.nseg, d, 1.0 / ((double)m * n), zbar);
+  if (p.nseg >= 512 && d <= 65536)
+    herd_prefix_block<<<(unsigned)d, 256, 0, st>>>(segsum, p.nseg, d, 1.0 / ((double)m * n), zbar);
+  else
+    herd_prefix<<<(unsigned)((d + 127) / 128), 128, 0, st>>>(segsum, p.nseg, d, 1.0 / ((double)m * n), zbar);
   herd_segment_max<<<gb, 256, 0, st>>>(z_dev, perms_dev, m, n, d, p.nseg, p.seglen, segsum, zbar,
                                        (unsigned long long *)out_dev);
   if (cudaGetLastError() != cudaSuccess) return CDGRAB_ERR_CUDA;
