@@ -9,8 +9,13 @@
 //   fused_step_kernel  one CTA does the whole step (Gram, the m decisions of Algorithm 6,
 //                      permutation slots of Algorithm 7, update of r): the step's inputs
 //                      come from HBM once and are re-read from cache for the update
+#include <cooperative_groups.h>
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "scan.cuh"
+
+namespace cg = cooperative_groups;
 
 template <int M>
 struct Tri {
@@ -172,7 +177,7 @@ __device__ __forceinline__ void fused_decide(const double *tot, int m, int n, in
                                              const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
                                              int8_t *__restrict__ signs, float *__restrict__ margins,
                                              double *__restrict__ rnorm2, int *__restrict__ status,
-                                             const CdgRule &rule, float *ssh) {
+                                             const CdgRule &rule, float *ssh, bool write_out = true) {
   double t[M];
 #pragma unroll
   for (int i = 0; i < M; ++i) t[i] = tot[Tri<M>::NPAIR + i];
@@ -189,19 +194,22 @@ __device__ __forceinline__ void fused_decide(const double *tot, int m, int n, in
       const double sd = (double)s;
 #pragma unroll
       for (int j = i + 1; j < M; ++j) t[j] += sd * tot[Tri<M>::idx(i, j)];
-      const size_t pos = (size_t)i * half + k;
-      signs[pos] = (int8_t)s;
-      const double den = rn2 * gii;
-      margins[pos] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
-      const int32_t first = perm_cur[(size_t)i * n + 2 * k];
-      const int32_t second = perm_cur[(size_t)i * n + 2 * k + 1];
-      perm_next[(size_t)i * n + k] = (s == 1) ? first : second;           // front slot
-      perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;  // back slot
+      if (write_out) {
+        const size_t pos = (size_t)i * half + k;
+        signs[pos] = (int8_t)s;
+        const double den = rn2 * gii;
+        margins[pos] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
+        const int32_t first = perm_cur[(size_t)i * n + 2 * k];
+        const int32_t second = perm_cur[(size_t)i * n + 2 * k + 1];
+        perm_next[(size_t)i * n + k] = (s == 1) ? first : second;           // front slot
+        perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;  // back slot
+      }
       rn2 += 2.0 * sd * ti + gii;
       if (rn2 < 0.0) rn2 = 0.0;
       ssh[i] = (float)s;
     }
   }
+  if (!write_out) return;
   *rnorm2 = rn2;
   if (bad) atomicOr(status, CDG_ST_NONFINITE);
   if (oob) atomicAdd(rule.oob, (unsigned long long)oob);
@@ -268,6 +276,77 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
 }
 
 // ------------------------------------------------------------------------------------
+// The same step spread over a thread-block cluster: CTA `rank` of C takes every C-th group of
+// columns, the C block totals of the Gram entries meet through distributed shared memory (each
+// CTA adds them in rank order, so all hold the same sums), every CTA takes the same decisions,
+// rank 0 writes them out, and each CTA updates the columns it read.  C SMs' worth of loads in
+// flight and of cache bandwidth instead of one; two cluster barriers per step.
+// ------------------------------------------------------------------------------------
+template <int M>
+struct ClusterCfg { static constexpr int THREADS = (M <= 8) ? 128 : 256; };   // >= the Gram entries of M
+
+template <typename T, int M>
+__global__ void __launch_bounds__(ClusterCfg<M>::THREADS)
+fused_step_cluster_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, int k, int count,
+                          const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
+                          int8_t *__restrict__ signs, float *__restrict__ margins,
+                          double *__restrict__ rnorm2, int *__restrict__ status, const CdgRule rule) {
+  extern __shared__ double dsh[];
+  constexpr int WARPS = ClusterCfg<M>::THREADS / 32;
+  double *red = dsh;                                  // [WARPS][NPAD]
+  double *mine = red + WARPS * Tri<M>::NPAD;          // [NPAD] this CTA's totals, read by the whole cluster
+  double *tot = mine + Tri<M>::NPAD;                  // [NPAD] totals of the cluster
+  float *ssh = reinterpret_cast<float *>(tot + Tri<M>::NPAD);  // [M]
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned rank = cluster.block_rank(), csize = cluster.num_blocks();
+  cdg_grid_dep_wait();            // r comes from the step before, the rows from the caller's last launch
+
+  const long long nvec = d / 4;
+  const long long v0 = (long long)rank * blockDim.x + threadIdx.x, vstride = (long long)csize * blockDim.x;
+  const size_t slab = (size_t)m * (size_t)d;
+  for (int kk = 0; kk < count; ++kk, ++k, g += 2 * slab) {
+    float acc[Tri<M>::NPAD];
+#pragma unroll
+    for (int e = 0; e < Tri<M>::NPAD; ++e) acc[e] = 0.f;
+    gram_accumulate<T, M>(g, r, m, d, v0, vstride, nvec, acc);
+    const double v = block_reduce_acc<M, WARPS>(acc, red);
+    if (threadIdx.x < Tri<M>::NACC) mine[threadIdx.x] = v;
+    cluster.sync();                                   // every CTA's totals are in place
+    if (threadIdx.x < Tri<M>::NACC) {
+      double sum = 0.0;
+      for (unsigned c = 0; c < csize; ++c) sum += cluster.map_shared_rank(mine, c)[threadIdx.x];
+      tot[threadIdx.x] = sum;
+    }
+    cluster.sync();                                   // all remote reads done: `mine` may be rewritten
+    if (threadIdx.x == 0)
+      fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh, rank == 0);
+    __syncthreads();
+
+    // r <- r + sum_i s_i c_i (i ascending) on this CTA's columns, inputs re-read through the cache
+    for (long long vv = v0; vv < nvec; vv += vstride) {
+      const size_t x = (size_t)vv * 4;
+      float rv[4];
+      ld4_r(r + x, rv);
+      double a4[4] = {(double)rv[0], (double)rv[1], (double)rv[2], (double)rv[3]};
+#pragma unroll
+      for (int i = 0; i < M; ++i) {
+        if (i < m) {
+          float a[4], b[4];
+          ld4<T>(g + (size_t)i * (size_t)d + x, a);
+          ld4<T>(g + slab + (size_t)i * (size_t)d + x, b);
+          const float s = ssh[i];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) a4[j] += (double)(s * (a[j] - b[j]));
+        }
+      }
+      *reinterpret_cast<float4 *>(r + x) =
+          make_float4((float)a4[0], (float)a4[1], (float)a4[2], (float)a4[3]);
+    }
+    __syncthreads();   // the shared arrays are settled before the next step reuses them
+  }
+}
+
+// ------------------------------------------------------------------------------------
 // Logistic regression without a gradient buffer: the whole step from the feature rows.
 // For worker i the pair's items are p = perm_cur[i][2k], q = perm_cur[i][2k+1]; with
 // a = sigma(<w,x_p>) - y_p and b = sigma(<w,x_q>) - y_q the difference is c_i = a x_p - b x_q
@@ -292,22 +371,31 @@ __device__ __forceinline__ void logreg_diffs(const float *__restrict__ X, const 
   }
 }
 
-template <int M>
-__global__ void __launch_bounds__(FusedCfg<M>::THREADS)
+// Runs as a cluster of C >= 1 CTAs: CTA `rank` takes every C-th group of columns; the 2m dot
+// products and the Gram entries are summed over the cluster through distributed shared memory in
+// rank order, so every CTA holds the same coefficients and takes the same decisions.
+template <int M, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ y, const float *__restrict__ w,
                          float *r, int m, int n, long long d, int k, const int32_t *__restrict__ perm_cur,
                          int32_t *__restrict__ perm_next, int8_t *__restrict__ signs, float *__restrict__ margins,
                          double *__restrict__ rnorm2, int *__restrict__ status, const CdgRule rule) {
   extern __shared__ double dsh[];
-  constexpr int WARPS = FusedCfg<M>::THREADS / 32;
+  constexpr int WARPS = THREADS / 32;
   double *red = dsh;                                  // [WARPS][NPAD]; first used as [WARPS][2M] for the dots
-  double *tot = red + WARPS * Tri<M>::NPAD;           // [NPAD]
-  float *ssh = reinterpret_cast<float *>(tot + Tri<M>::NPAD);  // [M]
+  double *mine = red + WARPS * Tri<M>::NPAD;          // [NPAD] this CTA's totals, read by the whole cluster
+  double *tot = mine + Tri<M>::NPAD;                  // [NPAD] totals of the cluster
+  double *dots = tot + Tri<M>::NPAD;                  // [2M] this CTA's share of <w, x>, read by the cluster
+  float *ssh = reinterpret_cast<float *>(dots + 2 * M);  // [M]
   float *coef = ssh + M;                              // [2M]: a_0..a_{m-1}, b_0..b_{m-1}
   float *yv = coef + 2 * M;                           // [2M]
   size_t *rowoff = reinterpret_cast<size_t *>(yv + 2 * M);      // [2M] element offsets of the rows in X
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned rank = cluster.block_rank(), csize = cluster.num_blocks();
   const long long nvec = d / 4;
+  const long long v0 = (long long)rank * THREADS + threadIdx.x, vstride = (long long)csize * THREADS;
+  cdg_grid_dep_wait();            // r and the current order come from earlier launches
 
   if (threadIdx.x < 2 * m) {
     const int q = threadIdx.x / m, i = threadIdx.x % m;
@@ -322,7 +410,7 @@ fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ 
     float z[2 * M];
 #pragma unroll
     for (int e = 0; e < 2 * M; ++e) z[e] = 0.f;
-    for (long long v = threadIdx.x; v < nvec; v += blockDim.x) {
+    for (long long v = v0; v < nvec; v += vstride) {
       const size_t x = (size_t)v * 4;
       float wv[4];
       ld4<float>(w + x, wv);
@@ -348,6 +436,12 @@ fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ 
   if (threadIdx.x < 2 * m) {
     double zz = 0.0;
     for (int wi = 0; wi < WARPS; ++wi) zz += red[wi * 2 * M + threadIdx.x];
+    dots[threadIdx.x] = zz;
+  }
+  cluster.sync();
+  if (threadIdx.x < 2 * m) {
+    double zz = 0.0;
+    for (unsigned c = 0; c < csize; ++c) zz += cluster.map_shared_rank(dots, c)[threadIdx.x];
     const float zf = (float)zz;
     // sigma(z) - y without cancellation for y in {0,1}: sigma(z) - 1 = -sigma(-z)
     coef[threadIdx.x] = (yv[threadIdx.x] > 0.5f) ? -1.f / (1.f + expf(zf)) : 1.f / (1.f + expf(-zf));
@@ -357,7 +451,7 @@ fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ 
   float acc[Tri<M>::NPAD];
 #pragma unroll
   for (int e = 0; e < Tri<M>::NPAD; ++e) acc[e] = 0.f;
-  for (long long v = threadIdx.x; v < nvec; v += blockDim.x) {
+  for (long long v = v0; v < nvec; v += vstride) {
     const size_t x = (size_t)v * 4;
     float c[M][4], rv[4];
     logreg_diffs<M>(X, rowoff, coef, m, x, c);
@@ -374,13 +468,19 @@ fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ 
     }
   }
   const double v = block_reduce_acc<M, WARPS>(acc, red);
-  if (threadIdx.x < Tri<M>::NACC) tot[threadIdx.x] = v;
-  __syncthreads();
+  if (threadIdx.x < Tri<M>::NACC) mine[threadIdx.x] = v;
+  cluster.sync();                                     // every CTA's totals are in place
+  if (threadIdx.x < Tri<M>::NACC) {
+    double sum = 0.0;
+    for (unsigned c = 0; c < csize; ++c) sum += cluster.map_shared_rank(mine, c)[threadIdx.x];
+    tot[threadIdx.x] = sum;
+  }
+  cluster.sync();                                     // remote reads done before any CTA moves on or leaves
   if (threadIdx.x == 0)
-    fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh);
+    fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh, rank == 0);
   __syncthreads();
 
-  for (long long vv = threadIdx.x; vv < nvec; vv += blockDim.x) {
+  for (long long vv = v0; vv < nvec; vv += vstride) {
     const size_t x = (size_t)vv * 4;
     float c[M][4], rv[4];
     logreg_diffs<M>(X, rowoff, coef, m, x, c);
@@ -398,27 +498,40 @@ fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ 
   }
 }
 
-template <int M>
-static cudaError_t launch_fused_logreg_t(cdgrab_ctx *h, const float *X, const float *y, const float *w,
-                                         cudaStream_t st) {
-  constexpr int WARPS = FusedCfg<M>::THREADS / 32;
-  const size_t smem = (WARPS * Tri<M>::NPAD + Tri<M>::NPAD) * sizeof(double) + (M + 4 * M) * sizeof(float) +
-                      2 * M * sizeof(size_t) + 16;
+template <int M> struct ClusterCfg;
+template <int M> static int fused_cluster_size(const cdgrab_ctx *h);
+
+template <int M, int THREADS>
+static cudaError_t launch_fused_logreg_tt(cdgrab_ctx *h, const float *X, const float *y, const float *w, int csize,
+                                          cudaStream_t st) {
+  constexpr int WARPS = THREADS / 32;
+  const size_t smem = (WARPS * Tri<M>::NPAD + 2 * Tri<M>::NPAD + 2 * M) * sizeof(double) +
+                      (M + 4 * M) * sizeof(float) + 2 * M * sizeof(size_t) + 16;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(fused_logreg_step_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(fused_logreg_step_kernel<M, THREADS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  {
-    CdgProfScope ps(h, CDGRAB_K_FUSED, st);
-    fused_logreg_step_kernel<M><<<1, FusedCfg<M>::THREADS, smem, st>>>(
-        X, y, w, h->r, h->m, h->n, h->d, h->k, h->perm_cur, h->perm_next, h->signs, h->margins, h->rnorm2,
-        h->status, cdg_rule_of(h));
-  }
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(csize); cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = csize; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = h->pdl ? 2 : 1;
+  CdgProfScope ps(h, CDGRAB_K_FUSED, st);
+  return cudaLaunchKernelEx(&cfg, fused_logreg_step_kernel<M, THREADS>, X, y, w, h->r, h->m, h->n, h->d, h->k,
+                            (const int32_t *)h->perm_cur, h->perm_next, h->signs, h->margins, h->rnorm2, h->status,
+                            cdg_rule_of(h));
 }
+
+template <int M>
+static cudaError_t launch_fused_logreg_t(cdgrab_ctx *h, const float *X, const float *y, const float *w,
+                                         cudaStream_t st);
 
 cudaError_t cdg_launch_fused_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w, cudaStream_t st) {
   const int M = h->m <= 4 ? 4 : (h->m <= 8 ? 8 : 16);
@@ -437,8 +550,49 @@ bool cdg_fused_supported(int m, long long d, int dtype) {
   return m <= 16 && d % 4 == 0;
 }
 
+// CTAs per cluster for the spread-out step: one per THREADS column groups, a power of two, at most 8
+template <int M>
+static int fused_cluster_size(const cdgrab_ctx *h) {
+  if (const char *e = getenv("CDGRAB_CLUSTER")) {
+    if (atoi(e) == 0) return 1;
+  }
+  const long long groups = (h->d / 4 + ClusterCfg<M>::THREADS - 1) / ClusterCfg<M>::THREADS;
+  int c = 1;
+  while (c < 8 && 2 * c <= groups) c *= 2;
+  return c;
+}
+
+template <int M>
+static cudaError_t launch_fused_logreg_t(cdgrab_ctx *h, const float *X, const float *y, const float *w,
+                                         cudaStream_t st) {
+  const int csize = fused_cluster_size<M>(h);
+  if (csize > 1) return launch_fused_logreg_tt<M, ClusterCfg<M>::THREADS>(h, X, y, w, csize, st);
+  return launch_fused_logreg_tt<M, FusedCfg<M>::THREADS>(h, X, y, w, 1, st);
+}
+
+template <typename T, int M>
+static cudaError_t launch_fused_cluster_t(cdgrab_ctx *h, const void *grads, int count, int csize, cudaStream_t st) {
+  constexpr int THREADS = ClusterCfg<M>::THREADS;
+  const size_t smem = ((THREADS / 32) * Tri<M>::NPAD + 2 * Tri<M>::NPAD) * sizeof(double) + M * sizeof(float);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(csize); cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = csize; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = h->pdl ? 2 : 1;
+  CdgProfScope ps(h, CDGRAB_K_FUSED, st);
+  return cudaLaunchKernelEx(&cfg, fused_step_cluster_kernel<T, M>, (const T *)grads, h->r, h->m, h->n, h->d, h->k,
+                            count, (const int32_t *)h->perm_cur, h->perm_next, h->signs, h->margins, h->rnorm2,
+                            h->status, cdg_rule_of(h));
+}
+
 template <typename T, int M>
 static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, int count, cudaStream_t st) {
+  const int csize = fused_cluster_size<M>(h);
+  if (csize > 1) return launch_fused_cluster_t<T, M>(h, grads, count, csize, st);
   const size_t smem = ((FusedCfg<M>::THREADS / 32) * Tri<M>::NPAD + Tri<M>::NPAD) * sizeof(double) +
                       M * sizeof(float);
   static bool attr_set = false;
