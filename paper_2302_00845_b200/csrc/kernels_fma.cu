@@ -9,6 +9,9 @@
 //   fused_step_kernel  one CTA does the whole step (Gram, the m decisions of Algorithm 6,
 //                      permutation slots of Algorithm 7, update of r): the step's inputs
 //                      come from HBM once and are re-read from cache for the update
+//   fused_step_cluster_kernel  the same step on a thread-block cluster (DSMEM reduction)
+//   fused_logreg_step_kernel   the step straight from logistic-regression feature rows
+//   gram_fma_tma_kernel        TMA-fed pass 1 for long rows; its last CTA combines and decides
 #include <cooperative_groups.h>
 #include <stdlib.h>
 

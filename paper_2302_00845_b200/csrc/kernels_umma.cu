@@ -11,18 +11,22 @@
 // falls out of the same MMA.
 //
 // One persistent CTA per SM owns a contiguous K range (split-K) in blocks of 64 columns.
-// A pipeline stage holds `subs` consecutive blocks.  Rows are loaded in groups of 8 by 3-D TMA
-// boxes {64 columns, 8 rows, subs blocks}: one instruction touches only 8 rows and
-// subs*128 contiguous bytes of each, which keeps address translation and DRAM pages local
-// even though consecutive rows lie hundreds of megabytes apart.  In shared memory a stage is
+// A pipeline stage holds `subs` consecutive blocks.  Rows are loaded in groups of 8: a TMA box
+// {64 columns, 8 rows, subs blocks} touches only 8 rows and subs*128 contiguous bytes of each,
+// which keeps address translation and DRAM pages local even though consecutive rows lie
+// hundreds of megabytes apart; a 4-D map {64 columns, 8 rows, blocks, groups} brings all full
+// groups of a stage with one instruction in the same order.  In shared memory a stage is
 // [row group][block][8 rows][128 B, 128-byte swizzle]; the MMA descriptors walk row groups
 // with a stride of subs*1024 bytes.  Row groups 0..box_rows/8-1 hold gradient rows (rows past
 // 2m are zero-filled by TMA), the next group holds the three r rows, and one more group of
 // zeros (written once) pads N to a multiple of 16.  The same bytes serve as operand A (16
 // row groups from the block base) and operand B (the first N = box_rows + 16 rows).  A ragged
 // last block (d not a multiple of 64) is loaded with 2-D boxes of 8 rows into the same layout.
-// Roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2..5 drain the
-// accumulator (tcgen05.ld) chunk by chunk into fp32 registers and write the CTA's partial H.
+// With 2m <= 64 one MMA takes two blocks at once (N = 160; layout at the top of the kernel).
+// Roles: warp 0 TMA producer, warp 1 MMA issuer (the warp loops converged, an elected lane
+// issues) and TMEM owner, warps 2..5 drain the accumulator (tcgen05.ld) chunk by chunk into
+// fp32 registers and write the CTA's partial H.  The combine kernel's last block also takes the
+// step's decisions.
 // Every wait is bounded: on expiry the CTA raises the time-out bit of the status word,
 // drains the copies it has in flight, frees its TMEM and returns.
 #include <cudaTypedefs.h>
