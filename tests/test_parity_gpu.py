@@ -111,6 +111,8 @@ def test_logreg_workload_three_epochs_reduced():
     (32, 4, 9000, "bf16"),
     (64, 2, 20008, "bf16"),
     (70, 2, 3000, "bf16"),     # more workers than one 128-row tile holds
+    (300, 2, 1000, "bf16"),    # scan with G left in global memory
+    (1024, 2, 64, "f32"),      # the largest m the library accepts
 ])
 def test_shapes(m, n, d, dtype):
     rep = run_random_epoch(m, n, d, dtype, seed=m * 7 + d % 13)
