@@ -172,50 +172,38 @@ fma_combine_kernel(const double *__restrict__ partials, int blocks, int m, doubl
   }
 }
 
-// One thread: Algorithm 6 for i = 0..m-1 on t_i = b_i + sum_{k<i} s_k G_ki from the block totals
-// (triangle entries, then b), signs / margins / permutation slots (Algorithm 7) written out, the
-// signs also left in ssh as +-1.0f for the update that follows.
+// Decisions of the single-launch kernels: Algorithm 6 for i = 0..m-1 on
+// t_i = b_i + sum_{k<i} s_k G_ki from the block totals (triangle entries, then b), signs /
+// margins / permutation slots (Algorithm 7) written out.  The block totals are spread into the
+// scan's shared arrays (full G, b, the current pairs fetched by 2m threads at once), warp 0
+// takes the decisions with the chain in registers, the block writes out, and the signs land
+// in ssh as +-1.0f.  (A one-thread loop paid two dependent global loads per worker.)
 template <int M>
-__device__ __forceinline__ void fused_decide(const double *tot, int m, int n, int k,
-                                             const int32_t *__restrict__ perm_cur, int32_t *__restrict__ perm_next,
-                                             int8_t *__restrict__ signs, float *__restrict__ margins,
-                                             double *__restrict__ rnorm2, int *__restrict__ status,
-                                             const CdgRule &rule, float *ssh, bool write_out = true) {
-  double t[M];
-#pragma unroll
-  for (int i = 0; i < M; ++i) t[i] = tot[Tri<M>::NPAIR + i];
-  double rn2 = *rnorm2;
-  bool bad = false;
-  int oob = 0;
-  const int half = n >> 1;
-#pragma unroll
-  for (int i = 0; i < M; ++i) {
-    if (i < m) {
-      const double ti = t[i], gii = tot[Tri<M>::idx(i, i)];
-      const int s = cdg_decide(rule, i, ti, oob);   // greedy: +1 iff ||r+c|| < ||r-c||, a tie gives -1
-      bad |= !(isfinite(ti) && isfinite(gii));
-      const double sd = (double)s;
-#pragma unroll
-      for (int j = i + 1; j < M; ++j) t[j] += sd * tot[Tri<M>::idx(i, j)];
-      if (write_out) {
-        const size_t pos = (size_t)i * half + k;
-        signs[pos] = (int8_t)s;
-        const double den = rn2 * gii;
-        margins[pos] = (den > 0.0) ? (float)(fabs(ti) / sqrt(den)) : 0.f;
-        const int32_t first = perm_cur[(size_t)i * n + 2 * k];
-        const int32_t second = perm_cur[(size_t)i * n + 2 * k + 1];
-        perm_next[(size_t)i * n + k] = (s == 1) ? first : second;           // front slot
-        perm_next[(size_t)i * n + (n - 1 - k)] = (s == 1) ? second : first;  // back slot
-      }
-      rn2 += 2.0 * sd * ti + gii;
-      if (rn2 < 0.0) rn2 = 0.0;
-      ssh[i] = (float)s;
+__device__ __forceinline__ void fused_decide_block(const double *tot, double *scan_sh, int m, int n, int k,
+                                                   const int32_t *__restrict__ perm_cur,
+                                                   int32_t *__restrict__ perm_next, int8_t *__restrict__ signs,
+                                                   float *__restrict__ margins, double *__restrict__ rnorm2,
+                                                   int *__restrict__ status, const CdgRule &rule, float *ssh,
+                                                   bool write_out) {
+  const ScanSmem S = scan_smem(scan_sh, m);
+  if (threadIdx.x < Tri<M>::NACC) {
+    const int e = threadIdx.x;
+    const double v = tot[e];
+    if (e < Tri<M>::NPAIR) {
+      int a = 0, rem = e;
+      while (rem >= M - a) { rem -= M - a; ++a; }
+      const int b = a + rem;
+      if (a < m && b < m) { S.g[a * m + b] = v; S.g[b * m + a] = v; }
+    } else {
+      const int a = e - Tri<M>::NPAIR;
+      if (a < m) S.t[a] = v;
     }
   }
-  if (!write_out) return;
-  *rnorm2 = rn2;
-  if (bad) atomicOr(status, CDG_ST_NONFINITE);
-  if (oob) atomicAdd(rule.oob, (unsigned long long)oob);
+  scan_load_pairs(S, perm_cur, m, n, k);
+  __syncthreads();
+  scan_decide_and_write(S, S.g, m, n, k, perm_next, signs, margins, rnorm2, status, rule, -1.0, write_out);
+  if (threadIdx.x < m) ssh[threadIdx.x] = (float)S.s[threadIdx.x];
+  __syncthreads();
 }
 
 // ------------------------------------------------------------------------------------
@@ -235,7 +223,8 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
   constexpr int WARPS = FusedCfg<M>::THREADS / 32;
   double *red = dsh;                                  // [WARPS][NPAD]
   double *tot = red + WARPS * Tri<M>::NPAD;           // [NPAD]
-  float *ssh = reinterpret_cast<float *>(tot + Tri<M>::NPAD);  // [M]
+  double *scan_sh = tot + Tri<M>::NPAD;               // [4M + M*M] the scan's arrays
+  float *ssh = reinterpret_cast<float *>(scan_sh + 4 * M + M * M);  // [M]
   cdg_grid_dep_wait();            // r comes from the step before, the rows from the caller's last launch
 
   // `count` consecutive steps ([count][2][m][d] rows): r stays in this SM's cache between them
@@ -248,10 +237,7 @@ fused_step_kernel(const T *__restrict__ g, float *r, int m, int n, long long d, 
   const double v = block_reduce_acc<M, WARPS>(acc, red);
   if (threadIdx.x < Tri<M>::NACC) tot[threadIdx.x] = v;
   __syncthreads();
-
-  if (threadIdx.x == 0)
-    fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh);
-  __syncthreads();
+  fused_decide_block<M>(tot, scan_sh, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh, true);
 
   // r <- r + sum_i s_i c_i (i ascending), inputs re-read through the cache
   const size_t slab = (size_t)m * (size_t)d;
@@ -299,7 +285,8 @@ fused_step_cluster_kernel(const T *__restrict__ g, float *r, int m, int n, long 
   double *red = dsh;                                  // [WARPS][NPAD]
   double *mine = red + WARPS * Tri<M>::NPAD;          // [NPAD] this CTA's totals, read by the whole cluster
   double *tot = mine + Tri<M>::NPAD;                  // [NPAD] totals of the cluster
-  float *ssh = reinterpret_cast<float *>(tot + Tri<M>::NPAD);  // [M]
+  double *scan_sh = tot + Tri<M>::NPAD;               // [4M + M*M] the scan's arrays
+  float *ssh = reinterpret_cast<float *>(scan_sh + 4 * M + M * M);  // [M]
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned rank = cluster.block_rank(), csize = cluster.num_blocks();
   cdg_grid_dep_wait();            // r comes from the step before, the rows from the caller's last launch
@@ -321,9 +308,8 @@ fused_step_cluster_kernel(const T *__restrict__ g, float *r, int m, int n, long 
       tot[threadIdx.x] = sum;
     }
     cluster.sync();                                   // all remote reads done: `mine` may be rewritten
-    if (threadIdx.x == 0)
-      fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh, rank == 0);
-    __syncthreads();
+    fused_decide_block<M>(tot, scan_sh, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh,
+                          rank == 0);
 
     // r <- r + sum_i s_i c_i (i ascending) on this CTA's columns, inputs re-read through the cache
     for (long long vv = v0; vv < nvec; vv += vstride) {
@@ -389,7 +375,8 @@ fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ 
   double *mine = red + WARPS * Tri<M>::NPAD;          // [NPAD] this CTA's totals, read by the whole cluster
   double *tot = mine + Tri<M>::NPAD;                  // [NPAD] totals of the cluster
   double *dots = tot + Tri<M>::NPAD;                  // [2M] this CTA's share of <w, x>, read by the cluster
-  float *ssh = reinterpret_cast<float *>(dots + 2 * M);  // [M]
+  double *scan_sh = dots + 2 * M;                     // [4M + M*M] the scan's arrays
+  float *ssh = reinterpret_cast<float *>(scan_sh + 4 * M + M * M);  // [M]
   float *coef = ssh + M;                              // [2M]: a_0..a_{m-1}, b_0..b_{m-1}
   float *yv = coef + 2 * M;                           // [2M]
   size_t *rowoff = reinterpret_cast<size_t *>(yv + 2 * M);      // [2M] element offsets of the rows in X
@@ -479,9 +466,8 @@ fused_logreg_step_kernel(const float *__restrict__ X, const float *__restrict__ 
     tot[threadIdx.x] = sum;
   }
   cluster.sync();                                     // remote reads done before any CTA moves on or leaves
-  if (threadIdx.x == 0)
-    fused_decide<M>(tot, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh, rank == 0);
-  __syncthreads();
+  fused_decide_block<M>(tot, scan_sh, m, n, k, perm_cur, perm_next, signs, margins, rnorm2, status, rule, ssh,
+                        rank == 0);
 
   for (long long vv = v0; vv < nvec; vv += vstride) {
     const size_t x = (size_t)vv * 4;
@@ -508,7 +494,7 @@ template <int M, int THREADS>
 static cudaError_t launch_fused_logreg_tt(cdgrab_ctx *h, const float *X, const float *y, const float *w, int csize,
                                           cudaStream_t st) {
   constexpr int WARPS = THREADS / 32;
-  const size_t smem = (WARPS * Tri<M>::NPAD + 2 * Tri<M>::NPAD + 2 * M) * sizeof(double) +
+  const size_t smem = (WARPS * Tri<M>::NPAD + 2 * Tri<M>::NPAD + 2 * M + 4 * M + M * M) * sizeof(double) +
                       (M + 4 * M) * sizeof(float) + 2 * M * sizeof(size_t) + 16;
   static bool attr_set = false;
   if (!attr_set) {
@@ -576,7 +562,8 @@ static cudaError_t launch_fused_logreg_t(cdgrab_ctx *h, const float *X, const fl
 template <typename T, int M>
 static cudaError_t launch_fused_cluster_t(cdgrab_ctx *h, const void *grads, int count, int csize, cudaStream_t st) {
   constexpr int THREADS = ClusterCfg<M>::THREADS;
-  const size_t smem = ((THREADS / 32) * Tri<M>::NPAD + 2 * Tri<M>::NPAD) * sizeof(double) + M * sizeof(float);
+  const size_t smem = ((THREADS / 32) * Tri<M>::NPAD + 2 * Tri<M>::NPAD + 4 * M + M * M) * sizeof(double) +
+                      M * sizeof(float);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(csize); cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute at[2];
@@ -596,7 +583,7 @@ template <typename T, int M>
 static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, int count, cudaStream_t st) {
   const int csize = fused_cluster_size<M>(h);
   if (csize > 1) return launch_fused_cluster_t<T, M>(h, grads, count, csize, st);
-  const size_t smem = ((FusedCfg<M>::THREADS / 32) * Tri<M>::NPAD + Tri<M>::NPAD) * sizeof(double) +
+  const size_t smem = ((FusedCfg<M>::THREADS / 32) * Tri<M>::NPAD + Tri<M>::NPAD + 4 * M + M * M) * sizeof(double) +
                       M * sizeof(float);
   static bool attr_set = false;
   if (!attr_set) {

@@ -92,12 +92,13 @@ __device__ __forceinline__ void scan_load_pairs(const ScanSmem &S, const int32_t
 // S.t = b, S.p = pairs and G (shared or global, row-major [m][m]) must be ready and visible
 // to the block (barrier before the call).  Warp 0 decides, the block writes out.
 // rn2_in: ||r||^2 before the step when the caller fetched it ahead of time, else negative
-// (the routine then reads *rnorm2 itself).
+// (the routine then reads *rnorm2 itself).  write_out = false: decide only (signs in S.s),
+// nothing is written to global memory.
 __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const double *G, int m, int n, int k,
                                                       int32_t *__restrict__ perm_next, int8_t *__restrict__ signs,
                                                       float *__restrict__ margins, double *__restrict__ rnorm2,
                                                       int *__restrict__ status, const CdgRule rule,
-                                                      double rn2_in = -1.0) {
+                                                      double rn2_in = -1.0, bool write_out = true) {
   const int tid = threadIdx.x;
   if (tid < 32) {
     const int lane = tid;
@@ -146,13 +147,14 @@ __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const d
         __syncwarp();
       }
     }
-    if (lane == 0) {
+    if (lane == 0 && write_out) {
       *rnorm2 = rn2;
       if (bad) atomicOr(status, CDG_ST_NONFINITE);
       if (oob) atomicAdd(rule.oob, (unsigned long long)oob);
     }
   }
   __syncthreads();
+  if (!write_out) return;       // a replica of the decisions: S.s is all the caller needs
   const int half = n >> 1;
   for (int i = tid; i < m; i += blockDim.x) {
     const int s = S.s[i];
