@@ -173,7 +173,7 @@ NCU_TRAFFIC.update({
     # mid, pass 2: bytes of a cold launch (ncu flushes L2 between replays); live, a part of the rows
     # is still in L2 from pass 1 (128 MiB of inputs against 126 MB of L2)
     ("update", "mid"): {"bytes": 142.587e6, "files": ["kernels_generic.cu"], "source": "a491688bb66c82b0"},
-    ("gram", "mid"): {"bytes": 143.863e6, "files": ["kernels_fma.cu", "ptx.cuh", "scan.cuh"], "source": "d8c3b7513bd15886"},
+    ("gram", "mid"): {"bytes": 143.863e6, "files": ["kernels_fma.cu", "ptx.cuh", "scan.cuh"], "source": "c450b307a596bdd8"},
 })
 
 

@@ -539,7 +539,7 @@ bool cdg_fused_supported(int m, long long d, int dtype) {
   return m <= 16 && d % 4 == 0;
 }
 
-// CTAs per cluster for the spread-out step: one per THREADS column groups, a power of two, at most 8
+// CTAs per cluster for the spread-out step: one per THREADS column groups, 4 or 8, else a single CTA
 template <int M>
 static int fused_cluster_size(const cdgrab_ctx *h) {
   if (const char *e = getenv("CDGRAB_CLUSTER")) {
@@ -548,7 +548,7 @@ static int fused_cluster_size(const cdgrab_ctx *h) {
   const long long groups = (h->d / 4 + ClusterCfg<M>::THREADS - 1) / ClusterCfg<M>::THREADS;
   int c = 1;
   while (c < 8 && 2 * c <= groups) c *= 2;
-  return c;
+  return c >= 4 ? c : 1;      // two CTAs do not pay for the cluster barriers (measured at d = 1024)
 }
 
 template <int M>
