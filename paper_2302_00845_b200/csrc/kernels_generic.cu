@@ -316,15 +316,27 @@ update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__re
 // per-example logistic-regression gradient for the current pair of every worker
 // grid = (m, 2): block (i, q) handles item perm_cur[i][2k+q]
 // ------------------------------------------------------------------------------------
+template <bool VEC4>
 __global__ void __launch_bounds__(256)
 logreg_kernel(const float *__restrict__ X, const float *__restrict__ y, const float *__restrict__ w,
               const int32_t *__restrict__ perm_cur, int m, int n, long long d, int k,
               float *__restrict__ out) {
+  cdg_grid_dep_wait();            // the buffer may still be read by the step launched before
   const int i = blockIdx.x, q = blockIdx.y;
   const int item = perm_cur[(size_t)i * n + 2 * k + q];
   const float *x = X + ((size_t)i * n + item) * (size_t)d;
   float part = 0.f;
-  for (long long c = threadIdx.x; c < d; c += blockDim.x) part = fmaf(w[c], x[c], part);
+  if constexpr (VEC4) {           // d % 4 == 0 and 16-byte aligned bases: the row stays in registers
+    const long long nvec = d / 4;
+    for (long long c = threadIdx.x; c < nvec; c += blockDim.x) {
+      const float4 wv = __ldg(reinterpret_cast<const float4 *>(w) + c);
+      const float4 xv = __ldg(reinterpret_cast<const float4 *>(x) + c);
+      part = fmaf(wv.x, xv.x, part); part = fmaf(wv.y, xv.y, part);
+      part = fmaf(wv.z, xv.z, part); part = fmaf(wv.w, xv.w, part);
+    }
+  } else {
+    for (long long c = threadIdx.x; c < d; c += blockDim.x) part = fmaf(w[c], x[c], part);
+  }
   __shared__ double red[8];
   __shared__ float coef;
   double v = (double)part;
@@ -343,7 +355,15 @@ logreg_kernel(const float *__restrict__ X, const float *__restrict__ y, const fl
   __syncthreads();
   const float cf = coef;
   float *o = out + ((size_t)q * m + i) * (size_t)d;
-  for (long long c = threadIdx.x; c < d; c += blockDim.x) o[c] = cf * x[c];
+  if constexpr (VEC4) {
+    const long long nvec = d / 4;
+    for (long long c = threadIdx.x; c < nvec; c += blockDim.x) {
+      const float4 xv = __ldg(reinterpret_cast<const float4 *>(x) + c);   // second read: from L1/L2
+      reinterpret_cast<float4 *>(o)[c] = make_float4(cf * xv.x, cf * xv.y, cf * xv.z, cf * xv.w);
+    }
+  } else {
+    for (long long c = threadIdx.x; c < d; c += blockDim.x) o[c] = cf * x[c];
+  }
 }
 
 // ------------------------------------------------------------------------------------
@@ -483,7 +503,13 @@ cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, con
   dim3 grid(h->m, 2);
   {
     CdgProfScope ps(h, CDGRAB_K_LOGREG, st);
-    logreg_kernel<<<grid, 256, 0, st>>>(X, y, w, h->perm_cur, h->m, h->n, h->d, h->k, out);
+    const bool vec4 = h->d % 4 == 0 && ((((uintptr_t)X) | ((uintptr_t)w) | ((uintptr_t)out)) & 15) == 0;
+    if (vec4)
+      cdg_launch_dep(h, logreg_kernel<true>, grid, dim3(256), 0, st, X, y, w, (const int32_t *)h->perm_cur, h->m,
+                     h->n, h->d, h->k, out);
+    else
+      cdg_launch_dep(h, logreg_kernel<false>, grid, dim3(256), 0, st, X, y, w, (const int32_t *)h->perm_cur, h->m,
+                     h->n, h->d, h->k, out);
   }
   return cudaGetLastError();
 }
