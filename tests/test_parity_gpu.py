@@ -221,6 +221,24 @@ def test_deterministic_bitwise():
 
 
 # ---- state machine and arguments ---------------------------------------------------------------
+@pytest.mark.parametrize("m,n,d,dtype", [(4, 6, 1024, "f32"), (8, 4, 4096, "f32"), (16, 4, 300_000, "f32"),
+                                       (32, 4, 100_032, "bf16"), (64, 4, 70_000, "bf16"), (5, 4, 1001, "f32")])
+def test_chained_launches_change_nothing(m, n, d, dtype, monkeypatch):
+    """Launches queued behind their predecessor (the default) and plain stream order give the same bits."""
+    outs = []
+    for pdl in ("1", "0"):
+        monkeypatch.setenv("CDGRAB_PDL", pdl)
+        with binding.CdGrab(m, n, d, dtype) as h:
+            h.begin_epoch()
+            for k in range(n // 2):
+                h.step(random_grads(m, d, dtype, 90 + k))
+            out = torch.empty(m, n, dtype=torch.int32, device="cuda")
+            h.end_epoch(out)
+            outs.append((h.signs().cpu(), h.r().cpu(), h.margins().cpu(), out.cpu()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
 def test_state_machine_and_argument_errors():
     m, n, d = 2, 4, 64
     L = binding.lib()
