@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcdgrab.so")
-SOURCES = ["api.cu", "kernels_generic.cu", "kernels_fma.cu", "kernels_umma.cu", "noalloc.cu", "herding.cu", "kernels_indep.cu"]
+SOURCES = ["api.cu", "kernels_generic.cu", "kernels_fma.cu", "kernels_umma.cu", "noalloc.cu", "herding.cu", "kernels_indep.cu", "kernels_block.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",

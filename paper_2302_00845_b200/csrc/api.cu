@@ -168,6 +168,10 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
       // sized for the larger of the two grids that may write it: this kernel's (<= 2 per SM)
       // and the TMA-fed kernel's (one CTA per SM whatever the row length)
       h->partials_bytes = sizeof(double) * 152 * (size_t)h->num_sms * 2;
+    } else if (m > 16 && !(getenv("CDGRAB_GRAM_BLOCK") && atoi(getenv("CDGRAB_GRAM_BLOCK")) == 0)) {
+      h->gram_block = 1;
+      h->gram_chunks = cdg_block_ctas(h);
+      h->partials_bytes = cdg_block_partials_bytes(h);
     } else {
       const int ntile = (m + CDG_TM - 1) / CDG_TM;
       const int npairs = ntile * (ntile + 1) / 2;

@@ -49,6 +49,7 @@ struct cdgrab_ctx {
   float *mean_out;       // [2][d] destination of the averaged gather buffers for the step being enqueued, or NULL
   size_t partials_bytes;
   int gram_chunks;       // grid.x of the FMA Gram kernels
+  int gram_block;        // 1: the generic pass 1 is the blocked kernel (m > 16)
 
   // TMA-pipelined FMA Gram
   int fma_tma;             // 1 when that kernel serves pass 1
@@ -139,6 +140,9 @@ inline cudaError_t cdg_launch_dep(const cdgrab_ctx *h, void (*kernel)(KArgs...),
 
 // ---- launchers (each returns a cudaError_t; every kernel launch sits in a CdgProfScope) ----------
 cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+cudaError_t cdg_launch_gram_block(cdgrab_ctx *h, const void *grads, cudaStream_t st);   // m > 16: 64-row blocks
+int cdg_block_ctas(const cdgrab_ctx *h);
+size_t cdg_block_partials_bytes(const cdgrab_ctx *h);
 cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st);
 cudaError_t cdg_launch_update(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 cudaError_t cdg_launch_mean(cdgrab_ctx *h, const void *grads, cudaStream_t st);

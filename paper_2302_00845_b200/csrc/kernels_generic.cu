@@ -370,6 +370,7 @@ logreg_kernel(const float *__restrict__ X, const float *__restrict__ y, const fl
 // launchers
 // ------------------------------------------------------------------------------------
 cudaError_t cdg_launch_gram_generic(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  if (h->gram_block) return cdg_launch_gram_block(h, grads, st);
   const int ntile = (h->m + CDG_TM - 1) / CDG_TM;
   const int npairs = ntile * (ntile + 1) / 2;
   dim3 grid(h->gram_chunks, npairs);
