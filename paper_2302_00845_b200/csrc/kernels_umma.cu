@@ -340,47 +340,42 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   }
 }
 
-// G and b from the per-CTA partial H in fp64.  A block handles 32 consecutive entries
-// (e < m*m: (k, i) = (e / m, e % m);  m*m <= e < m*m + m: b_i); warp w sums the CTAs
-// w, w+8, w+16, ... in that order, the eight warp sums are then added in warp order.
+// G and b from the per-CTA partial H in fp64.  A warp handles one entry (e < m*m: (k, i) =
+// (e / m, e % m);  m*m <= e < m*m + m: b_i): lane l adds the CTAs l, l+32, ... in that order, the
+// 32 lane sums are then added by a fixed butterfly.  Eight entries per block spread the loads
+// over many SMs (an SM can keep only so many of these scattered loads in flight).
 __global__ void __launch_bounds__(256)
 umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows, int m,
                     double *__restrict__ gram, int *__restrict__ status, const CdgTail tail) {
-  __shared__ double part[8][32];
   __shared__ double scan_sh[4 * 64 + 64 * 64];     // m <= 64 on this path
   __shared__ int is_last;
-  const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   cdg_grid_dep_wait();            // the partial H come from the launch before this one
   const int total = m * m + m;
-  const int e = blockIdx.x * 32 + lane;
+  const int e = blockIdx.x * 8 + warp;
   const size_t cs = (size_t)128 * ncols;   // one CTA's partial H
   double acc = 0.0;
   if (e < m * m) {
     const int k = e / m, i = e % m;
     const size_t o00 = (size_t)k * ncols + i, o01 = o00 + m, o10 = (size_t)(m + k) * ncols + i, o11 = o10 + m;
-#pragma unroll 4
-    for (int c = slice; c < ctas; c += 8) {
+#pragma unroll 5
+    for (int c = lane; c < ctas; c += 32) {
       const float *P = partials + (size_t)c * cs;
       acc += ((double)P[o00] - (double)P[o01]) - ((double)P[o10] - (double)P[o11]);
     }
   } else if (e < total) {
     const int i = e - m * m;
     const size_t o0 = (size_t)i * ncols + box_rows, o1 = (size_t)(m + i) * ncols + box_rows;
-#pragma unroll 4
-    for (int c = slice; c < ctas; c += 8) {
+#pragma unroll 5
+    for (int c = lane; c < ctas; c += 32) {
       const float *P = partials + (size_t)c * cs;
       acc += (((double)P[o0] - (double)P[o1]) + ((double)P[o0 + 1] - (double)P[o1 + 1])) +
              ((double)P[o0 + 2] - (double)P[o1 + 2]);
     }
   }
-  part[slice][lane] = acc;
-  __syncthreads();
-  if (slice == 0 && e < total) {
-    double v = 0.0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) v += part[w][lane];
-    gram[e] = v;
-  }
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (lane == 0 && e < total) gram[e] = acc;
   if (!tail.enabled) return;
 
   // ---- the block that takes the last ticket has all of (G, b) before it: it decides ----
@@ -597,7 +592,7 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
     const int total = h->m * h->m + h->m;
-    cdg_launch_dep(h, umma_combine_kernel, dim3((total + 31) / 32), dim3(256), 0, st, h->umma_partials, h->umma_ctas,
+    cdg_launch_dep(h, umma_combine_kernel, dim3((total + 7) / 8), dim3(256), 0, st, h->umma_partials, h->umma_ctas,
                    h->umma_ncols, h->umma_box_rows, h->m, h->gram, h->status, cdg_tail_of(h, h->umma_fused));
   }
   return cudaGetLastError();
