@@ -128,3 +128,13 @@ def test_sharded_wrapper_all_reduces_the_partial_sums_world_size_2_gloo():
         assert p.exitcode == 0
     want = [3.0 * i for i in range(3 * 3 + 3)]          # rank 0 gives i, rank 1 gives 2 i
     assert out[0] == [want, want] and out[1] == out[0]  # both ranks finish on the same bits
+
+
+def test_traffic_figures_match_the_kernel_sources():
+    """Every DRAM-traffic figure bench.py reports is tied to the kernel files it was captured with;
+    a figure whose files changed reads null in the bench line, and this test says which one to
+    capture again (or to re-key, when the edit left the kernel itself alone)."""
+    sys.path.insert(0, ROOT)
+    import bench
+    stale = [k for k, v in bench.NCU_TRAFFIC.items() if v["source"] != bench.source_hash(v["files"])]
+    assert not stale, f"ncu traffic figures out of date for {stale}"
