@@ -90,6 +90,9 @@ struct cdgrab_ctx {
   int umma_g4;             // row groups one 4-D copy brings in (0: per-group copies only)
   int umma_paired;         // 2m <= 64: one MMA covers two 64-column blocks
   int umma_fused;          // the combine launch also takes the decisions (last block)
+  int umma_split3;         // fp32 inputs: the MMA rows are the differences as three bf16 terms each
+  int umma_rows;           // rows of the MMA operand: 2m (bf16 gradients) or 3m (split differences)
+  __nv_bfloat16 *umma_csplit;   // [3m][d_pad] hi / mid / lo terms of c_i = z1_i - z2_i (fp32 inputs)
 };
 
 template <typename T>

@@ -345,7 +345,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
 // 32 lane sums are then added by a fixed butterfly.  Eight entries per block spread the loads
 // over many SMs (an SM can keep only so many of these scattered loads in flight).
 __global__ void __launch_bounds__(256)
-umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows, int m,
+umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows, int m, int split3,
                     double *__restrict__ gram, int *__restrict__ status, const CdgTail tail) {
   __shared__ double scan_sh[4 * 64 + 64 * 64];     // m <= 64 on this path
   __shared__ int is_last;
@@ -355,7 +355,34 @@ umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int
   const int e = blockIdx.x * 8 + warp;
   const size_t cs = (size_t)128 * ncols;   // one CTA's partial H
   double acc = 0.0;
-  if (e < m * m) {
+  if (split3) {
+    // rows p*m + i hold term p (hi, mid, lo) of c_i:  G_ki = sum over the nine term pairs,
+    // b_i = sum over the three terms of row i and the three terms of r
+    if (e < m * m) {
+      const int k = e / m, i = e % m;
+      for (int c = lane; c < ctas; c += 32) {
+        const float *P = partials + (size_t)c * cs;
+        double v = 0.0;
+#pragma unroll
+        for (int pa = 0; pa < 3; ++pa)
+#pragma unroll
+          for (int pb = 0; pb < 3; ++pb) v += (double)P[(size_t)(pa * m + k) * ncols + pb * m + i];
+        acc += v;
+      }
+    } else if (e < total) {
+      const int i = e - m * m;
+      for (int c = lane; c < ctas; c += 32) {
+        const float *P = partials + (size_t)c * cs;
+        double v = 0.0;
+#pragma unroll
+        for (int pa = 0; pa < 3; ++pa) {
+          const size_t o = (size_t)(pa * m + i) * ncols + box_rows;
+          v += ((double)P[o] + (double)P[o + 1]) + (double)P[o + 2];
+        }
+        acc += v;
+      }
+    }
+  } else if (e < m * m) {
     const int k = e / m, i = e % m;
     const size_t o00 = (size_t)k * ncols + i, o01 = o00 + m, o10 = (size_t)(m + k) * ncols + i, o11 = o10 + m;
 #pragma unroll 5
@@ -393,6 +420,45 @@ umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int
   __syncthreads();
   scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
                         tail.rule);
+}
+
+// fp32 gradients: c_i = z1_i - z2_i (rounded to fp32 like every other path forms it) written as
+// three bf16 terms hi + mid + lo = c exactly (3 x 8 significand bits), rows [term][worker] of
+// out[3m][d_pad].  Products of bf16 terms are exact in the fp32 accumulator, so the nine term
+// products of a pair add up to c_k c_i without a rounded product.  grid (column chunks, m).
+__global__ void __launch_bounds__(256)
+split_diff_kernel(const float *__restrict__ g, int m, long long d, long long d_pad,
+                  __nv_bfloat16 *__restrict__ out) {
+  cdg_grid_dep_wait();            // the last launch may still read the terms of the step before
+  const int i = blockIdx.y;
+  const float *z1 = g + (size_t)i * (size_t)d, *z2 = g + ((size_t)m + i) * (size_t)d;
+  __nv_bfloat16 *o0 = out + (size_t)i * (size_t)d_pad;
+  __nv_bfloat16 *o1 = out + ((size_t)m + i) * (size_t)d_pad;
+  __nv_bfloat16 *o2 = out + (2 * (size_t)m + i) * (size_t)d_pad;
+  const long long nvec = d / 8;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += (long long)gridDim.x * blockDim.x) {
+    const size_t x = (size_t)v * 8;
+    float a[8], b[8];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const float4 fa = __ldg(reinterpret_cast<const float4 *>(z1 + x) + q);
+      const float4 fb = __ldg(reinterpret_cast<const float4 *>(z2 + x) + q);
+      a[4 * q] = fa.x; a[4 * q + 1] = fa.y; a[4 * q + 2] = fa.z; a[4 * q + 3] = fa.w;
+      b[4 * q] = fb.x; b[4 * q + 1] = fb.y; b[4 * q + 2] = fb.z; b[4 * q + 3] = fb.w;
+    }
+    __nv_bfloat16 hi[8], mid[8], lo[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float c = a[j] - b[j];
+      hi[j] = __float2bfloat16_rn(c);
+      const float r1 = c - __bfloat162float(hi[j]);
+      mid[j] = __float2bfloat16_rn(r1);
+      lo[j] = __float2bfloat16_rn(r1 - __bfloat162float(mid[j]));
+    }
+    *reinterpret_cast<uint4 *>(o0 + x) = *reinterpret_cast<const uint4 *>(hi);
+    *reinterpret_cast<uint4 *>(o1 + x) = *reinterpret_cast<const uint4 *>(mid);
+    *reinterpret_cast<uint4 *>(o2 + x) = *reinterpret_cast<const uint4 *>(lo);
+  }
 }
 
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
@@ -478,16 +544,25 @@ cudaError_t cdg_launch_wait_selftest(cdgrab_ctx *h, long long cycles, long long 
 void *cdg_tensor_map_encoder() { return (void *)encode_fn(); }
 
 bool cdg_umma_supported(int m, long long d, int dtype) {
-  // bf16 rows whose pitch is a multiple of 16 bytes; 2m rows fit one 128-row MMA tile
-  return dtype == CDGRAB_BF16 && m <= 64 && d % 8 == 0 && d >= 4096 && encode_fn() != nullptr;
+  // rows whose pitch is a multiple of 16 bytes
+  if (d % 8 != 0 || d < 4096 || encode_fn() == nullptr) return false;
+  // bf16 gradients: the 2m rows fit one 128-row MMA tile
+  if (dtype == CDGRAB_BF16) return m <= 64;
+  // fp32 gradients: the differences as three bf16 terms each, 3m rows (CDGRAB_UMMA_F32=0: not used)
+  if (const char *e = getenv("CDGRAB_UMMA_F32")) {
+    if (atoi(e) == 0) return false;
+  }
+  return 3 * m <= 128;
 }
 
 int cdg_umma_setup(cdgrab_ctx *h) {
-  h->umma_paired = (2 * h->m <= 64) ? 1 : 0;      // CDGRAB_UMMA_PAIRED=0: one block per MMA
+  h->umma_split3 = (h->dtype == CDGRAB_F32) ? 1 : 0;
+  h->umma_rows = h->umma_split3 ? 3 * h->m : 2 * h->m;
+  h->umma_paired = (h->umma_rows <= 64) ? 1 : 0;  // CDGRAB_UMMA_PAIRED=0: one block per MMA
   if (const char *e = getenv("CDGRAB_UMMA_PAIRED")) {
     if (atoi(e) == 0) h->umma_paired = 0;
   }
-  const int box_rows = h->umma_paired ? 64 : ((2 * h->m + 15) / 16) * 16;
+  const int box_rows = h->umma_paired ? 64 : ((h->umma_rows + 15) / 16) * 16;
   h->umma_box_rows = box_rows;
   h->umma_ncols = box_rows + kRBoxRows;
   // 64-column blocks per stage: stages of roughly 70-80 KB measured best (4 blocks at m = 64,
@@ -502,7 +577,9 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   if (h->umma_paired && (subs & 1)) ++subs;      // two halves per stage
   h->umma_subs_per_stage = subs;
   // TMEM chunk length in pipeline iterations (about 4096 columns); CDGRAB_UMMA_DRAIN overrides
-  h->umma_drain = 4096 / (subs * kSubCols) > 0 ? 4096 / (subs * kSubCols) : 1;
+  // (fp32 inputs are held to a tighter sign tolerance: chunks of about 512 columns)
+  const int chunk_cols = h->umma_split3 ? 512 : 4096;
+  h->umma_drain = chunk_cols / (subs * kSubCols) > 0 ? chunk_cols / (subs * kSubCols) : 1;
   if (const char *e = getenv("CDGRAB_UMMA_DRAIN")) {
     const int v = atoi(e);
     if (v >= 1 && v <= (1 << 20)) h->umma_drain = v;
@@ -530,6 +607,11 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     cudaGetLastError();
     return CDGRAB_ERR_NOMEM;
   }
+  if (h->umma_split3) {
+    const size_t bytes = sizeof(__nv_bfloat16) * 3 * (size_t)h->m * (size_t)h->d_pad;
+    if (cudaMalloc(&h->umma_csplit, bytes) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_NOMEM; }
+    if (cudaMemset(h->umma_csplit, 0, bytes) != cudaSuccess) return CDGRAB_ERR_CUDA;
+  }
   if (cudaMemset(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
       cudaMemset(h->umma_partials, 0, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess)
     return CDGRAB_ERR_CUDA;
@@ -552,31 +634,45 @@ int cdg_umma_setup(cdgrab_ctx *h) {
 void cdg_umma_teardown(cdgrab_ctx *h) {
   cudaFree(h->r_split);
   cudaFree(h->umma_partials);
+  cudaFree(h->umma_csplit);
+  h->umma_csplit = nullptr;
   h->r_split = nullptr;
   h->umma_partials = nullptr;
 }
 
 cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
   const long long nblk_full = h->d / kSubCols;
-  if (grads != h->tm_g_base) {
+  // the MMA's rows: the caller's bf16 gradients, or the split differences of fp32 gradients
+  const void *src = h->umma_split3 ? (const void *)h->umma_csplit : grads;
+  const long long pitch = h->umma_split3 ? h->d_pad : h->d;
+  const int rows = h->umma_rows;
+  if (h->umma_split3) {
+    long long chunks = (h->d / 8 + 255) / 256;
+    const long long cap = (8ll * h->num_sms + h->m - 1) / h->m;
+    if (chunks > cap) chunks = cap;
+    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
+    cdg_launch_dep(h, split_diff_kernel, dim3((unsigned)chunks, h->m), dim3(256), 0, st, (const float *)grads, h->m,
+                   h->d, h->d_pad, h->umma_csplit);
+  }
+  if (src != h->tm_g_base) {
     const int box_blocks = h->umma_paired ? h->umma_subs_per_stage / 2 : h->umma_subs_per_stage;
-    if (!encode_map_3d(&h->tm_g, grads, nblk_full, 2 * h->m, h->d, box_blocks) ||
-        !encode_map_2d(&h->tm_g2, grads, h->d, 2 * h->m, h->d))
+    if (!encode_map_3d(&h->tm_g, src, nblk_full, rows, pitch, box_blocks) ||
+        !encode_map_2d(&h->tm_g2, src, h->d, rows, pitch))
       return cudaErrorInvalidValue;
     // one copy for all full row groups of a (half) stage; CDGRAB_UMMA_G4=0: per-group copies only
-    h->umma_g4 = (2 * h->m) / 8;
+    h->umma_g4 = rows / 8;
     if (const char *e = getenv("CDGRAB_UMMA_G4")) {
       if (atoi(e) == 0) h->umma_g4 = 0;
     }
-    if ((long long)h->d * 16 >= (1ll << 40)) h->umma_g4 = 0;     // the group stride must fit the map
-    if (h->umma_g4 > 0 && !encode_map_4d(&h->tm_g4, grads, nblk_full, h->umma_g4, h->d, box_blocks)) h->umma_g4 = 0;
+    if (pitch * 16 >= (1ll << 40)) h->umma_g4 = 0;               // the group stride must fit the map
+    if (h->umma_g4 > 0 && !encode_map_4d(&h->tm_g4, src, nblk_full, h->umma_g4, pitch, box_blocks)) h->umma_g4 = 0;
     if (h->umma_g4 == 0) h->tm_g4 = h->tm_g;
-    h->tm_g_base = grads;
+    h->tm_g_base = src;
   }
   UmmaParams p;
   p.box_rows = h->umma_box_rows;
   p.ncols = h->umma_ncols;
-  p.rows_used = 2 * h->m;
+  p.rows_used = rows;
   p.subs = h->umma_subs_per_stage;
   p.stages = h->umma_stages;
   p.nblk_full = nblk_full;
@@ -593,7 +689,8 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
     const int total = h->m * h->m + h->m;
     cdg_launch_dep(h, umma_combine_kernel, dim3((total + 7) / 8), dim3(256), 0, st, h->umma_partials, h->umma_ctas,
-                   h->umma_ncols, h->umma_box_rows, h->m, h->gram, h->status, cdg_tail_of(h, h->umma_fused));
+                   h->umma_ncols, h->umma_box_rows, h->m, h->umma_split3, h->gram, h->status,
+                   cdg_tail_of(h, h->umma_fused));
   }
   return cudaGetLastError();
 }

@@ -27,6 +27,31 @@ def run(m, n, d, seed, mean=0.0, scale=1.0):
 
 
 @pytest.mark.parametrize("m,n,d", [
+    (17, 4, 5000),           # 51 rows of bf16 terms: two blocks per MMA, ragged last block
+    (24, 4, 200_000),        # 72 rows: one block per MMA
+    (42, 4, 70_000),         # 126 rows: the largest m of this mode
+    (32, 6, 1_000_000 + 8),  # many accumulator chunks per CTA
+    (8, 4, 100_000),         # forced onto this path (the FMA kernels are the default for m <= 16)
+])
+def test_fp32_gradients_on_the_tensor_cores(m, n, d, monkeypatch):
+    """fp32 inputs: the differences go through the MMA as three bf16 terms each; the fp32 sign
+    tolerance (1e-6) applies."""
+    monkeypatch.setenv("CDGRAB_FORCE_PATH", "umma")
+    pr = Pair(m, n, d, "f32")
+    try:
+        assert pr.gpu.path == "umma"
+        pr.begin()
+        g = torch.Generator(device="cuda").manual_seed(m + d % 11)
+        for k in range(n // 2):
+            pr.step(torch.randn(2, m, d, generator=g, device="cuda") + 0.1)
+        rep = pr.end()
+        print(f"umma fp32 m={m} n={n} d={d}:", rep)
+        assert rep.raw_agreement > 0.95
+    finally:
+        pr.close()
+
+
+@pytest.mark.parametrize("m,n,d", [
     (4, 4, 4096),          # one 16-row box, few K blocks: fewer CTAs than SMs
     (64, 4, 8192),         # full 128-row tile
     (32, 4, 64 * 148 * 3 + 8),   # every SM busy, ragged last K block
