@@ -25,6 +25,8 @@ def grads(m, d, dtype, seed):
     (4, 4_096, "f32", [0, 2_048, 4_096]),                # small: register Gram, never the one-launch path
     (16, 300_000, "f32", [0, 70_000, 200_000, 300_000]), # three uneven shards
     (5, 3_003, "f32", [0, 1_001, 3_003]),                # generic tiles
+    (24, 80_000, "f32", [0, 40_000, 80_000]),            # fp32 on the tensor cores (three bf16 terms)
+    (48, 10_000, "f32", [0, 6_000, 10_000]),             # blocked FMA Gram
 ])
 def test_sharded_steps_match_oracle(m, d, dtype, cuts):
     n = 6
