@@ -15,7 +15,8 @@ def grads(m, d, dtype, seed):
 
 
 @pytest.mark.parametrize("m,d,dtype,independent", [(4, 2048, "f32", False), (16, 150_000, "f32", False),
-                                                    (32, 40_000, "bf16", False), (6, 30_000, "bf16", True)])
+                                                    (32, 40_000, "bf16", False), (6, 30_000, "bf16", True),
+                                                    (24, 40_000, "f32", False), (48, 6_000, "f32", False)])
 def test_resume_is_bit_identical(m, d, dtype, independent):
     n = 8
     steps = [grads(m, d, dtype, 50 + k) for k in range(n)]          # two epochs of n/2 steps
