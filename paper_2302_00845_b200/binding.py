@@ -303,13 +303,14 @@ class ShardedCdGrab:
     """One rank of a column-sharded order server over ``torch.distributed``: this rank owns
     d_local columns; every step all-reduces m*m + m doubles (NCCL on GPUs)."""
 
-    def __init__(self, m: int, n: int, d_local: int, dtype="f32", group=None, handle=None,
-                 device="cuda"):
-        """``handle``: an object with step_begin / step_finish / begin_epoch / end_epoch / destroy
-        to drive instead of a new shard handle (host-side tests of the exchange)."""
-        import torch
-        self.h = handle if handle is not None else CdGrab(m, n, d_local, dtype, shard=True)
+    def __init__(self, m: int, n: int, d_local: int, dtype="f32", group=None):
         self.group = group
+        self._attach(CdGrab(m, n, d_local, dtype, shard=True), m, "cuda")
+
+    def _attach(self, handle, m: int, device):
+        """The shard handle this rank drives and the buffer its partial (G, b) is exchanged in."""
+        import torch
+        self.h = handle
         self.gram = torch.empty(m * m + m, dtype=torch.float64, device=device)
 
     def begin_epoch(self):

@@ -14,6 +14,14 @@ namespace {
 
 inline bool valid(const cdgrab_ctx *h) { return h && h->magic == CDG_MAGIC; }
 
+// A handle's buffers, tensor maps and kernel attributes belong to the device it was created on;
+// work may only be enqueued while that device is current.
+inline bool on_own_device(const cdgrab_ctx *h) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return false; }
+  return dev == h->device;
+}
+
 inline size_t elem_size(int dtype) { return dtype == CDGRAB_F32 ? 4 : 2; }
 
 __global__ void iota_perm_kernel(int32_t *p, int m, int n) {
@@ -118,6 +126,7 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
   h->shard = shard;
   h->pdl = 1;                      // CDGRAB_PDL=0: plain stream order between the launches of a step
   if (const char *e = getenv("CDGRAB_PDL")) h->pdl = atoi(e) ? 1 : 0;
+  if (const char *e = getenv("CDGRAB_CLUSTER")) h->cluster_off = atoi(e) ? 0 : 1;
 
   // ---- choose the path ------------------------------------------------------------
   const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);
@@ -260,6 +269,7 @@ int cdgrab_set_perms(cdgrab_t *h, const int32_t *perms_in) {
 
 int cdgrab_begin_epoch(cdgrab_t *h, void *stream) {
   if (!valid(h)) return CDGRAB_ERR_INVALID;
+  if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (h->epoch_open) return CDGRAB_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e = cudaMemsetAsync(h->r, 0, sizeof(float) * (size_t)h->d * (h->independent ? (size_t)h->m : 1), st);
@@ -285,6 +295,7 @@ static cudaError_t launch_pass1(cdgrab_ctx *h, const void *grads_dev, cudaStream
 int cdgrab_step_begin(cdgrab_t *h, const void *grads_dev, double *gram_out_dev, void *stream) {
   if (!valid(h) || !grads_dev || !gram_out_dev || !h->shard) return CDGRAB_ERR_INVALID;
   if ((((uintptr_t)grads_dev & 15) | ((uintptr_t)gram_out_dev & 7)) != 0) return CDGRAB_ERR_INVALID;
+  if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (!h->epoch_open || h->k >= h->n / 2 || h->shard_pending) return CDGRAB_ERR_STATE;
   double *own = h->gram;
   h->gram = gram_out_dev;                       // pass 1 leaves this shard's partial (G, b) there
@@ -297,6 +308,9 @@ int cdgrab_step_begin(cdgrab_t *h, const void *grads_dev, double *gram_out_dev, 
 
 int cdgrab_step_finish(cdgrab_t *h, const void *grads_dev, const double *gram_in_dev, void *stream) {
   if (!valid(h) || !grads_dev || !gram_in_dev || !h->shard) return CDGRAB_ERR_INVALID;
+  // pass 2 reads the rows with 16-byte vector loads, the scan reads doubles
+  if ((((uintptr_t)grads_dev & 15) | ((uintptr_t)gram_in_dev & 7)) != 0) return CDGRAB_ERR_INVALID;
+  if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (!h->epoch_open || !h->shard_pending) return CDGRAB_ERR_STATE;
   double *own = h->gram;
   h->gram = const_cast<double *>(gram_in_dev);  // the sum over all shards
@@ -313,6 +327,7 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
   if (!valid(h) || !grads_dev) return CDGRAB_ERR_INVALID;
   if (((uintptr_t)grads_dev & 15) != 0) return CDGRAB_ERR_INVALID;
   if (h->shard) return CDGRAB_ERR_INVALID;   // a shard steps through cdgrab_step_begin / _finish
+  if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
@@ -335,6 +350,7 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
 int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream) {
   if (!valid(h) || !grads_dev || count < 1) return CDGRAB_ERR_INVALID;
   if (((uintptr_t)grads_dev & 15) != 0 || h->shard) return CDGRAB_ERR_INVALID;
+  if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (!h->epoch_open || h->k + count > h->n / 2) return CDGRAB_ERR_STATE;
   const size_t step_bytes = 2 * (size_t)h->m * (size_t)h->d * (h->dtype == CDGRAB_F32 ? 4 : 2);
   if (h->path == CDGRAB_PATH_FUSED && !h->independent && !h->rule_randomized && !h->mean_out) {
@@ -357,6 +373,7 @@ int cdgrab_step_logreg(cdgrab_t *h, const float *X, const float *y, const float 
   if (!valid(h) || !X || !y || !w) return CDGRAB_ERR_INVALID;
   if (h->dtype != CDGRAB_F32 || h->path != CDGRAB_PATH_FUSED) return CDGRAB_ERR_INVALID;
   if ((((uintptr_t)X | (uintptr_t)w) & 15) != 0) return CDGRAB_ERR_INVALID;
+  if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
   if (cdg_launch_fused_logreg(h, X, y, w, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   h->k++;
@@ -381,6 +398,7 @@ long long cdgrab_out_of_bound(cdgrab_t *h) {
 
 int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, void *stream) {
   if (!valid(h) || !mean_out_dev) return CDGRAB_ERR_INVALID;
+  if (((uintptr_t)mean_out_dev & 15) != 0) return CDGRAB_ERR_INVALID;   // written with 16-byte vector stores
   h->mean_out = mean_out_dev;
   int rc = cdgrab_step(h, grads_dev, stream);
   if (rc == CDGRAB_OK && h->path == CDGRAB_PATH_FUSED) {
@@ -590,6 +608,7 @@ int cdgrab_logreg_grads(cdgrab_t *h, const float *X, const float *y, const float
                         void *stream) {
   if (!valid(h) || !X || !y || !w || !grads_out) return CDGRAB_ERR_INVALID;
   if (h->dtype != CDGRAB_F32) return CDGRAB_ERR_INVALID;
+  if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
   if (cdg_launch_logreg(h, X, y, w, grads_out, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();

@@ -18,6 +18,26 @@
 #define CDG_TM 8
 #define CDG_TILE_ENTRIES (CDG_TM * CDG_TM + CDG_TM)
 
+// Tensor maps are encoded for a base address.  Callers alternate between a few gradient buffers
+// (double buffering), so the maps of the last kCdgMapSlots bases are kept; a new base replaces
+// the oldest entry.
+constexpr int kCdgMapSlots = 4;
+template <int N>
+struct CdgMapCache {
+  const void *base[kCdgMapSlots];
+  CUtensorMap maps[kCdgMapSlots][N];
+  int next;
+  // slot holding the maps of `b`, or -1
+  int find(const void *b) const {
+    for (int i = 0; i < kCdgMapSlots; ++i)
+      if (base[i] == b) return i;
+    return -1;
+  }
+  // slot to encode the maps of a new base into (its old entry is forgotten until commit())
+  int victim() { const int i = next; base[i] = nullptr; return i; }
+  void commit(int i, const void *b) { base[i] = b; next = (i + 1) % kCdgMapSlots; }
+};
+
 struct cdgrab_ctx {
   uint32_t magic;
   int m, n;
@@ -57,12 +77,12 @@ struct cdgrab_ctx {
   int fma_tma_boxrows;     // rows per bulk-tensor copy
   int fma_tma_contig;      // 1: each CTA owns a contiguous range of tiles
   int pdl;                 // 1: dependent launches start early and wait on the device for their predecessor
+  int cluster_off;         // 1: the one-launch step never spreads over a thread-block cluster (CDGRAB_CLUSTER=0)
   int fma_tma_fused;       // 1: the last CTA of pass 1 also combines and decides (no scan launch)
   unsigned *ticket;        // [1] arrival counter of that hand-over, zero between launches
   size_t fma_tma_smem;
   CUtensorMap tm_fr;       // 2-D map over r (one row)
-  const void *tm_fg_base;
-  CUtensorMap tm_fg;       // 2-D map over the gradient rows
+  CdgMapCache<1> tm_fg;    // 2-D maps over the gradient rows of the last few buffers
 
   // optional per-kernel timing (cdgrab_profile_*): event pairs recorded around launches
   int prof_on;
@@ -83,10 +103,9 @@ struct cdgrab_ctx {
   size_t umma_smem;
   CUtensorMap tm_r;        // 3-D tensor map over r_split
   CUtensorMap tm_r2;       // 2-D map over r_split (ragged last block)
-  const void *tm_g_base;   // gradient buffer the cached maps were encoded for
-  CUtensorMap tm_g;        // 3-D map over the gradient rows
-  CUtensorMap tm_g2;       // 2-D map over the gradient rows (ragged last block)
-  CUtensorMap tm_g4;       // 4-D map over the full 8-row groups of the gradient rows
+  // maps over the gradient rows of the last few buffers: [0] 3-D, [1] 2-D (ragged last block),
+  // [2] 4-D over the full 8-row groups
+  CdgMapCache<3> tm_g;
   int umma_g4;             // row groups one 4-D copy brings in (0: per-group copies only)
   int umma_paired;         // 2m <= 64: one MMA covers two 64-column blocks
   int umma_fused;          // the combine launch also takes the decisions (last block)
@@ -102,6 +121,22 @@ __device__ __forceinline__ float cdg_ld<float>(const float *p) { return *p; }
 template <>
 __device__ __forceinline__ float cdg_ld<__nv_bfloat16>(const __nv_bfloat16 *p) {
   return __bfloat162float(*p);
+}
+
+// The limit is per kernel, not per handle: handles of different shapes share a kernel, so the
+// TMA-fed kernels are always opened up to the architecture's maximum (227 KB per CTA).
+constexpr int kCdgMaxDynSmem = 227 * 1024;
+
+// cudaFuncSetAttribute acts on the device that is current at the call, so a raised dynamic
+// shared-memory limit has to be set once per (kernel, device): one flag array per call site.
+struct CdgPerDevice { unsigned char done[64]; };
+template <typename K>
+inline cudaError_t cdg_raise_smem_limit(CdgPerDevice &flags, int device, K *kernel, size_t bytes) {
+  const bool tracked = device >= 0 && device < 64;
+  if (tracked && flags.done[device]) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && tracked) flags.done[device] = 1;
+  return e;
 }
 
 // Event pair around one launch when profiling is on; a full pool stops recording.

@@ -203,13 +203,10 @@ static cudaError_t launch_gram_block_t(cdgrab_ctx *h, const void *grads, cudaStr
   const int ctas = h->gram_chunks;
   long long cols = (h->d + ctas - 1) / ctas;
   cols = (cols + kKT - 1) / kKT * kKT;            // whole stages per CTA
-  static bool attr_set = false;
-  if (!attr_set) {
-    const cudaError_t e = cudaFuncSetAttribute(gram_block_kernel<T, BR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)sizeof(BlockSmem<BR>));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static CdgPerDevice attr_set;
+  if (const cudaError_t e = cdg_raise_smem_limit(attr_set, h->device, gram_block_kernel<T, BR>, sizeof(BlockSmem<BR>));
+      e != cudaSuccess)
+    return e;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     cdg_launch_dep(h, gram_block_kernel<T, BR>, dim3(ctas, npairs), dim3(256), sizeof(BlockSmem<BR>), st,

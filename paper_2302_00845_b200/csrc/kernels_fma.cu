@@ -496,13 +496,10 @@ static cudaError_t launch_fused_logreg_tt(cdgrab_ctx *h, const float *X, const f
   constexpr int WARPS = THREADS / 32;
   const size_t smem = (WARPS * Tri<M>::NPAD + 2 * Tri<M>::NPAD + 2 * M + 4 * M + M * M) * sizeof(double) +
                       (M + 4 * M) * sizeof(float) + 2 * M * sizeof(size_t) + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(fused_logreg_step_kernel<M, THREADS>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static CdgPerDevice attr_set;
+  if (const cudaError_t e = cdg_raise_smem_limit(attr_set, h->device, fused_logreg_step_kernel<M, THREADS>, smem);
+      e != cudaSuccess)
+    return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(csize); cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute at[2];
@@ -542,9 +539,7 @@ bool cdg_fused_supported(int m, long long d, int dtype) {
 // CTAs per cluster for the spread-out step: one per THREADS column groups, 4 or 8, else a single CTA
 template <int M>
 static int fused_cluster_size(const cdgrab_ctx *h) {
-  if (const char *e = getenv("CDGRAB_CLUSTER")) {
-    if (atoi(e) == 0) return 1;
-  }
+  if (h->cluster_off) return 1;
   const long long groups = (h->d / 4 + ClusterCfg<M>::THREADS - 1) / ClusterCfg<M>::THREADS;
   int c = 1;
   while (c < 8 && 2 * c <= groups) c *= 2;
@@ -585,13 +580,9 @@ static cudaError_t launch_fused_t(cdgrab_ctx *h, const void *grads, int count, c
   if (csize > 1) return launch_fused_cluster_t<T, M>(h, grads, count, csize, st);
   const size_t smem = ((FusedCfg<M>::THREADS / 32) * Tri<M>::NPAD + Tri<M>::NPAD + 4 * M + M * M) * sizeof(double) +
                       M * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(fused_step_kernel<T, M>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static CdgPerDevice attr_set;
+  if (const cudaError_t e = cdg_raise_smem_limit(attr_set, h->device, fused_step_kernel<T, M>, smem); e != cudaSuccess)
+    return e;
   {
     CdgProfScope ps(h, CDGRAB_K_FUSED, st);
     cdg_launch_dep(h, fused_step_kernel<T, M>, dim3(1), dim3(FusedCfg<M>::THREADS), smem, st, (const T *)grads, h->r,
@@ -943,14 +934,13 @@ static bool ft_encode(CUtensorMap *map, const void *base, long long d, int rows,
   cuuint32_t estr[2] = {1, 1};
   return fn(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
             const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_NONE,
-            getenv("CDGRAB_FT_L2P") ? (CUtensorMapL2promotion)atoi(getenv("CDGRAB_FT_L2P")) : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <typename T, int M>
 static cudaError_t ft_set_smem(size_t smem) {
-  return cudaFuncSetAttribute(gram_fma_tma_kernel<T, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  return cudaFuncSetAttribute(gram_fma_tma_kernel<T, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCdgMaxDynSmem);
 }
 
 int cdg_fma_tma_setup(cdgrab_ctx *h) {
@@ -989,18 +979,17 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
                : M == 8 ? ft_set_smem<__nv_bfloat16, 8>(h->fma_tma_smem)
                         : ft_set_smem<__nv_bfloat16, 16>(h->fma_tma_smem);
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
-  h->tm_fg_base = nullptr;
   h->fma_tma = 1;
   return CDGRAB_OK;
 }
 
 template <typename T, int M>
-static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, cudaStream_t st) {
+static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g, cudaStream_t st) {
   const FtTail tail = cdg_tail_of(h, h->fma_tma_fused);
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     cdg_launch_dep(h, gram_fma_tma_kernel<T, M>, dim3(h->gram_chunks), dim3(kFtThreads), h->fma_tma_smem, st,
-                   h->tm_fg, h->tm_fr, h->m, h->d, h->fma_tma_stages, h->fma_tma_boxrows, h->fma_tma_contig,
+                   tm_g, h->tm_fr, h->m, h->d, h->fma_tma_stages, h->fma_tma_boxrows, h->fma_tma_contig,
                    h->partials, h->status, tail);
   }
   if (!h->fma_tma_fused) {
@@ -1011,18 +1000,21 @@ static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, cudaStream_t st) {
 }
 
 cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
-  if (grads != h->tm_fg_base) {
-    if (!ft_encode(&h->tm_fg, grads, h->d, 2 * h->m, h->fma_tma_boxrows, h->dtype == CDGRAB_F32 ? 4 : 2))
+  int slot = h->tm_fg.find(grads);
+  if (slot < 0) {
+    slot = h->tm_fg.victim();
+    if (!ft_encode(&h->tm_fg.maps[slot][0], grads, h->d, 2 * h->m, h->fma_tma_boxrows, h->dtype == CDGRAB_F32 ? 4 : 2))
       return cudaErrorInvalidValue;
-    h->tm_fg_base = grads;
+    h->tm_fg.commit(slot, grads);
   }
+  const CUtensorMap &tm = h->tm_fg.maps[slot][0];
   const int M = pick_M(h->m);
   if (h->dtype == CDGRAB_F32) {
-    if (M == 4) return launch_gram_fma_tma_t<float, 4>(h, st);
-    if (M == 8) return launch_gram_fma_tma_t<float, 8>(h, st);
-    return launch_gram_fma_tma_t<float, 16>(h, st);
+    if (M == 4) return launch_gram_fma_tma_t<float, 4>(h, tm, st);
+    if (M == 8) return launch_gram_fma_tma_t<float, 8>(h, tm, st);
+    return launch_gram_fma_tma_t<float, 16>(h, tm, st);
   }
-  if (M == 4) return launch_gram_fma_tma_t<__nv_bfloat16, 4>(h, st);
-  if (M == 8) return launch_gram_fma_tma_t<__nv_bfloat16, 8>(h, st);
-  return launch_gram_fma_tma_t<__nv_bfloat16, 16>(h, st);
+  if (M == 4) return launch_gram_fma_tma_t<__nv_bfloat16, 4>(h, tm, st);
+  if (M == 8) return launch_gram_fma_tma_t<__nv_bfloat16, 8>(h, tm, st);
+  return launch_gram_fma_tma_t<__nv_bfloat16, 16>(h, tm, st);
 }

@@ -398,13 +398,9 @@ cudaError_t cdg_launch_scan(cdgrab_ctx *h, cudaStream_t st) {
   const size_t with_g = scan_smem_bytes(m, true);
   const int use_smem = with_g <= 160 * 1024;
   const size_t smem = use_smem ? with_g : small;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         160 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static CdgPerDevice attr_set;
+  if (const cudaError_t e = cdg_raise_smem_limit(attr_set, h->device, scan_kernel, 160 * 1024); e != cudaSuccess)
+    return e;
   {
     CdgProfScope ps(h, CDGRAB_K_SCAN, st);
     cdg_launch_dep(h, scan_kernel, dim3(1), dim3(256), smem, st, h->gram, m, h->n, h->k, h->perm_cur, h->perm_next,

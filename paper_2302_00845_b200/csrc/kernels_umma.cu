@@ -618,12 +618,18 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   if (!encode_map_3d(&h->tm_r, h->r_split, nblk_full, 3, h->d_pad, h->umma_paired ? subs / 2 : subs))
     return CDGRAB_ERR_CUDA;
   if (!encode_map_2d(&h->tm_r2, h->r_split, h->d, 3, h->d_pad)) return CDGRAB_ERR_CUDA;
-  if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->umma_smem) !=
+  if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCdgMaxDynSmem) !=
       cudaSuccess) {
     cudaGetLastError();
     return CDGRAB_ERR_CUDA;
   }
-  h->tm_g_base = nullptr;
+  // one copy for all full row groups of a (half) stage; CDGRAB_UMMA_G4=0: per-group copies only
+  h->umma_g4 = h->umma_rows / 8;
+  if (const char *e = getenv("CDGRAB_UMMA_G4")) {
+    if (atoi(e) == 0) h->umma_g4 = 0;
+  }
+  const long long row_pitch = h->umma_split3 ? h->d_pad : h->d;
+  if (row_pitch * 16 >= (1ll << 40)) h->umma_g4 = 0;             // the group stride must fit the map
   h->umma_fused = h->shard ? 0 : 1;      // a shard's decisions wait for the sum over shards
   if (const char *e = getenv("CDGRAB_UMMA_FUSE_TAIL")) {
     if (atoi(e) == 0) h->umma_fused = 0;
@@ -654,21 +660,19 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
     cdg_launch_dep(h, split_diff_kernel, dim3((unsigned)chunks, h->m), dim3(256), 0, st, (const float *)grads, h->m,
                    h->d, h->d_pad, h->umma_csplit);
   }
-  if (src != h->tm_g_base) {
+  int slot = h->tm_g.find(src);
+  if (slot < 0) {
+    slot = h->tm_g.victim();
+    CUtensorMap *mp = h->tm_g.maps[slot];
     const int box_blocks = h->umma_paired ? h->umma_subs_per_stage / 2 : h->umma_subs_per_stage;
-    if (!encode_map_3d(&h->tm_g, src, nblk_full, rows, pitch, box_blocks) ||
-        !encode_map_2d(&h->tm_g2, src, h->d, rows, pitch))
+    if (!encode_map_3d(&mp[0], src, nblk_full, rows, pitch, box_blocks) || !encode_map_2d(&mp[1], src, h->d, rows, pitch))
       return cudaErrorInvalidValue;
-    // one copy for all full row groups of a (half) stage; CDGRAB_UMMA_G4=0: per-group copies only
-    h->umma_g4 = rows / 8;
-    if (const char *e = getenv("CDGRAB_UMMA_G4")) {
-      if (atoi(e) == 0) h->umma_g4 = 0;
-    }
-    if (pitch * 16 >= (1ll << 40)) h->umma_g4 = 0;               // the group stride must fit the map
-    if (h->umma_g4 > 0 && !encode_map_4d(&h->tm_g4, src, nblk_full, h->umma_g4, pitch, box_blocks)) h->umma_g4 = 0;
-    if (h->umma_g4 == 0) h->tm_g4 = h->tm_g;
-    h->tm_g_base = src;
+    // a driver that refuses the 4-D map sends this handle to per-group copies for good
+    if (h->umma_g4 > 0 && !encode_map_4d(&mp[2], src, nblk_full, h->umma_g4, pitch, box_blocks)) h->umma_g4 = 0;
+    if (h->umma_g4 == 0) mp[2] = mp[0];
+    h->tm_g.commit(slot, src);
   }
+  const CUtensorMap *mp = h->tm_g.maps[slot];
   UmmaParams p;
   p.box_rows = h->umma_box_rows;
   p.ncols = h->umma_ncols;
@@ -682,8 +686,8 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
   p.paired = h->umma_paired;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
-    cdg_launch_dep(h, gram_umma_kernel, dim3(h->umma_ctas), dim3(kThreads), h->umma_smem, st, h->tm_g, h->tm_r,
-                   h->tm_g2, h->tm_r2, h->tm_g4, p, h->umma_partials, h->status);
+    cdg_launch_dep(h, gram_umma_kernel, dim3(h->umma_ctas), dim3(kThreads), h->umma_smem, st, mp[0], h->tm_r,
+                   mp[1], h->tm_r2, mp[2], p, h->umma_partials, h->status);
   }
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);

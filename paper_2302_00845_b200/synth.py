@@ -118,18 +118,19 @@ class GradientStream:
         else:
             raise ValueError(wl.kind)
 
-    def _row(self, gen) -> torch.Tensor:
+    def _rows(self, gen, count: int) -> torch.Tensor:
+        """`count` gradient rows [count][d] in fp32 from one pass over the generator."""
         wl, d, dev = self.wl, self.wl.d, self.device
         if wl.kind == "mean_offset":
-            return self.mu + torch.randn(d, generator=gen, device=dev)
+            return self.mu + torch.randn(count, d, generator=gen, device=dev)
         if wl.kind == "heavy_tail":
-            return self.mu + torch.randn(d, generator=gen, device=dev) * (math.sqrt(0.5) * self.scale)
+            return self.mu + torch.randn(count, d, generator=gen, device=dev) * (math.sqrt(0.5) * self.scale)
         if wl.kind == "layer_scale":
-            return torch.randn(d, generator=gen, device=dev) * (math.sqrt(1e-3) * self.scale)
+            return torch.randn(count, d, generator=gen, device=dev) * (math.sqrt(1e-3) * self.scale)
         # low_rank: per-coordinate variance 1e-4, half in the shared rank-16 subspace
-        a = torch.randn(self.rank, generator=gen, device=dev)
+        a = torch.randn(count, self.rank, generator=gen, device=dev)
         low = (a.to(torch.bfloat16) @ self.U).float() / math.sqrt(2.0 * self.rank)
-        eps = torch.randn(d, generator=gen, device=dev) / math.sqrt(2.0)
+        eps = torch.randn(count, d, generator=gen, device=dev) / math.sqrt(2.0)
         return (low + eps) * 1e-2
 
     def step(self, k: int, epoch: int = 0, out: torch.Tensor | None = None) -> torch.Tensor:
@@ -137,9 +138,13 @@ class GradientStream:
         if out is None:
             out = torch.empty(2, wl.m, wl.d, dtype=wl.torch_dtype, device=self.device)
         gen = _gen(self.device, wl.seed, 0xB22, epoch, k)
-        for slab in range(2):
-            for i in range(wl.m):
-                out[slab, i] = self._row(gen).to(wl.torch_dtype)
+        # as many rows per draw as keep the fp32 temporaries near 1 GiB: small shapes come out of a
+        # single call, the largest ones two rows at a time
+        flat = out.view(2 * wl.m, wl.d)
+        per = max(1, min(2 * wl.m, (1 << 28) // wl.d))
+        for lo in range(0, 2 * wl.m, per):
+            hi = min(2 * wl.m, lo + per)
+            flat[lo:hi] = self._rows(gen, hi - lo).to(wl.torch_dtype)
         return out
 
 

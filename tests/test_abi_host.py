@@ -79,3 +79,21 @@ def test_product_does_not_import_the_oracle():
                 src = open(os.path.join(dirpath, f)).read()
                 assert not re.search(r"^\s*(import|from)\s+oracle\b", src, flags=re.M), f
                 assert "liboracle" not in src and "pairbalance_oracle" not in src, f
+
+
+def test_environment_is_read_at_create_time_only():
+    """Launch paths run every few microseconds: knobs are read when a handle is created (create_impl
+    and the *_setup / *_supported routines it calls), never per step."""
+    csrc = os.path.join(ROOT, "paper_2302_00845_b200", "csrc")
+    allowed = ("create_impl", "forced_path", "cdg_fma_tma_setup", "cdg_umma_setup", "cdg_umma_supported")
+    for f in sorted(os.listdir(csrc)):
+        src = open(os.path.join(csrc, f)).read()
+        for mt in re.finditer(r"getenv\(", src):
+            head = src[:mt.start()]
+            # name of the innermost function definition that starts at column 0 before the call
+            defs = re.findall(r"^(?:static\s+)?(?:inline\s+)?[A-Za-z_][\w \*:<>]*?\b(\w+)\([^;{]*\)\s*\{", head, flags=re.M)
+            assert defs and defs[-1] in allowed, (f, defs[-1] if defs else None)
+
+
+def test_wrong_device_has_its_own_code(lib):
+    assert "device" in lib.cdgrab_strerror(binding.ERR_DEVICE).decode()

@@ -107,7 +107,13 @@ def _shard_worker(rank, world, port, out):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     m = 3
     fake = _FakeShard(rank)
-    sh = binding.ShardedCdGrab(m, 4, 16, "f32", handle=fake, device="cpu")
+
+    class OnFake(binding.ShardedCdGrab):          # the wrapper's exchange, driven without a GPU
+        def __init__(self):
+            self.group = None
+            self._attach(fake, m, "cpu")
+
+    sh = OnFake()
     sh.begin_epoch()
     sh.step(None)
     sh.step(None)

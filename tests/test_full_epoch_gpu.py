@@ -1,6 +1,7 @@
-"""Whole-epoch parity at the full sizes of the large workloads (opt-in: several minutes each).
+"""Whole-epoch parity at the full sizes of the large workloads.
 
-Run with CDGRAB_LONG_TESTS=1.  Every step of one epoch is balanced on the GPU (through the C
+The mid-size epoch (under half a minute) always runs; the two bf16 epochs take several minutes
+each and are opt-in: CDGRAB_LONG_TESTS=1.  Every step of one epoch is balanced on the GPU (through the C
 ABI) and replayed by the CPU oracle on the same bytes, streamed to the host through a pinned
 buffer one worker pair at a time; signs (outside the tie band), the final running sum and the
 next-epoch permutations are compared."""
@@ -15,9 +16,9 @@ from oracle import PairBalanceOracle
 from paper_2302_00845_b200 import binding, synth
 from parity import TAU, R_TOL, rel_l2
 
-pytestmark = [pytest.mark.gpu, pytest.mark.slow,
-              pytest.mark.skipif(os.environ.get("CDGRAB_LONG_TESTS") != "1",
-                                 reason="set CDGRAB_LONG_TESTS=1 to run whole epochs at full size")]
+pytestmark = [pytest.mark.gpu, pytest.mark.slow]
+long_only = pytest.mark.skipif(os.environ.get("CDGRAB_LONG_TESTS") != "1",
+                               reason="set CDGRAB_LONG_TESTS=1 to run the bf16 epochs at full size")
 
 
 def run_epoch(name):
@@ -44,6 +45,7 @@ def run_epoch(name):
                 cpu.balance_one(i, view[0], view[1], replay=int(s[i]), tau=TAU[wl.dtype])
             raw += int((cpu.own_signs()[:, k] == s).sum())
         assert cpu.mismatches == 0
+        assert raw >= 0.999 * (m * n // 2), raw
         err = rel_l2(gpu.r().cpu().numpy().astype(np.float64), cpu.r())
         assert err <= R_TOL[wl.dtype], err
         out = torch.empty(m, n, dtype=torch.int32, device="cuda")
@@ -64,9 +66,11 @@ def test_mid_full_epoch():
     run_epoch("mid")
 
 
+@long_only
 def test_lstm_full_epoch():
     run_epoch("lstm")
 
 
+@long_only
 def test_gpt2_full_epoch():
     run_epoch("gpt2")

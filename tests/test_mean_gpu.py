@@ -48,3 +48,18 @@ def test_mean_argument_errors():
         h.begin_epoch()
         rc = binding.lib().cdgrab_step_mean(h._h, grads(2, 64, "f32", 1).data_ptr(), None, None)
         assert rc == binding.ERR_INVALID
+
+
+def test_misaligned_destination_is_refused_on_the_host():
+    """The averages are written with 16-byte vector stores; a destination off that boundary is an
+    argument error, not a device fault."""
+    m, n, d = 4, 4, 4096
+    with binding.CdGrab(m, n, d, "f32") as h:
+        h.begin_epoch()
+        g = torch.zeros(2, m, d, device="cuda")
+        out = torch.zeros(2 * d + 4, device="cuda")[1:1 + 2 * d]
+        with pytest.raises(binding.CdgrabError) as e:
+            h.step_mean(g, out)
+        assert e.value.code == binding.ERR_INVALID
+        assert h.launch_count == 0
+        h.step_mean(g, torch.zeros(2, d, device="cuda"))

@@ -27,6 +27,7 @@ def grads(m, d, dtype, seed):
     (5, 3_003, "f32", [0, 1_001, 3_003]),                # generic tiles
     (24, 80_000, "f32", [0, 40_000, 80_000]),            # fp32 on the tensor cores (three bf16 terms)
     (48, 10_000, "f32", [0, 6_000, 10_000]),             # blocked FMA Gram
+    (80, 6_000, "bf16", [0, 2_000, 6_000]),              # scan with G staged above the default 48 KB of shared memory
 ])
 def test_sharded_steps_match_oracle(m, d, dtype, cuts):
     n = 6
@@ -86,6 +87,15 @@ def test_shard_state_machine():
             h.step_begin(g, p)                     # finish first
         assert e.value.code == binding.ERR_STATE
         h.step_finish(g, p)
+        # pointers the kernels would touch with vector accesses are refused on the host
+        h.step_begin(g, p)
+        odd = torch.zeros(2 * m * d + 4, device="cuda")[1:1 + 2 * m * d].view(2, m, d)
+        pp = torch.zeros(2 * (m * m + m) + 2, dtype=torch.float32, device="cuda")[1:1 + 2 * (m * m + m)]
+        L = binding.lib()
+        st = torch.cuda.current_stream().cuda_stream
+        assert L.cdgrab_step_finish(h._h, odd.data_ptr(), p.data_ptr(), st) == binding.ERR_INVALID
+        assert L.cdgrab_step_finish(h._h, g.data_ptr(), pp.data_ptr(), st) == binding.ERR_INVALID
+        h.step_finish(g, p)                        # still pending after the refusals
     with binding.CdGrab(m, n, d, "f32") as h:
         h.begin_epoch()
         with pytest.raises(binding.CdgrabError):
