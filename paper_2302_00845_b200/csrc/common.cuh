@@ -126,6 +126,14 @@ __device__ __forceinline__ float cdg_ld<__nv_bfloat16>(const __nv_bfloat16 *p) {
 // The limit is per kernel, not per handle: handles of different shapes share a kernel, so the
 // TMA-fed kernels are always opened up to the architecture's maximum (227 KB per CTA).
 constexpr int kCdgMaxDynSmem = 227 * 1024;
+template <typename K>
+inline cudaError_t cdg_open_smem_limit(K *kernel) {
+  cudaFuncAttributes fa;
+  const cudaError_t e = cudaFuncGetAttributes(&fa, kernel);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kCdgMaxDynSmem - (int)fa.sharedSizeBytes);   // static and dynamic share the 227 KB
+}
 
 // cudaFuncSetAttribute acts on the device that is current at the call, so a raised dynamic
 // shared-memory limit has to be set once per (kernel, device): one flag array per call site.

@@ -940,7 +940,7 @@ static bool ft_encode(CUtensorMap *map, const void *base, long long d, int rows,
 
 template <typename T, int M>
 static cudaError_t ft_set_smem(size_t smem) {
-  return cudaFuncSetAttribute(gram_fma_tma_kernel<T, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCdgMaxDynSmem);
+  return cdg_open_smem_limit(gram_fma_tma_kernel<T, M>);
 }
 
 int cdg_fma_tma_setup(cdgrab_ctx *h) {

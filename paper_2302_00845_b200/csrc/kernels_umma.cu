@@ -618,7 +618,7 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   if (!encode_map_3d(&h->tm_r, h->r_split, nblk_full, 3, h->d_pad, h->umma_paired ? subs / 2 : subs))
     return CDGRAB_ERR_CUDA;
   if (!encode_map_2d(&h->tm_r2, h->r_split, h->d, 3, h->d_pad)) return CDGRAB_ERR_CUDA;
-  if (cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCdgMaxDynSmem) !=
+  if (cdg_open_smem_limit(gram_umma_kernel) !=
       cudaSuccess) {
     cudaGetLastError();
     return CDGRAB_ERR_CUDA;
