@@ -11,7 +11,8 @@ import ctypes as C
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libcdgrab.so")
+# CDGRAB_LIB: file name (inside the package) of a diagnostic build to load instead
+LIB_PATH = os.path.join(HERE, os.path.basename(os.environ.get("CDGRAB_LIB", "libcdgrab.so")))
 
 F32, BF16 = 0, 1
 OK = 0

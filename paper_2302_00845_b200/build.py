@@ -9,6 +9,11 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcdgrab.so")
+# Diagnostic variants, built beside the product library and loaded instead of it when the
+# environment variable CDGRAB_LIB names them:
+#   --stamp  -DCDGRAB_STAMP  kernels record phase time stamps (libcdgrab_stamp.so)
+#   --debug  -DCDGRAB_DEBUG  index checks and guard words around scratch (libcdgrab_debug.so)
+VARIANTS = {"stamp": ("-DCDGRAB_STAMP", "libcdgrab_stamp.so"), "debug": ("-DCDGRAB_DEBUG", "libcdgrab_debug.so")}
 SOURCES = ["api.cu", "kernels_generic.cu", "kernels_fma.cu", "kernels_umma.cu", "noalloc.cu", "herding.cu", "kernels_indep.cu", "kernels_block.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -25,21 +30,23 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "cdgrab.h")]
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, variant: str | None = None) -> str:
     """Compile every translation unit and link the shared library next to the package."""
-    if not force and not needs_build():
-        return LIB
-    objdir = os.path.join(HERE, "_build")
+    define, name = VARIANTS[variant] if variant else (None, os.path.basename(LIB))
+    lib = os.path.join(HERE, name)
+    if not force and not needs_build(lib):
+        return lib
+    objdir = os.path.join(HERE, "_build", variant or "release")
     os.makedirs(objdir, exist_ok=True)
-    flags = list(NVCC_FLAGS)
+    flags = list(NVCC_FLAGS) + ([define] if define else [])
     if verbose:
         flags += ["-Xptxas", "-v"]
     objs, procs = [], []
@@ -59,9 +66,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed")
     # cudart is linked statically (nvcc default); the driver API is reached through
     # cudaGetDriverEntryPoint, so the library has no link-time CUDA dependency
-    subprocess.check_call([_nvcc(), "-shared", "-o", LIB, *objs])
-    return LIB
+    subprocess.check_call([_nvcc(), "-shared", "-o", lib, *objs])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    which = next((v for v in VARIANTS if "--" + v in sys.argv), None)
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, variant=which))

@@ -35,6 +35,8 @@ void free_all(cdgrab_ctx *h) {
   cudaFree(h->margins); cudaFree(h->rnorm2); cudaFree(h->status); cudaFree(h->gram);
   cudaFree(h->partials);
   cudaFree(h->ticket);
+  cudaFree(h->ft_ctr);
+  cudaFree(h->ft_group_partials);
   cudaFree(h->oob);
   if (h->prof_ev) {
     for (int i = 0; i < 2 * h->prof_cap; ++i) if (h->prof_ev[i]) cudaEventDestroy(h->prof_ev[i]);
@@ -340,7 +342,8 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
     e = launch_pass1(h, grads_dev, st);
     const bool decided = (h->path == CDGRAB_PATH_UMMA) ? h->umma_fused : (h->fma_tma && h->fma_tma_fused);
     if (e == cudaSuccess && !decided) e = cdg_launch_scan(h, st);
-    if (e == cudaSuccess) e = cdg_launch_update(h, grads_dev, st);
+    const bool updated = h->fma_tma && h->ft_whole_launched;     // pass 2 ran inside the pass-1 launch
+    if (e == cudaSuccess && !updated) e = cdg_launch_update(h, grads_dev, st);
   }
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   h->k++;
@@ -526,6 +529,12 @@ int cdgrab_clear_status(cdgrab_t *h) {
     cudaGetLastError();
     return CDGRAB_ERR_CUDA;
   }
+  // a launch that gave up may have left the arrival counters of the reduction tree short
+  if (h->ft_ctr) {
+    if (cudaMemset(h->ft_ctr, 0, sizeof(unsigned long long) * 65) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+    h->ft_gen = 0;
+  }
+  if (h->ticket && cudaMemset(h->ticket, 0, sizeof(unsigned)) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   return CDGRAB_OK;
 }
 

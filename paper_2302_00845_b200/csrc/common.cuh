@@ -79,7 +79,15 @@ struct cdgrab_ctx {
   int pdl;                 // 1: dependent launches start early and wait on the device for their predecessor
   int cluster_off;         // 1: the one-launch step never spreads over a thread-block cluster (CDGRAB_CLUSTER=0)
   int fma_tma_fused;       // 1: the last CTA of pass 1 also combines and decides (no scan launch)
-  unsigned *ticket;        // [1] arrival counter of that hand-over, zero between launches
+  unsigned *ticket;        // [1] arrival counter of the tensor-core path's hand-over, zero between launches
+  int fma_tma_whole;       // 1: that launch also runs pass 2 (cooperative launch, no update launch)
+  int ft_whole_launched;   // the last pass-1 launch was a whole step
+  int ft_coop;             // 1: the whole-step launch is a cooperative launch
+  int ft_coop_no_pdl;      // the driver refused cooperative + programmatic serialization together
+  int ft_gsize;            // CTAs per group of the reduction tree
+  unsigned long long ft_gen;          // launches of the tree so far (its counters only grow)
+  unsigned long long *ft_ctr;         // [groups + 1] arrival counters of the tree
+  double *ft_group_partials;          // [groups][152]
   size_t fma_tma_smem;
   CUtensorMap tm_fr;       // 2-D map over r (one row)
   CdgMapCache<1> tm_fg;    // 2-D maps over the gradient rows of the last few buffers

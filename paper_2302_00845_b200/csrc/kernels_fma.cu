@@ -651,6 +651,7 @@ cudaError_t cdg_launch_gram_fma(cdgrab_ctx *h, const void *grads, cudaStream_t s
 
 constexpr int kFtCols = 256;       // columns per tile
 constexpr int kFtMaxStages = 8;
+constexpr int kFtMaxGroups = 64;   // groups of the reduction tree over the CTAs
 constexpr int kFtThreads = 2 * kFtCols + 32;   // two compute groups + the producer warp
 
 template <typename T>
@@ -742,19 +743,100 @@ struct SplitMap {
 template <int M>
 __constant__ SplitMap<M> kSplitMap = SplitMap<M>();
 
-// When enabled, the last CTA to finish also runs the scalar part of the step.
+// When enabled, the scalar part of the step runs inside this kernel (no scan launch).
 using FtTail = CdgTail;
+
+// Built with -DCDGRAB_STAMP (python -m paper_2302_00845_b200.build --stamp) every CTA of the
+// TMA-fed kernel records %globaltimer at the phase boundaries of its last launch;
+// cdgrab_debug_ft_stamps copies the table out ([CTA][slot], nanoseconds).  Off by default.
+#ifdef CDGRAB_STAMP
+constexpr int kFtStampSlots = 16;   // slot 10: kernel entry; slot 11: slot 9 of the launch before
+__device__ unsigned long long ft_stamps[1024][kFtStampSlots];
+__device__ __forceinline__ void ft_stamp(int slot) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  if (blockIdx.x < 1024) ft_stamps[blockIdx.x][slot] = t;
+}
+extern "C" int cdgrab_debug_ft_stamps(unsigned long long *host_out, int ctas) {
+  if (ctas < 1 || ctas > 1024) return CDGRAB_ERR_INVALID;
+  cudaDeviceSynchronize();
+  return cudaMemcpyFromSymbol(host_out, ft_stamps, sizeof(unsigned long long) * kFtStampSlots * ctas) == cudaSuccess
+             ? CDGRAB_OK : CDGRAB_ERR_CUDA;
+}
+#define FT_STAMP(cond, slot) do { if (cond) ft_stamp(slot); } while (0)
+#else
+#define FT_STAMP(cond, slot) do { } while (0)
+#endif
+
+// Fixed-order reduction tree over the CTAs, and what the whole-step mode needs.  The block
+// partials are summed in two levels: CTAs form groups of `gsize`; the CTA that arrives last in
+// its group (a counter per group) adds the group's partials in CTA order and publishes the group
+// partial; a top counter counts finished groups.  The counters only ever grow: launch number
+// `gen` (1, 2, ...) of a handle expects gen * (arrivals per launch), so nothing has to be reset
+// and no CTA waits to take a ticket.
+//   whole = 0: the CTA that finishes the last group combines the group partials, decides, leaves.
+//   whole = 1: every CTA waits (bounded) until all groups are finished, combines the group
+//              partials itself (same order everywhere, same bits), takes the same decisions, and
+//              runs pass 2 over its own tiles in reverse: first the tiles still in its
+//              shared-memory ring, then the ones most recently read (the likeliest to sit in L2).
+//              CTAs wait on one another, so this mode is launched cooperatively.
+struct FtTree {
+  int whole;
+  int gsize;                           // CTAs per group
+  unsigned long long gen;              // launch number of this handle, from 1
+  unsigned long long *group_ctr;       // [groups] arrivals, monotonic
+  unsigned long long *top_ctr;         // [1] finished groups, monotonic
+  double *group_partials;              // [groups][NACC]
+  float *r;                            // whole-step mode: the running sum, updated in place
+};
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long *p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
+template <typename T> struct FtAcc { typedef float type; };      // bf16 rows: fp32 adds, i ascending
+template <> struct FtAcc<float> { typedef double type; };        // fp32 rows: one rounding of r per step
+
+// pass 2 on one tile held in shared memory: r <- r + sum_i s_i (z1_i - z2_i), i ascending.
+// All 2m values of the column are fetched before the first add, so the only serial part is the
+// chain of m additions.
+template <typename T, int M>
+__device__ __forceinline__ void ft_update_tile(const T *gt, const float *rt, const float *ssh, int m, int col,
+                                               long long gcol, long long d, float *__restrict__ r) {
+  if (gcol >= d) return;
+  float c[M];
+#pragma unroll
+  for (int i = 0; i < M; ++i) {
+    c[i] = 0.f;
+    if (i < m)
+      c[i] = ssh[i] * (ft_widen<T>(gt[(size_t)i * kFtCols + col]) - ft_widen<T>(gt[(size_t)(m + i) * kFtCols + col]));
+  }
+  typename FtAcc<T>::type acc = (typename FtAcc<T>::type)rt[col];
+#pragma unroll
+  for (int i = 0; i < M; ++i)
+    if (i < m) acc += (typename FtAcc<T>::type)c[i];
+  r[gcol] = (float)acc;
+}
 
 template <typename T, int M>
 __global__ void __launch_bounds__(kFtThreads, 1)
 gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
                     int m, long long d, int stages, int box_rows, int contiguous,
-                    double *__restrict__ partials, int *__restrict__ status, const FtTail tail) {
+                    double *__restrict__ partials, int *__restrict__ status, const FtTail tail, const FtTree tree) {
   extern __shared__ uint8_t ft_smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kFtMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kFtMaxStages];
-  __shared__ double red[16 * Split<M>::NLPAD];      // [warp][local entry]
+  __shared__ double red[16 * Split<M>::NLPAD];      // [warp][local entry]; afterwards the scan's arrays
+  __shared__ float ssh[M];                          // signs of the step as +-1.0f (whole-step mode)
+  __shared__ int flag_sh[3];                        // last of its group / finished the last group / wait ended well
+  __shared__ int bad_sh;                            // a wait of this CTA has run out
 
+#ifdef CDGRAB_STAMP
+  if (threadIdx.x == 0 && blockIdx.x < 1024) ft_stamps[blockIdx.x][11] = ft_stamps[blockIdx.x][9];
+  FT_STAMP(threadIdx.x == 0, 10);
+#endif
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = warp >> 3;                       // 0, 1: compute groups; 2: producer
   const uint32_t base = (smem_u32(ft_smem_raw) + 127u) & ~127u;
@@ -769,6 +851,8 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   const long long t_hi = contiguous ? ntiles * (blockIdx.x + 1) / gridDim.x : ntiles;
   const long long t_step = contiguous ? 1 : gridDim.x;
   const int n_iter = (int)((t_hi - t_lo + t_step - 1) / t_step);
+  // whole-step mode: the last `keep` tiles of pass 1 stay in the ring for pass 2
+  const int keep = tree.whole ? min(stages, n_iter) : 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -776,9 +860,14 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       mbar_init(smem_u32(&bar_empty[s]), 16);  // one arrival per compute warp
     }
     mbar_init_fence();
+    bad_sh = 0;
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_g) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_r) : "memory");
   }
   __syncthreads();
+  FT_STAMP(threadIdx.x == 0, 0);
   cdg_grid_dep_wait();      // r is written by the launch before this one
+  FT_STAMP(threadIdx.x == 0, 1);
   const long long deadline = clock64() + kCdgWaitCycles;
 
   float acc[Split<M>::NLPAD];
@@ -788,6 +877,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   // what the scalar tail will need, fetched now by idle lanes of the producer warp
   int32_t pf_first = 0, pf_second = 0;
   double pf_rn2 = 0.0;
+  bool prod_ok = true;                               // producer lane: no wait has run out so far
   if (group == 2) {
     if (tail.enabled && lane >= 1 && lane <= m) {
       pf_first = tail.perm_cur[(size_t)(lane - 1) * tail.n + 2 * tail.k];
@@ -814,9 +904,11 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       }
       if (!ok) {
         atomicOr(status, CDG_ST_TIMEOUT);
+        bad_sh = 1;
         for (int it = max(0, issued - stages); it < issued; ++it)
           mbar_wait(smem_u32(&bar_full[it % stages]), (it / stages) & 1, clock64() + kCdgWaitCycles);
       }
+      prod_ok = ok;
     }
   } else {
     const int col = threadIdx.x & (kFtCols - 1);
@@ -826,15 +918,18 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     for (int it = 0; it < n_iter && ok; ++it) {
       ok = mbar_wait(smem_u32(&bar_full[s]), parity, deadline);
       if (!ok) break;
+      FT_STAMP(threadIdx.x == 0 && it == 0, 2);
       const T *gt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes);
       const float *rt = reinterpret_cast<const float *>(base_ptr + (size_t)s * stage_bytes + g_bytes);
       if (group == 0) ft_consume<T, M, 0>(gt, rt, m, col, acc);
       else ft_consume<T, M, 1>(gt, rt, m, col, acc);
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));   // this warp is done with the stage
+      // this warp is done with the stage (a tile kept for pass 2 is released there instead)
+      if (lane == 0 && it < n_iter - keep) mbar_arrive(smem_u32(&bar_empty[s]));
       if (++s == stages) { s = 0; parity ^= 1u; }
     }
-    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+    if (!ok && lane == 0) { atomicOr(status, CDG_ST_TIMEOUT); bad_sh = 1; }
+    FT_STAMP(threadIdx.x == 0, 3);
     // warp totals of the local entries, as doubles
     warp_reduce_vec<Split<M>::NLPAD>(acc, lane);
 #pragma unroll
@@ -853,54 +948,84 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       partials[(size_t)blockIdx.x * Tri<M>::NACC + e] = v;
     }
   }
+  // a compute warp gave up on a tile: let the copies still under way land before the CTA can leave
+  if (bad_sh && group == 2 && lane == 0 && prod_ok) {
+    for (int it = max(0, n_iter - stages); it < n_iter; ++it)
+      mbar_wait(smem_u32(&bar_full[it % stages]), (it / stages) & 1, clock64() + kCdgWaitCycles);
+  }
   if (!tail.enabled) return;
 
-  // ---- the CTA that takes the last ticket finishes the step: combine, decide, write ----
-  // (no waiting: a CTA either is last and sees every partial, or leaves)
-  __shared__ int is_last;
+  // ---- two-level tree over the CTAs (no CTA waits to take a ticket) ----
+  constexpr int NACC = Tri<M>::NACC;
+  const int grp = blockIdx.x / tree.gsize;
+  const int ngroups = ((int)gridDim.x + tree.gsize - 1) / tree.gsize;
+  const int gcount = min(tree.gsize, (int)gridDim.x - grp * tree.gsize);
   __threadfence();
-  __syncthreads();
+  __syncthreads();                                   // red is free from here on
   if (threadIdx.x == 0) {
-    const unsigned t = atomicAdd(tail.ticket, 1u);
-    is_last = (t == gridDim.x - 1);
+    const unsigned long long old = atomicAdd(tree.group_ctr + grp, 1ull);
+    flag_sh[0] = (old + 1 == tree.gen * (unsigned long long)gcount);
+    flag_sh[1] = 0;
+    FT_STAMP(true, 4);
   }
   __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  // the stage ring is idle now; reuse it (all copies were consumed before the partials went out)
-  double *sh = reinterpret_cast<double *>(base_ptr);
-  const ScanSmem S = scan_smem(sh, m);
-  double *slices = S.g + (size_t)m * m;                       // [3][NPAD] block-list slices
-  double *rn2_sh = slices + 3 * Tri<M>::NPAD;
-  constexpr int NP = Tri<M>::NPAD;
-  if (threadIdx.x < 3 * NP) {
-    // slice p adds blocks p, p+3, ... in that order; the slices are then added in order
-    const int e = threadIdx.x % NP, p = threadIdx.x / NP;
-    double v = 0.0;
-    if (e < Tri<M>::NACC) {
+  if (flag_sh[0]) {
+    // last of its group: the group's block partials in CTA order (all loads in flight first)
+    __threadfence();
+    if (threadIdx.x < NACC) {
+      const double *src = partials + (size_t)grp * tree.gsize * NACC + threadIdx.x;
+      double v = 0.0;
 #pragma unroll 1
-      for (int b0 = p; b0 < (int)gridDim.x; b0 += 3 * 26) {
-        double x[26];            // all loads of a batch in flight before the first add
+      for (int b0 = 0; b0 < gcount; b0 += 12) {
+        double x[12];
 #pragma unroll
-        for (int q = 0; q < 26; ++q) {
-          const int b = b0 + 3 * q;
-          x[q] = (b < (int)gridDim.x) ? __ldcg(partials + (size_t)b * Tri<M>::NACC + e) : 0.0;
-        }
+        for (int q = 0; q < 12; ++q) x[q] = (b0 + q < gcount) ? __ldcg(src + (size_t)(b0 + q) * NACC) : 0.0;
 #pragma unroll
-        for (int q = 0; q < 26; ++q)
-          if (b0 + 3 * q < (int)gridDim.x) v += x[q];
+        for (int q = 0; q < 12; ++q)
+          if (b0 + q < gcount) v += x[q];
       }
+      tree.group_partials[(size_t)grp * NACC + threadIdx.x] = v;
     }
-    slices[p * NP + e] = v;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const unsigned long long old = atomicAdd(tree.top_ctr, 1ull);
+      flag_sh[1] = (old + 1 == tree.gen * (unsigned long long)ngroups);
+    }
+    __syncthreads();
   }
-  if (group == 2) {
-    if (lane >= 1 && lane <= m) { S.p[2 * (lane - 1)] = pf_first; S.p[2 * (lane - 1) + 1] = pf_second; }
-    if (lane == 17) *rn2_sh = pf_rn2;
+  if (!tree.whole) {
+    if (!flag_sh[1]) return;                         // only the CTA that finished the last group goes on
+  } else {
+    // every CTA needs the totals: bounded wait until all groups are finished
+    if (threadIdx.x == 0) {
+      const unsigned long long want = tree.gen * (unsigned long long)ngroups;
+      bool ok = true;
+      while (ld_acquire_u64(tree.top_ctr) < want) {
+        if (clock64() > deadline) { ok = false; break; }
+      }
+      if (!ok) atomicOr(status, CDG_ST_TIMEOUT);
+      flag_sh[2] = ok;
+      FT_STAMP(true, 5);
+    }
+    __syncthreads();
+    if (!flag_sh[2]) return;                         // nothing of this CTA is in flight at this point
   }
-  __syncthreads();
-  if (threadIdx.x < Tri<M>::NACC) {
+  __threadfence();
+  FT_STAMP(threadIdx.x == 0, 12);
+  const ScanSmem S = scan_smem(red, m);
+  double *rn2_sh = S.g + (size_t)m * m;
+  if (threadIdx.x < NACC) {
     const int e = threadIdx.x;
-    const double v = (slices[e] + slices[NP + e]) + slices[2 * NP + e];
+    double v = 0.0;
+    for (int b0 = 0; b0 < ngroups; b0 += 16) {       // group partials in group order
+      double x[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) x[q] = (b0 + q < ngroups) ? __ldcg(tree.group_partials + (size_t)(b0 + q) * NACC + e) : 0.0;
+#pragma unroll
+      for (int q = 0; q < 16; ++q)
+        if (b0 + q < ngroups) v += x[q];
+    }
     if (e < Tri<M>::NPAIR) {
       int a = 0, rem = e;
       while (rem >= M - a) { rem -= M - a; ++a; }
@@ -911,10 +1036,72 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       if (a < m) S.t[a] = v;
     }
   }
-  if (threadIdx.x == 0) *tail.ticket = 0u;                    // ready for the next launch
+  if (group == 2) {
+    if (lane >= 1 && lane <= m) { S.p[2 * (lane - 1)] = pf_first; S.p[2 * (lane - 1) + 1] = pf_second; }
+    if (lane == 17) *rn2_sh = pf_rn2;
+  }
   __syncthreads();
+  FT_STAMP(threadIdx.x == 0, 13);
+  // in whole-step mode every CTA takes the decisions, CTA 0 records them
   scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
-                        tail.rule, *rn2_sh);
+                        tail.rule, *rn2_sh, !tree.whole || blockIdx.x == 0);
+  FT_STAMP(threadIdx.x == 0, 14);
+  if (!tree.whole || bad_sh) return;                 // (after a failed pass 1 the sums mean nothing)
+  if (threadIdx.x < m) ssh[threadIdx.x] = (float)S.s[threadIdx.x];
+  __syncthreads();
+  FT_STAMP(threadIdx.x == 0, 6);
+
+  // ---- pass 2 over this CTA's tiles, newest first ----
+  // Step j < keep takes the tile of pass-1 iteration n_iter - keep + j straight from the ring; step
+  // j >= keep is load number n_iter + (j - keep) of the ring and brings tile n_iter - 1 - j back.
+  // The compute groups take the tiles in turn; both release every stage so the ring's arrival
+  // counts stay as in pass 1.
+  if (group == 2) {
+    if (lane == 0 && prod_ok) {
+      int issued_lo = n_iter, issued = n_iter;
+      bool ok = true;
+      for (int j = keep; j < n_iter; ++j) {
+        const int L = n_iter + (j - keep), s = L % stages;
+        ok = mbar_wait(smem_u32(&bar_empty[s]), ((L / stages) - 1) & 1, deadline);
+        if (!ok) break;
+        const long long tile = t_lo + (long long)(n_iter - 1 - j) * t_step;
+        const int col = (int)(tile * kFtCols);
+        const uint32_t full = smem_u32(&bar_full[s]);
+        const uint32_t dst = base + s * stage_bytes;
+        mbar_expect_tx(full, stage_bytes);
+        for (int q = 0; q < nbox; ++q) tma_load_2d(dst + q * box_bytes, &tm_g, col, q * box_rows, full);
+        tma_load_2d(dst + g_bytes, &tm_r, col, 0, full);
+        issued = L + 1;
+      }
+      if (!ok) {
+        atomicOr(status, CDG_ST_TIMEOUT);
+        for (int L = max(issued_lo, issued - stages); L < issued; ++L)
+          mbar_wait(smem_u32(&bar_full[L % stages]), (L / stages) & 1, clock64() + kCdgWaitCycles);
+      }
+    }
+  } else {
+    const int col = threadIdx.x & (kFtCols - 1);
+    bool ok = true;
+    for (int j = 0; j < n_iter; ++j) {
+      const int L = (j < keep) ? n_iter - keep + j : n_iter + (j - keep);
+      const int it = (j < keep) ? n_iter - keep + j : n_iter - 1 - j;
+      const int s = L % stages;
+      FT_STAMP(threadIdx.x == 0 && j == keep, 7);
+      if (j >= keep) ok = mbar_wait(smem_u32(&bar_full[s]), (L / stages) & 1, deadline);
+      if (!ok) break;
+      FT_STAMP(threadIdx.x == 0 && j == keep, 8);
+      if ((j & 1) == group) {
+        const T *gt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes);
+        const float *rt = reinterpret_cast<const float *>(base_ptr + (size_t)s * stage_bytes + g_bytes);
+        const long long tile = t_lo + (long long)it * t_step;
+        ft_update_tile<T, M>(gt, rt, ssh, m, col, tile * kFtCols + col, d, tree.r);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
+    }
+    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+    FT_STAMP(threadIdx.x == 0, 9);
+  }
 }
 
 bool cdg_fma_tma_supported(int m, long long d, int dtype) {
@@ -979,6 +1166,30 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
                : M == 8 ? ft_set_smem<__nv_bfloat16, 8>(h->fma_tma_smem)
                         : ft_set_smem<__nv_bfloat16, 16>(h->fma_tma_smem);
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  // reduction tree over the CTAs: groups of 12 (more when the grid is wider than 64 groups of 12)
+  h->ft_gsize = 12;
+  while ((h->gram_chunks + h->ft_gsize - 1) / h->ft_gsize > kFtMaxGroups) ++h->ft_gsize;
+  const size_t ctr_bytes = sizeof(unsigned long long) * (kFtMaxGroups + 1);
+  const size_t gp_bytes = sizeof(double) * 152 * kFtMaxGroups;
+  if (cudaMalloc(&h->ft_ctr, ctr_bytes) != cudaSuccess || cudaMalloc(&h->ft_group_partials, gp_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_NOMEM;
+  }
+  if (cudaMemset(h->ft_ctr, 0, ctr_bytes) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  h->ft_gen = 0;
+  // CDGRAB_FT_WHOLE=1: pass 2 runs inside the pass-1 launch (measured slower than two chained
+  // launches at every size tried, so off by default); needs a device that can keep the whole grid
+  // resident (cooperative launch)
+  h->fma_tma_whole = 0;
+  if (const char *e = getenv("CDGRAB_FT_WHOLE")) h->fma_tma_whole = atoi(e) ? 1 : 0;
+  h->ft_coop = 1;
+  if (const char *e = getenv("CDGRAB_FT_COOP")) h->ft_coop = atoi(e) ? 1 : 0;
+
+  int coop = 0;
+  if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h->device) != cudaSuccess || !coop) {
+    cudaGetLastError();
+    h->fma_tma_whole = 0;
+  }
   h->fma_tma = 1;
   return CDGRAB_OK;
 }
@@ -986,11 +1197,46 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
 template <typename T, int M>
 static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g, cudaStream_t st) {
   const FtTail tail = cdg_tail_of(h, h->fma_tma_fused);
+  // the whole step in this launch unless something has to happen between the passes' launches
+  const int whole = h->fma_tma_whole && h->fma_tma_fused && !h->mean_out && !h->shard;
+  FtTree tree;
+  tree.whole = whole;
+  tree.gsize = h->ft_gsize;
+  tree.gen = h->fma_tma_fused ? ++h->ft_gen : 0;
+  tree.group_ctr = h->ft_ctr;
+  tree.top_ctr = h->ft_ctr + kFtMaxGroups;
+  tree.group_partials = h->ft_group_partials;
+  tree.r = h->r;
+  h->ft_whole_launched = whole;
   {
-    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
-    cdg_launch_dep(h, gram_fma_tma_kernel<T, M>, dim3(h->gram_chunks), dim3(kFtThreads), h->fma_tma_smem, st,
-                   tm_g, h->tm_fr, h->m, h->d, h->fma_tma_stages, h->fma_tma_boxrows, h->fma_tma_contig,
-                   h->partials, h->status, tail);
+    CdgProfScope ps(h, whole ? CDGRAB_K_FUSED : CDGRAB_K_GRAM, st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(h->gram_chunks); cfg.blockDim = dim3(kFtThreads);
+    cfg.dynamicSmemBytes = h->fma_tma_smem; cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    int na = 0;
+    if (whole && h->ft_coop) {   // its CTAs wait on one another: all of them must be resident
+      at[na].id = cudaLaunchAttributeCooperative;
+      at[na].val.cooperative = 1;
+      ++na;
+    }
+    if (h->pdl && !(whole && h->ft_coop_no_pdl)) {
+      at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      at[na].val.programmaticStreamSerializationAllowed = 1;
+      ++na;
+    }
+    cfg.attrs = at; cfg.numAttrs = na;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, h->m, h->d, h->fma_tma_stages,
+                                       h->fma_tma_boxrows, h->fma_tma_contig, h->partials, h->status, tail, tree);
+    if (e != cudaSuccess && whole && h->ft_coop && na == 2) {
+      // a driver that does not take both attributes together: cooperative alone from now on
+      cudaGetLastError();
+      h->ft_coop_no_pdl = 1;
+      cfg.numAttrs = 1;
+      e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, h->m, h->d, h->fma_tma_stages,
+                             h->fma_tma_boxrows, h->fma_tma_contig, h->partials, h->status, tail, tree);
+    }
+    if (e != cudaSuccess) return e;
   }
   if (!h->fma_tma_fused) {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);

@@ -107,10 +107,13 @@ __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const d
     int oob = 0;
     if (m <= 64) {
       // The chain stays in registers: lane j holds t_j and t_{j+32}; row i of G is fetched one
-      // decision ahead, so a decision costs two shuffles and one multiply-add.
+      // decision ahead.  Only what the next decision depends on sits in the loop (broadcast t_i,
+      // decide, one multiply-add per lane); signs, norms and the non-finite check follow from the
+      // final t_j of every lane afterwards, in parallel.
       const bool h0 = lane < m, h1 = lane + 32 < m;
       double t0 = h0 ? S.t[lane] : 0.0, t1 = h1 ? S.t[lane + 32] : 0.0;
       double g0 = h0 ? G[lane] : 0.0, g1 = h1 ? G[lane + 32] : 0.0;
+      const double d0 = h0 ? G[(size_t)lane * m + lane] : 0.0, d1 = h1 ? G[(size_t)(lane + 32) * m + lane + 32] : 0.0;
       for (int i = 0; i < m; ++i) {
         double n0 = 0.0, n1 = 0.0;
         if (i + 1 < m) {
@@ -118,21 +121,35 @@ __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const d
           if (h1) n1 = G[(size_t)(i + 1) * m + lane + 32];
         }
         const double ti = __shfl_sync(0xffffffffu, (i < 32) ? t0 : t1, i & 31);
-        const double gii = __shfl_sync(0xffffffffu, (i < 32) ? g0 : g1, i & 31);
         // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0 (or the randomized rule)
-        const int s = cdg_decide(rule, i, ti, oob);
-        bad |= !(isfinite(ti) && isfinite(gii));
-        const double sd = (double)s;
+        int dummy = 0;
+        const double sd = rule.randomized ? (double)cdg_decide(rule, i, ti, dummy) : ((ti < 0.0) ? 1.0 : -1.0);
         // every later t_j gains s_i G_ij, summed in the order i = 0, 1, ...
-        if (lane > i) t0 += sd * g0;
-        if (lane + 32 > i) t1 += sd * g1;
-        if (lane == 0) { S.s[i] = s; S.rn[i] = rn2; }
-        rn2 += 2.0 * sd * ti + gii;  // ||r + s c||^2
-        if (rn2 < 0.0) rn2 = 0.0;
+        if (lane > i) t0 = fma(sd, g0, t0);
+        if (lane + 32 > i) t1 = fma(sd, g1, t1);
         g0 = n0; g1 = n1;
       }
-      if (h0) S.t[lane] = t0;
-      if (h1) S.t[lane + 32] = t1;
+      // lane j now holds t_j = <r_{j-1}, c_j> (and t_{j+32}); its sign follows from it alone
+      const int s0 = h0 ? cdg_decide(rule, lane, t0, oob) : 0, s1 = h1 ? cdg_decide(rule, lane + 32, t1, oob) : 0;
+      bad = (h0 && !(isfinite(t0) && isfinite(d0))) || (h1 && !(isfinite(t1) && isfinite(d1)));
+      // ||r||^2 seen by worker j: ||r_0||^2 + sum_{i<j} (2 s_i t_i + G_ii), an exclusive prefix sum
+      // over the lanes (first the lower 32 workers, then the upper ones)
+      double inc0 = h0 ? 2.0 * (double)s0 * t0 + d0 : 0.0, inc1 = h1 ? 2.0 * (double)s1 * t1 + d1 : 0.0;
+      double p0 = inc0, p1 = inc1;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const double u0 = __shfl_up_sync(0xffffffffu, p0, off), u1 = __shfl_up_sync(0xffffffffu, p1, off);
+        if (lane >= off) { p0 += u0; p1 += u1; }
+      }
+      const double tot0 = __shfl_sync(0xffffffffu, p0, 31);
+      const double before0 = rn2 + (p0 - inc0), before1 = rn2 + tot0 + (p1 - inc1);
+      if (h0) { S.s[lane] = s0; S.rn[lane] = before0 > 0.0 ? before0 : 0.0; S.t[lane] = t0; }
+      if (h1) { S.s[lane + 32] = s1; S.rn[lane + 32] = before1 > 0.0 ? before1 : 0.0; S.t[lane + 32] = t1; }
+      rn2 = rn2 + tot0 + __shfl_sync(0xffffffffu, p1, 31);
+      if (rn2 < 0.0) rn2 = 0.0;
+      bad = __any_sync(0xffffffffu, bad);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) oob += __shfl_xor_sync(0xffffffffu, oob, off);
     } else {
       for (int i = 0; i < m; ++i) {
         const double ti = S.t[i];

@@ -327,6 +327,38 @@ def test_tma_fma_gram_matches_register_kernel(monkeypatch):
     np.testing.assert_allclose(out[0][2].numpy(), out[1][2].numpy(), rtol=1e-4, atol=1e-7)
 
 
+@pytest.mark.parametrize("m,d,dtype", [
+    (16, 1 << 20, "f32"),            # 27-28 tiles per CTA: six stay in the ring, the rest come back in reverse
+    (16, 65_536 + 4 * 33, "f32"),    # fewer tiles than CTAs, ragged last tile
+    (9, 148 * 256 * 5, "f32"),       # exactly five tiles per CTA: fewer than the ring holds
+    (5, 148 * 256 * 9 + 8, "bf16"),  # bf16 rows, fp32 adds in pass 2
+    (16, 3_000_000, "f32"),          # long rows: pass 2 mostly from memory
+])
+def test_whole_step_launch_matches_two_launches(m, d, dtype, monkeypatch):
+    """The TMA-fed FMA path runs pass 2 inside the pass-1 launch (its CTAs meet at a bounded wait
+    between the passes); with that switched off pass 2 is the separate update kernel.  Same sums in
+    the same order: signs, r, margins and permutations must agree bit for bit, over several steps
+    (the arrival counters of the reduction tree carry over from launch to launch)."""
+    n = 8
+    outs = []
+    for whole in ("1", "0"):
+        monkeypatch.setenv("CDGRAB_FT_WHOLE", whole)
+        with binding.CdGrab(m, n, d, dtype) as h:
+            assert h.path == "fma"
+            h.begin_epoch()
+            l0 = h.launch_count
+            for k in range(n // 2):
+                h.step(random_grads(m, d, dtype, 5100 + k, mean=0.05))
+            assert h.launch_count - l0 == (n // 2) * (1 if whole == "1" else 2)
+            out = torch.empty(m, n, dtype=torch.int32, device="cuda")
+            h.end_epoch(out)
+            assert h.status() == binding.OK
+            outs.append((h.signs().cpu(), h.r().cpu(), h.margins().cpu(), out.cpu()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    assert float(outs[0][1].abs().max()) > 0
+
+
 @pytest.mark.parametrize("m,d,dtype", [(16, 100_000, "f32"), (8, 65_536, "bf16"), (32, 50_048, "bf16")])
 def test_handles_side_by_side_do_not_disturb_each_other(m, d, dtype):
     """Three handles of the same shape alive at once, stepped in turn on the same inputs: each
