@@ -53,6 +53,9 @@ def parse_args():
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="do not record per-kernel events inside the timed region")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-side-workloads", action="store_true",
+                    help="skip the brief runs of the other configurations after the headline one")
+    ap.add_argument("--oracle-child", default="", help=argparse.SUPPRESS)
     ap.add_argument("--d", type=int, default=0, help="override d (smaller cases for profiler captures)")
     ap.add_argument("--m", type=int, default=0, help="override m")
     return ap.parse_args()
@@ -254,8 +257,258 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------
+class Run:
+    """One workload set up on the current device: handle, input buffers, the step closure."""
+
+    def __init__(self, wl, local: int):
+        from paper_2302_00845_b200 import binding
+        self.wl = wl
+        m, n, d = wl.m, wl.n, wl.d
+        self.step_bytes = 2 * m * d * wl.elem_bytes
+        total_mem = torch.cuda.get_device_properties(local).total_memory
+        self.nbuf = 2 if 2 * self.step_bytes < 0.5 * total_mem else 1
+        # consecutive steps read different buffers: once those exceed L2 nothing survives between steps
+        self.flush_mode = ("inputs_larger_than_l2" if self.step_bytes * self.nbuf >= 2 * L2_BYTES
+                           else "l2_flush_between_steps")
+        self.prob = None
+        if wl.kind == "logreg":
+            # gradients are produced on the device by the library's own kernel, every step
+            self.prob = synth.LogregProblem(wl, device="cuda")
+            self.bufs = [torch.empty(2, m, d, device="cuda") for _ in range(self.nbuf)]
+        else:
+            gs = synth.GradientStream(wl, device="cuda")
+            self.bufs = [gs.step(k) for k in range(self.nbuf)]
+        self.flush = (torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+                      if self.flush_mode != "inputs_larger_than_l2" else None)
+        self.h = binding.CdGrab(m, n, d, wl.dtype)
+        self.stream = torch.cuda.current_stream()
+        self.state = {"step": 0}
+
+    def one_step(self):
+        h, wl, st = self.h, self.wl, self.state
+        if st["step"] % (wl.n // 2) == 0:
+            if st["step"]:
+                h.end_epoch()
+            h.begin_epoch()
+        buf = self.bufs[st["step"] % self.nbuf]
+        if self.prob is not None:
+            h.logreg_grads(self.prob.X, self.prob.y, self.prob.w, buf)   # gradient kernel, then the step
+        h.step(buf)                                                       # (faster than cdgrab_step_logreg)
+        st["step"] += 1
+
+    def timed_region(self, steps: int, barrier) -> float:
+        """CUDA-event time of `steps` steps in ms (the L2 flushes between them are not timed)."""
+        stream = self.stream
+        if self.flush is None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            barrier()
+            e0.record(stream)
+            for _ in range(steps):
+                self.one_step()
+            e1.record(stream)
+            barrier()
+            return e0.elapsed_time(e1)
+        evs = []
+        barrier()
+        for _ in range(steps):
+            self.flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            self.one_step()
+            b.record(stream)
+            evs.append((a, b))
+        barrier()
+        return sum(a.elapsed_time(b) for a, b in evs)
+
+    def measure(self, steps: int, warmup: int, barrier, want_events: bool):
+        """Warm up, time `steps` steps, and time the kernels.  Per-kernel event pairs sit inside the
+        timed region when a step is long enough not to notice them; a step of tens of microseconds
+        would be slowed by the records themselves (and they keep a launch from queueing behind its
+        predecessor), so there the kernels are timed over a second pass of the same steps."""
+        h = self.h
+        for _ in range(max(3, warmup)):
+            self.one_step()
+        barrier()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(self.stream)
+        for _ in range(3):
+            self.one_step()
+        p1.record(self.stream)
+        barrier()
+        events_inside = want_events and p0.elapsed_time(p1) / 3 >= 1.0
+        launches0 = h.launch_count
+        if events_inside:
+            h.profile_enable(True)
+        t0 = time.time()
+        ms = self.timed_region(steps, barrier)
+        t1 = time.time()
+        launches = h.launch_count - launches0
+        prof = h.profile_read() if events_inside else {}
+        h.profile_enable(False)
+        if want_events and not events_inside:
+            h.profile_enable(True)
+            self.timed_region(steps, barrier)
+            prof = h.profile_read()
+            h.profile_enable(False)
+        h.check_status()
+        kernel_events = "none" if not want_events else ("timed_region" if events_inside else "second_pass_of_same_steps")
+        return {"ms": ms, "launches": launches, "prof": prof, "kernel_events": kernel_events, "wall": (t0, t1)}
+
+    def model_bytes(self) -> float:
+        b2 = 2.0 * self.step_bytes + 12.0 * self.wl.d
+        b1 = 1.0 * self.step_bytes + 8.0 * self.wl.d
+        return b1 if self.h.path == "fused" else b2
+
+    def close(self):
+        self.h.destroy()
+        self.bufs = None
+        self.flush = None
+        self.prob = None
+        torch.cuda.empty_cache()
+
+
+NOMINAL_HBM_GBS = 8000.0     # the public HBM3e figure for the part, beside the measured copy rate
+
+
+def roofline_of(prof: dict, wl, peak: float, peak_kind: str):
+    """Roofline of the kernel with the largest summed time among the event pairs."""
+    if not prof:
+        return None
+    dom = max(prof, key=lambda kname: prof[kname][0])
+    tot_ms, cnt = prof[dom]
+    avg_ms = tot_ms / cnt
+    ab = algorithmic_bytes(dom, wl)
+    achieved = ab / (avg_ms * 1e-3) / 1e9
+    tr = NCU_TRAFFIC.get((dom, wl.name))
+    traffic = tr["bytes"] if tr and tr.get("source") == source_hash(tr.get("files")) else None
+    return {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
+            "peak_nominal": NOMINAL_HBM_GBS, "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
+            "above_measured_peak": achieved > peak,   # the measured peak is a copy, not a bound on reads
+            "avg_launch_ms": avg_ms, "algorithmic_bytes_per_launch": ab,
+            "kernels": {kname: {"ms_total": v[0], "launches": v[1],
+                                "share": v[0] / sum(x[0] for x in prof.values())}
+                        for kname, v in prof.items()}}
+
+
+# steps timed for the workloads reported beside the headline one (each well under two seconds)
+SIDE_STEPS = {"tiny": 200, "logreg": 200, "mid": 400, "lstm": 100, "gpt2": 10}
+
+
+def side_workloads(main_name: str, local: int, barrier, peak: float, with_oracle: bool):
+    """The other configurations of the metric, each timed briefly on the same device: path, time
+    per step, model bytes per second.  With the CPU-baseline leg on, the first steps of an epoch
+    are also replayed through the oracle (near-tie count and raw sign agreement)."""
+    out = []
+    for name in ("tiny", "logreg", "mid", "lstm", "gpt2"):
+        if name == main_name:
+            continue
+        wl = synth.WORKLOADS[name]
+        free = torch.cuda.mem_get_info()[0]
+        if 2.2 * 2 * wl.m * wl.d * wl.elem_bytes > free:
+            out.append({"workload": name, "skipped": "not enough free device memory"})
+            continue
+        run = Run(wl, local)
+        res = run.measure(SIDE_STEPS[name], 3, barrier, True)
+        ms_step = res["ms"] / SIDE_STEPS[name]
+        gbs = run.model_bytes() / (ms_step * 1e-3) / 1e9
+        entry = {"workload": name, "m": wl.m, "n": wl.n, "d": wl.d, "storage": wl.dtype, "path": run.h.path,
+                 "steps": SIDE_STEPS[name], "ms_per_step": ms_step, "cache": run.flush_mode,
+                 "launches_per_step": res["launches"] / SIDE_STEPS[name],
+                 "step_model_bytes": run.model_bytes(), "step_model_gbs": gbs, "frac_of_peak": gbs / peak,
+                 "frac_of_nominal": gbs / NOMINAL_HBM_GBS,
+                 "kernels_ms_per_launch": {k: v[0] / v[1] for k, v in res["prof"].items() if v[1]}}
+        run.close()
+        if with_oracle:
+            entry.update(first_steps_vs_oracle(wl))
+        out.append(entry)
+    return out
+
+
+def first_steps_vs_oracle(wl, seconds: float = 4.0):
+    """Part of the CPU-baseline leg: the first steps of an epoch on the device and, on the same
+    bytes, through the oracle in replay mode (it adopts the device's sign inside the tie band and
+    counts those positions; its own signs give the raw agreement)."""
+    import numpy as np
+    import oracle
+    from paper_2302_00845_b200 import binding
+    tau = 1e-6 if wl.dtype == "f32" else 1e-3
+    n_o = min(wl.n, 64)
+    h = binding.CdGrab(wl.m, n_o, wl.d, wl.dtype)
+    o = oracle.PairBalanceOracle(wl.m, n_o, wl.d)
+    prob = synth.LogregProblem(wl.scaled(n=n_o), device="cuda") if wl.kind == "logreg" else None
+    gs = None if prob is not None else synth.GradientStream(wl, device="cuda")
+    buf = torch.empty(2, wl.m, wl.d, dtype=wl.torch_dtype, device="cuda")
+    h.begin_epoch(); o.begin_epoch()
+    t0 = time.perf_counter()
+    k = 0
+    equal = 0
+    while k < n_o // 2:
+        if prob is not None:
+            h.logreg_grads(prob.X, prob.y, prob.w, buf)
+        else:
+            gs.step(k, out=buf)
+        h.step(buf)
+        s = h.signs()[:, k].cpu().numpy()
+        o.step(synth.to_host(buf), replay=s, tau=tau)
+        equal += int((o.own_signs()[:, k] == s).sum())
+        k += 1
+        if time.perf_counter() - t0 > seconds:
+            break
+    res = {"oracle_steps": k, "near_ties": o.near_ties, "mismatches_outside_band": o.mismatches,
+           "raw_agreement": equal / float(k * wl.m)}
+    h.destroy(); o.close()
+    return res
+
+
+def one_thread_oracle(name: str, seconds: float):
+    """The oracle on one host thread (a child process, OMP_NUM_THREADS=1, inputs drawn on the CPU)."""
+    env = dict(os.environ, OMP_NUM_THREADS="1", CUDA_VISIBLE_DEVICES="")
+    try:
+        res = subprocess.run([sys.executable, os.path.abspath(__file__), "--oracle-child", name,
+                              "--cpu-seconds", str(seconds)], env=env, capture_output=True, text=True, timeout=300)
+        return json.loads(res.stdout.strip().splitlines()[-1])
+    except Exception as e:  # noqa: BLE001
+        return {"workload": name, "error": str(e)[:200]}
+
+
+def oracle_child(name: str, seconds: float):
+    """Child of one_thread_oracle: times whole balancing steps of one workload on this process's threads."""
+    import numpy as np
+    import oracle
+    wl = synth.WORKLOADS[name]
+    n_o = min(wl.n, 64)
+    if wl.kind == "logreg":
+        prob = synth.LogregProblem(wl.scaled(n=n_o), device="cpu")
+        X, y, w = prob.X.numpy(), prob.y.numpy(), prob.w.numpy()
+
+        def step_rows(k):
+            g = np.empty((2, wl.m, wl.d), dtype=np.float32)
+            for i in range(wl.m):
+                for q in range(2):
+                    g[q, i] = oracle.logistic_grad(X[i, 2 * k + q], y[i, 2 * k + q], w).astype(np.float32)
+            return g
+        rows = [step_rows(k) for k in range(2)]
+    else:
+        gs = synth.GradientStream(wl, device="cpu")
+        rows = [synth.to_host(gs.step(k)) for k in range(2)]
+    o = oracle.PairBalanceOracle(wl.m, 1 << 20, wl.d)
+    o.begin_epoch()
+    done = 0
+    t0 = time.perf_counter()
+    while True:
+        o.step(rows[done % 2])
+        done += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds or done >= (1 << 19):
+            break
+    o.close()
+    print(json.dumps({"workload": name, "value": 2.0 * wl.m * done / dt, "unit": UNIT, "cores": oracle.threads(),
+                      "ms_per_step": 1e3 * dt / done, "steps": done}), flush=True)
+
+
 def run_native(args):
-    from paper_2302_00845_b200 import binding, build
+    from paper_2302_00845_b200 import build
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -270,154 +523,62 @@ def run_native(args):
     if world > 1:
         dist.barrier()
 
-    wl = pick_workload(args)
-    m, n, d = wl.m, wl.n, wl.d
-    step_bytes = 2 * m * d * wl.elem_bytes
-    total_mem = torch.cuda.get_device_properties(local).total_memory
-    nbuf = 2 if 2 * step_bytes < 0.5 * total_mem else 1
-    # consecutive steps read different buffers: once those exceed L2 nothing survives between steps
-    flush_mode = "inputs_larger_than_l2" if step_bytes * nbuf >= 2 * L2_BYTES else "l2_flush_between_steps"
-
-    prob = None
-    if wl.kind == "logreg":
-        # gradients are produced on the device by the library's own kernel, every step
-        prob = synth.LogregProblem(wl, device="cuda")
-        bufs = [torch.empty(2, m, d, device="cuda") for _ in range(nbuf)]
-    else:
-        gs = synth.GradientStream(wl, device="cuda")
-        bufs = [gs.step(k) for k in range(nbuf)]
-    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if flush_mode != "inputs_larger_than_l2" else None
-    h = binding.CdGrab(m, n, d, wl.dtype)
-    stream = torch.cuda.current_stream()
-
-    state = {"step": 0}
-
-    def one_step():
-        if state["step"] % (n // 2) == 0:
-            if state["step"]:
-                h.end_epoch()
-            h.begin_epoch()
-        buf = bufs[state["step"] % nbuf]
-        if prob is not None:
-            h.logreg_grads(prob.X, prob.y, prob.w, buf)   # gradient kernel, then the step (faster than
-        h.step(buf)                                        # the one-launch cdgrab_step_logreg: 27 vs 33 us)
-        state["step"] += 1
-
     def barrier():
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(3, args.warmup)):
-        one_step()
-    barrier()
-
-    # Per-kernel event pairs sit inside the timed region when a step is long enough not to notice
-    # them; a step of tens of microseconds would be slowed by the records themselves (and they keep
-    # a launch from queueing behind its predecessor), so there the kernels are timed over a second
-    # pass of the same K steps right after the timed one.
-    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    p0.record(stream)
-    for _ in range(3):
-        one_step()
-    p1.record(stream)
-    barrier()
-    probe_ms = p0.elapsed_time(p1) / 3
-    events_inside = (not args.no_kernel_events) and probe_ms >= 1.0
-
-    def timed_region():
-        if flush is None:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            barrier()
-            e0.record(stream)
-            for _ in range(args.steps):
-                one_step()
-            e1.record(stream)
-            barrier()
-            return e0.elapsed_time(e1)
-        evs = []
-        barrier()
-        for _ in range(args.steps):
-            flush.fill_(1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            one_step()
-            b.record(stream)
-            evs.append((a, b))
-        barrier()
-        return sum(a.elapsed_time(b) for a, b in evs)
-
+    wl = pick_workload(args)
+    m, n, d = wl.m, wl.n, wl.d
+    run = Run(wl, local)
+    h = run.h
     sampler = ClockSampler(local) if rank == 0 else None
-    launches0 = h.launch_count
-    if events_inside:
-        h.profile_enable(True)
-    t_wall0 = time.time()
-    ms = timed_region()
-    t_wall1 = time.time()
-    launches = h.launch_count - launches0
-    prof = h.profile_read() if events_inside else {}
-    h.profile_enable(False)
-    if not events_inside and not args.no_kernel_events:
-        h.profile_enable(True)
-        timed_region()
-        prof = h.profile_read()
-        h.profile_enable(False)
-    h.check_status()
-    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    res = run.measure(args.steps, args.warmup, barrier, not args.no_kernel_events)
+    clocks = sampler.stop(*res["wall"]) if sampler else None
+    value, ms = aggregate_replicas(res["ms"], 2 * m * args.steps, world, "cuda")
 
-    value, ms = aggregate_replicas(ms, 2 * m * args.steps, world, "cuda")
-
-    # ---- roofline of the dominant kernel ---------------------------------------------------
     peak, peak_kind = peaks()
-    roof = None
-    if prof:
-        dom = max(prof, key=lambda kname: prof[kname][0])
-        tot_ms, cnt = prof[dom]
-        avg_ms = tot_ms / cnt
-        ab = algorithmic_bytes(dom, wl)
-        achieved = ab / (avg_ms * 1e-3) / 1e9
-        tr = NCU_TRAFFIC.get((dom, wl.name))
-        traffic = tr["bytes"] if tr and tr.get("source") == source_hash(tr.get("files")) else None
-        roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
-                "avg_launch_ms": avg_ms, "algorithmic_bytes_per_launch": ab,
-                "kernels": {kname: {"ms_total": v[0], "launches": v[1],
-                                    "share": v[0] / sum(x[0] for x in prof.values())}
-                            for kname, v in prof.items()}}
-    step_model_b2 = 2.0 * step_bytes + 12.0 * d
-    step_model_b1 = 1.0 * step_bytes + 8.0 * d
-    model = step_model_b1 if h.path == "fused" else step_model_b2
+    roof = roofline_of(res["prof"], wl, peak, peak_kind)
+    model = run.model_bytes()
     step_gbs = model / (ms / args.steps * 1e-3) / 1e9
 
     # ---- end to end through the host-buffer call ----------------------------------------------
     e2e = None
     if not args.no_e2e and world == 1:
-        e2e = run_e2e(h, wl, bufs[0], state, one_step)
+        e2e = run_e2e(h, wl, run.bufs[0], run.state, run.one_step)
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    with_oracle = rank == 0 and world == 1 and not args.no_cpu_baseline
+    if with_oracle:
         torch.cuda.synchronize()
-        cpu = oracle_sample(wl, bufs[0], args.cpu_seconds)
+        cpu = oracle_sample(wl, run.bufs[0], args.cpu_seconds)
+    path, step_bytes, nbuf, flush_mode = h.path, run.step_bytes, run.nbuf, run.flush_mode
+    run.close()
+
+    # ---- the other configurations of the metric, briefly, after the headline one ---------------
+    side = None
+    if rank == 0 and world == 1 and not args.no_side_workloads and not args.d and not args.m:
+        side = side_workloads(wl.name, local, barrier, peak, with_oracle)
+        if with_oracle:
+            cpu["one_thread"] = [one_thread_oracle(name, 3.0) for name in ("tiny", "logreg", "mid")]
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "m": m, "n": n, "d": d, "storage": wl.dtype,
-                       "path": h.path, "step_input_bytes": step_bytes, "input_buffers": nbuf,
-                       "cache": flush_mode,
-                       "kernel_events": "none" if args.no_kernel_events else
-                                        ("timed_region" if events_inside else "second_pass_of_same_steps"),
+            "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "m": m, "n": n, "d": d, "storage": wl.dtype, "accumulate": "f32",
+                       "path": path, "step_input_bytes": step_bytes, "input_buffers": nbuf,
+                       "cache": flush_mode, "kernel_events": res["kernel_events"],
                        "parallelism": "replicas" if world > 1 else "single",
                        "step_model_bytes": model, "step_model_gbs": step_gbs,
-                       "step_model_frac_of_peak": step_gbs / peak},
-            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-            "clocks": clocks,
+                       "step_model_frac_of_peak": step_gbs / peak,
+                       "step_model_frac_of_nominal": step_gbs / NOMINAL_HBM_GBS},
+            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": res["launches"],
+            "clocks": clocks, "workloads": side,
         }
         print(json.dumps(line), flush=True)
-    h.destroy()
     if world > 1:
         dist.destroy_process_group()
 
@@ -463,7 +624,9 @@ def run_e2e(h, wl, dev_buf, state, one_step):
 
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.oracle_child:
+        oracle_child(args.oracle_child, args.cpu_seconds)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_native(args)

@@ -353,9 +353,19 @@ int cdgrab_herding_objective(const float *z_dev, const int32_t *perms_dev, int m
  * words that must start at zero are cleared on `stream` at every call.  Two calls whose
  * device work may overlap (different streams without ordering, or several host threads)
  * race on the scratch: order them.
+ *
+ * Device-side conditions (a NaN/Inf met in a reduction) are recorded in a status word inside
+ * the scratch; it stays set over later calls until cdgrab_noalloc_status reads it.
  */
 int cdgrab_step_noalloc(int m, long long d, int dtype, const void *grads_dev, float *r_dev,
                         int8_t *signs_out_dev, void *stream);
+
+/* What the kernels of cdgrab_step_noalloc reported on the current device since the last call of
+ * this function (the paper has no counterpart): CDGRAB_OK, CDGRAB_ERR_NONFINITE or
+ * CDGRAB_ERR_TIMEOUT.  Synchronises the device, copies one word out of the fixed scratch and
+ * clears it when set; allocates nothing.  CDGRAB_OK when no step has run on this device yet.
+ * Not to be called while a stream capture is open (it synchronises). */
+int cdgrab_noalloc_status(void);
 
 #ifdef __cplusplus
 }

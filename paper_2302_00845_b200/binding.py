@@ -63,6 +63,7 @@ SIGNATURES = {
                                            C.c_longlong, C.c_void_p, C.c_void_p]),
     "cdgrab_step_noalloc": (C.c_int, [C.c_int, C.c_longlong, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p]),
+    "cdgrab_noalloc_status": (C.c_int, []),
 }
 
 _lib = None
@@ -286,6 +287,11 @@ def step_noalloc(grads, r, signs_out, stream=None):
     code = F32 if grads.dtype == torch.float32 else BF16
     _check(lib().cdgrab_step_noalloc(m, d, code, _ptr(grads), _ptr(r), _ptr(signs_out), _stream_ptr(stream)),
            "cdgrab_step_noalloc")
+
+
+def noalloc_status() -> int:
+    """cdgrab_noalloc_status: the device status of the step_noalloc calls so far (read and cleared)."""
+    return int(lib().cdgrab_noalloc_status())
 
 
 def herding_objective(z, perms, stream=None) -> float:

@@ -111,11 +111,39 @@ extern "C" int cdgrab_step_noalloc(int m, long long d, int dtype, const void *gr
   if (blocks > cap) blocks = cap;
   c.gram_chunks = (int)blocks;
 
-  // the tracked squared norm and the status word are read before they are written
-  if (cudaMemsetAsync(nd.scratch + kOffRnorm2, 0, 16, st) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  // the tracked squared norm is read before it is written; the status word beside it is sticky
+  // (bits only ever get set by the kernels) until cdgrab_noalloc_status reads and clears it
+  if (cudaMemsetAsync(nd.scratch + kOffRnorm2, 0, 8, st) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
   cudaError_t e = cdg_launch_gram_fma(&c, grads_dev, st);
   if (e == cudaSuccess) e = cdg_launch_scan(&c, st);
   if (e == cudaSuccess) e = cdg_launch_update(&c, grads_dev, st);
   if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  return CDGRAB_OK;
+}
+
+// What the kernels of cdgrab_step_noalloc reported on the current device since the last call of
+// this function: the status word sits in the fixed scratch, where no caller could read it.
+// Synchronises the device, copies the word out, clears it when it is set.  Allocates nothing.
+extern "C" int cdgrab_noalloc_status(void) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_DEVICE; }
+  if (dev < 0 || dev >= kNaMaxDevices) return CDGRAB_ERR_DEVICE;
+  const NaDevice &nd = g_na_dev[dev];
+  if (!nd.ready) return CDGRAB_OK;             // no step has run on this device yet
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  int st = 0;
+  if (cudaMemcpy(&st, nd.scratch + kOffStatus, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  if (st != 0) {
+    const int zero = 0;
+    if (cudaMemcpy(nd.scratch + kOffStatus, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaGetLastError();
+      return CDGRAB_ERR_CUDA;
+    }
+  }
+  if (st & CDG_ST_TIMEOUT) return CDGRAB_ERR_TIMEOUT;
+  if (st & CDG_ST_NONFINITE) return CDGRAB_ERR_NONFINITE;
   return CDGRAB_OK;
 }
