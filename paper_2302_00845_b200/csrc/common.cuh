@@ -89,6 +89,9 @@ struct cdgrab_ctx {
   unsigned long long *ft_ctr;         // [groups + 1] arrival counters of the tree
   double *ft_group_partials;          // [groups][152]
   size_t fma_tma_smem;
+  int fma_tma_defer;       // 1: cdgrab_step_many folds pass 2 of a step into pass 1 of the next one
+  int fma_tma_stages2;     // ring depth and shared memory of that form (a stage holds two steps' rows)
+  size_t fma_tma_smem2;
   CUtensorMap tm_fr;       // 2-D map over r (one row)
   CdgMapCache<1> tm_fg;    // 2-D maps over the gradient rows of the last few buffers
 
@@ -117,9 +120,21 @@ struct cdgrab_ctx {
   int umma_g4;             // row groups one 4-D copy brings in (0: per-group copies only)
   int umma_paired;         // 2m <= 64: one MMA covers two 64-column blocks
   int umma_fused;          // the combine launch also takes the decisions (last block)
-  int umma_split3;         // fp32 inputs: the MMA rows are the differences as three bf16 terms each
-  int umma_rows;           // rows of the MMA operand: 2m (bf16 gradients) or 3m (split differences)
-  __nv_bfloat16 *umma_csplit;   // [3m][d_pad] hi / mid / lo terms of c_i = z1_i - z2_i (fp32 inputs)
+  int umma_rows;           // rows of the MMA operand: 2m
+
+  // tcgen05 path for fp32 gradients with the bf16 terms formed inside the kernel
+  int umma_f32;            // 1: that kernel serves pass 1
+  int f32_npad;            // MMA N: 3m rounded up to 16
+  int f32_nsub;            // 64-column blocks per stage
+  int f32_nops;            // operand buffers
+  int f32_stages;
+  int f32_drain;           // 64-column blocks per TMEM accumulation chunk
+  int f32_ctas;
+  size_t f32_smem;
+  double *f32_bpart;       // [ctas][64] per-CTA partial b
+  double *f32_dsum;        // [128][192] the partial D summed over the CTAs
+  CUtensorMap tm_f32r;     // 2-D map over r (one row)
+  CdgMapCache<1> tm_f32g;  // 2-D maps over the gradient rows of the last few buffers
 };
 
 template <typename T>
@@ -215,6 +230,8 @@ void *cdg_tensor_map_encoder();
 bool cdg_fma_tma_supported(int m, long long d, int dtype);
 int cdg_fma_tma_setup(cdgrab_ctx *h);
 cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+// ... that first applies the open update of the step before (rows at grads_prev, signs at k - 1)
+cudaError_t cdg_launch_gram_fma_tma_deferred(cdgrab_ctx *h, const void *grads, const void *grads_prev, cudaStream_t st);
 
 // ID-GraB (independent workers)
 int cdg_indep_chunks(const cdgrab_ctx *h);
@@ -227,3 +244,8 @@ bool cdg_umma_supported(int m, long long d, int dtype);
 int cdg_umma_setup(cdgrab_ctx *h);   // allocations + tensor maps; CDGRAB_* code
 void cdg_umma_teardown(cdgrab_ctx *h);
 cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
+// ... for fp32 gradients, terms formed in the kernel (17 <= m <= 64)
+bool cdg_umma_f32_supported(int m, long long d);
+int cdg_umma_f32_setup(cdgrab_ctx *h);
+void cdg_umma_f32_teardown(cdgrab_ctx *h);
+cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStream_t st);

@@ -31,6 +31,7 @@
 // drains the copies it has in flight, frees its TMEM and returns.
 #include <cudaTypedefs.h>
 #include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -345,7 +346,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
 // 32 lane sums are then added by a fixed butterfly.  Eight entries per block spread the loads
 // over many SMs (an SM can keep only so many of these scattered loads in flight).
 __global__ void __launch_bounds__(256)
-umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows, int m, int split3,
+umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int box_rows, int m,
                     double *__restrict__ gram, int *__restrict__ status, const CdgTail tail) {
   __shared__ double scan_sh[4 * 64 + 64 * 64];     // m <= 64 on this path
   __shared__ int is_last;
@@ -355,34 +356,7 @@ umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int
   const int e = blockIdx.x * 8 + warp;
   const size_t cs = (size_t)128 * ncols;   // one CTA's partial H
   double acc = 0.0;
-  if (split3) {
-    // rows p*m + i hold term p (hi, mid, lo) of c_i:  G_ki = sum over the nine term pairs,
-    // b_i = sum over the three terms of row i and the three terms of r
-    if (e < m * m) {
-      const int k = e / m, i = e % m;
-      for (int c = lane; c < ctas; c += 32) {
-        const float *P = partials + (size_t)c * cs;
-        double v = 0.0;
-#pragma unroll
-        for (int pa = 0; pa < 3; ++pa)
-#pragma unroll
-          for (int pb = 0; pb < 3; ++pb) v += (double)P[(size_t)(pa * m + k) * ncols + pb * m + i];
-        acc += v;
-      }
-    } else if (e < total) {
-      const int i = e - m * m;
-      for (int c = lane; c < ctas; c += 32) {
-        const float *P = partials + (size_t)c * cs;
-        double v = 0.0;
-#pragma unroll
-        for (int pa = 0; pa < 3; ++pa) {
-          const size_t o = (size_t)(pa * m + i) * ncols + box_rows;
-          v += ((double)P[o] + (double)P[o + 1]) + (double)P[o + 2];
-        }
-        acc += v;
-      }
-    }
-  } else if (e < m * m) {
+  if (e < m * m) {
     const int k = e / m, i = e % m;
     const size_t o00 = (size_t)k * ncols + i, o01 = o00 + m, o10 = (size_t)(m + k) * ncols + i, o11 = o10 + m;
 #pragma unroll 5
@@ -420,45 +394,6 @@ umma_combine_kernel(const float *__restrict__ partials, int ctas, int ncols, int
   __syncthreads();
   scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
                         tail.rule);
-}
-
-// fp32 gradients: c_i = z1_i - z2_i (rounded to fp32 like every other path forms it) written as
-// three bf16 terms hi + mid + lo = c exactly (3 x 8 significand bits), rows [term][worker] of
-// out[3m][d_pad].  Products of bf16 terms are exact in the fp32 accumulator, so the nine term
-// products of a pair add up to c_k c_i without a rounded product.  grid (column chunks, m).
-__global__ void __launch_bounds__(256)
-split_diff_kernel(const float *__restrict__ g, int m, long long d, long long d_pad,
-                  __nv_bfloat16 *__restrict__ out) {
-  cdg_grid_dep_wait();            // the last launch may still read the terms of the step before
-  const int i = blockIdx.y;
-  const float *z1 = g + (size_t)i * (size_t)d, *z2 = g + ((size_t)m + i) * (size_t)d;
-  __nv_bfloat16 *o0 = out + (size_t)i * (size_t)d_pad;
-  __nv_bfloat16 *o1 = out + ((size_t)m + i) * (size_t)d_pad;
-  __nv_bfloat16 *o2 = out + (2 * (size_t)m + i) * (size_t)d_pad;
-  const long long nvec = d / 8;
-  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += (long long)gridDim.x * blockDim.x) {
-    const size_t x = (size_t)v * 8;
-    float a[8], b[8];
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const float4 fa = __ldg(reinterpret_cast<const float4 *>(z1 + x) + q);
-      const float4 fb = __ldg(reinterpret_cast<const float4 *>(z2 + x) + q);
-      a[4 * q] = fa.x; a[4 * q + 1] = fa.y; a[4 * q + 2] = fa.z; a[4 * q + 3] = fa.w;
-      b[4 * q] = fb.x; b[4 * q + 1] = fb.y; b[4 * q + 2] = fb.z; b[4 * q + 3] = fb.w;
-    }
-    __nv_bfloat16 hi[8], mid[8], lo[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float c = a[j] - b[j];
-      hi[j] = __float2bfloat16_rn(c);
-      const float r1 = c - __bfloat162float(hi[j]);
-      mid[j] = __float2bfloat16_rn(r1);
-      lo[j] = __float2bfloat16_rn(r1 - __bfloat162float(mid[j]));
-    }
-    *reinterpret_cast<uint4 *>(o0 + x) = *reinterpret_cast<const uint4 *>(hi);
-    *reinterpret_cast<uint4 *>(o1 + x) = *reinterpret_cast<const uint4 *>(mid);
-    *reinterpret_cast<uint4 *>(o2 + x) = *reinterpret_cast<const uint4 *>(lo);
-  }
 }
 
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
@@ -545,19 +480,21 @@ void *cdg_tensor_map_encoder() { return (void *)encode_fn(); }
 
 bool cdg_umma_supported(int m, long long d, int dtype) {
   // rows whose pitch is a multiple of 16 bytes
+  if (dtype == CDGRAB_F32) {
+    // fp32 gradients: the differences go in as three bf16 terms each, formed inside the kernel
+    // (CDGRAB_UMMA_F32=0: fp32 gradients stay off the tensor cores)
+    const char *e = getenv("CDGRAB_UMMA_F32");
+    if (e && !strcmp(e, "0")) return false;
+    return cdg_umma_f32_supported(m, d);
+  }
   if (d % 8 != 0 || d < 4096 || encode_fn() == nullptr) return false;
   // bf16 gradients: the 2m rows fit one 128-row MMA tile
-  if (dtype == CDGRAB_BF16) return m <= 64;
-  // fp32 gradients: the differences as three bf16 terms each, 3m rows (CDGRAB_UMMA_F32=0: not used)
-  if (const char *e = getenv("CDGRAB_UMMA_F32")) {
-    if (atoi(e) == 0) return false;
-  }
-  return 3 * m <= 128;
+  return m <= 64;
 }
 
 int cdg_umma_setup(cdgrab_ctx *h) {
-  h->umma_split3 = (h->dtype == CDGRAB_F32) ? 1 : 0;
-  h->umma_rows = h->umma_split3 ? 3 * h->m : 2 * h->m;
+  if (h->dtype == CDGRAB_F32) return cdg_umma_f32_setup(h);
+  h->umma_rows = 2 * h->m;
   h->umma_paired = (h->umma_rows <= 64) ? 1 : 0;  // CDGRAB_UMMA_PAIRED=0: one block per MMA
   if (const char *e = getenv("CDGRAB_UMMA_PAIRED")) {
     if (atoi(e) == 0) h->umma_paired = 0;
@@ -577,8 +514,7 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   if (h->umma_paired && (subs & 1)) ++subs;      // two halves per stage
   h->umma_subs_per_stage = subs;
   // TMEM chunk length in pipeline iterations (about 4096 columns); CDGRAB_UMMA_DRAIN overrides
-  // (fp32 inputs are held to a tighter sign tolerance: chunks of about 512 columns)
-  const int chunk_cols = h->umma_split3 ? 512 : 4096;
+  const int chunk_cols = 4096;
   h->umma_drain = chunk_cols / (subs * kSubCols) > 0 ? chunk_cols / (subs * kSubCols) : 1;
   if (const char *e = getenv("CDGRAB_UMMA_DRAIN")) {
     const int v = atoi(e);
@@ -607,11 +543,6 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     cudaGetLastError();
     return CDGRAB_ERR_NOMEM;
   }
-  if (h->umma_split3) {
-    const size_t bytes = sizeof(__nv_bfloat16) * 3 * (size_t)h->m * (size_t)h->d_pad;
-    if (cudaMalloc(&h->umma_csplit, bytes) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_NOMEM; }
-    if (cudaMemset(h->umma_csplit, 0, bytes) != cudaSuccess) return CDGRAB_ERR_CUDA;
-  }
   if (cudaMemset(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
       cudaMemset(h->umma_partials, 0, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess)
     return CDGRAB_ERR_CUDA;
@@ -628,8 +559,7 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   if (const char *e = getenv("CDGRAB_UMMA_G4")) {
     if (atoi(e) == 0) h->umma_g4 = 0;
   }
-  const long long row_pitch = h->umma_split3 ? h->d_pad : h->d;
-  if (row_pitch * 16 >= (1ll << 40)) h->umma_g4 = 0;             // the group stride must fit the map
+  if (h->d * 16 >= (1ll << 40)) h->umma_g4 = 0;             // the group stride must fit the map
   h->umma_fused = h->shard ? 0 : 1;      // a shard's decisions wait for the sum over shards
   if (const char *e = getenv("CDGRAB_UMMA_FUSE_TAIL")) {
     if (atoi(e) == 0) h->umma_fused = 0;
@@ -638,28 +568,19 @@ int cdg_umma_setup(cdgrab_ctx *h) {
 }
 
 void cdg_umma_teardown(cdgrab_ctx *h) {
+  cdg_umma_f32_teardown(h);
   cudaFree(h->r_split);
   cudaFree(h->umma_partials);
-  cudaFree(h->umma_csplit);
-  h->umma_csplit = nullptr;
   h->r_split = nullptr;
   h->umma_partials = nullptr;
 }
 
 cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  if (h->umma_f32) return cdg_launch_gram_umma_f32(h, grads, st);
   const long long nblk_full = h->d / kSubCols;
-  // the MMA's rows: the caller's bf16 gradients, or the split differences of fp32 gradients
-  const void *src = h->umma_split3 ? (const void *)h->umma_csplit : grads;
-  const long long pitch = h->umma_split3 ? h->d_pad : h->d;
+  const void *src = grads;             // the MMA's rows are the caller's bf16 gradients as they lie in HBM
+  const long long pitch = h->d;
   const int rows = h->umma_rows;
-  if (h->umma_split3) {
-    long long chunks = (h->d / 8 + 255) / 256;
-    const long long cap = (8ll * h->num_sms + h->m - 1) / h->m;
-    if (chunks > cap) chunks = cap;
-    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
-    cdg_launch_dep(h, split_diff_kernel, dim3((unsigned)chunks, h->m), dim3(256), 0, st, (const float *)grads, h->m,
-                   h->d, h->d_pad, h->umma_csplit);
-  }
   int slot = h->tm_g.find(src);
   if (slot < 0) {
     slot = h->tm_g.victim();
@@ -693,7 +614,7 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
     const int total = h->m * h->m + h->m;
     cdg_launch_dep(h, umma_combine_kernel, dim3((total + 7) / 8), dim3(256), 0, st, h->umma_partials, h->umma_ctas,
-                   h->umma_ncols, h->umma_box_rows, h->m, h->umma_split3, h->gram, h->status,
+                   h->umma_ncols, h->umma_box_rows, h->m, h->gram, h->status,
                    cdg_tail_of(h, h->umma_fused));
   }
   return cudaGetLastError();

@@ -1,0 +1,625 @@
+// Pass 1 on the tensor cores (tcgen05) for fp32 gradients, 17 <= m <= 64.
+//
+// The pair differences c_i = z1_i - z2_i (rounded to fp32, as every other path forms them) are
+// written as three bf16 terms hi + mid + lo = c exactly (3 x 8 significand bits).  Products of
+// bf16 terms are exact in the fp32 accumulator, so <c_k, c_i> is the sum of the nine term
+// products; the lo x lo one (below 2^-32 of the product) is left out, the other eight come out
+// of ONE product per 16 columns:  D = A B^T with B = [hi_0..hi_{m-1} | mid_0.. | lo_0..] (3m
+// rows, the MMA's N) and A = the first 128 of those rows (hi and mid, the MMA's M):
+//     G_ki = D[k][i] + D[k][m+i] + D[k][2m+i] + D[m+k][i] + D[m+k][m+i] + D[m+k][2m+i]
+//            + D[i][2m+k] + D[m+i][2m+k]          (the last two are lo_k x hi_i and lo_k x mid_i).
+// The terms are formed inside the kernel: TMA brings fp32 tiles [2m rows][64 s columns] and the
+// matching piece of r into a ring of stages; six converter warps read them, subtract, split,
+// and store the bf16 terms into an operand buffer in the K-major 128-byte-swizzled layout the
+// MMA reads ([8-row group][8 rows][128 B], 16-byte chunk c of row q at chunk c ^ (q & 7)).  The
+// same warps add up b_i = <r, c_i> on the FMA pipe (fp32 products, moved into fp64 every 32
+// blocks), so r needs no bf16 copy on this path.  Nothing but the caller's rows and r is read
+// from HBM: 2mde + 4d bytes per launch.
+//
+// Roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2..7
+// converters, warps 8..15 read the accumulator back.  The sum stays in TMEM for `drain` blocks
+// of 64 columns only (the tensor core's fp32 accumulation truncates), then the read-back warps
+// add the chunk to fp32 registers (round to nearest) while the MMAs fill the other buffer.
+// One persistent CTA per SM owns a contiguous range of 64-column blocks; its partial D and b
+// go to global memory, a second kernel adds the CTAs in index order in fp64, forms G and takes
+// the step's decisions.  Every wait is bounded: on expiry the CTA raises the time-out bit of the
+// status word, lets its copies land, frees its TMEM and returns.
+#include <cudaTypedefs.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+#include "scan.cuh"
+
+namespace {
+
+#ifndef CDG_F32_CONV_WARPS
+#define CDG_F32_CONV_WARPS 6
+#endif
+constexpr int kConvWarps = CDG_F32_CONV_WARPS;
+constexpr int kConvThreads = 32 * kConvWarps;       // 16 float4 of a 64-column block x kConvRows rows at a time
+constexpr int kConvRows = kConvThreads / 16;
+constexpr int kDrainWarps = 8;
+constexpr int kThreads = 64 + kConvThreads + 32 * kDrainWarps;
+constexpr int kMaxStages = 8;
+constexpr int kMaxOps = 4;                           // operand buffers (one 64-column block each)
+constexpr int kRowSlots = (64 + kConvRows - 1) / kConvRows;   // rows per converter thread at m = 64
+constexpr int kBlockCols = 64;                       // columns per MMA block = one 128-byte swizzle row of bf16
+constexpr int kFlushBlocks = 32;                     // blocks between two moves of the fp32 b sums into fp64
+constexpr int kMaxN = 192;                           // 3 m at m = 64
+
+struct F32Params {
+  int m;
+  int npad;            // MMA N: 3m rounded up to 16
+  int nsub;            // 64-column blocks per stage
+  int stages;
+  int nops;            // operand buffers
+  int drain;           // blocks accumulated in TMEM before the sum is read back
+  long long nblk;      // ceil(d / 64)
+};
+
+__device__ __forceinline__ uint64_t f32_umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address
+  d |= (uint64_t)1 << 16;                          // leading byte offset (unused for this layout)
+  d |= (uint64_t)(1024u >> 4) << 32;               // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                          // descriptor version
+  d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+  return d;
+}
+__device__ __forceinline__ void f32_umma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ __forceinline__ bool f32_elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+  return pred != 0;
+}
+__device__ __forceinline__ void f32_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// two floats rounded to bf16 (to nearest even), x in the low half
+__device__ __forceinline__ uint32_t pack_bf16x2(float x, float y) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+  return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+// NS: rows each converter thread takes = ceil(m / kConvRows), a compile-time count so that the
+// NS x 2 split chains of a block sit in one basic block and the scheduler can interleave them.
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1)
+gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
+                     const F32Params p, float *__restrict__ partials, double *__restrict__ bpart,
+                     int *__restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[kMaxStages];     // stage s holds a landed tile
+  __shared__ __align__(8) uint64_t bar_empty[kMaxStages];    // ... has been converted
+  __shared__ __align__(8) uint64_t bar_op_full[kMaxOps];     // operand buffer o holds the terms of a block
+  __shared__ __align__(8) uint64_t bar_op_empty[kMaxOps];    // ... has been read by its MMAs
+  __shared__ __align__(8) uint64_t bar_acc_full[2];
+  __shared__ __align__(8) uint64_t bar_acc_empty[2];
+  __shared__ uint32_t tmem_base_sh;
+  __shared__ double bred[kConvThreads * NS];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = p.m;
+  const int scols = p.nsub * kBlockCols;
+  const int rows8 = (2 * m + 7) & ~7;                                      // rows a stage holds (8-row boxes)
+  const uint32_t stage_bytes = (uint32_t)(rows8 + 1) * scols * 4u;         // the rows, then the piece of r
+  const int op_rows = p.npad > 128 ? p.npad : 128;                         // operand A spans 128 rows
+  const uint32_t op_bytes = (uint32_t)op_rows * 128u;
+  const uint32_t ops_base = (smem_u32(smem_raw) + 1023u) & ~1023u;         // swizzle atoms need 1024-B alignment
+  uint8_t *ops_ptr = smem_raw + (ops_base - smem_u32(smem_raw));
+  const uint32_t stages_base = ops_base + (uint32_t)p.nops * op_bytes;
+  uint8_t *stages_ptr = ops_ptr + (size_t)p.nops * op_bytes;
+
+  const long long blk_lo = p.nblk * (long long)blockIdx.x / gridDim.x;
+  const long long blk_hi = p.nblk * (long long)(blockIdx.x + 1) / gridDim.x;
+  const int nsb = (int)(blk_hi - blk_lo);                                  // 64-column blocks of this CTA
+  const int n_iter = (nsb + p.nsub - 1) / p.nsub;                          // stages it streams
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), kConvWarps);
+    }
+    for (int o = 0; o < p.nops; ++o) {
+      mbar_init(smem_u32(&bar_op_full[o]), kConvWarps);
+      mbar_init(smem_u32(&bar_op_empty[o]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bar_acc_full[b]), 1);
+      mbar_init(smem_u32(&bar_acc_empty[b]), kDrainWarps);
+    }
+    mbar_init_fence();
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_g) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_r) : "memory");
+  }
+  // operand rows no converter ever writes (past the 3m term rows) are zeroed once
+  for (int o = 0; o < p.nops; ++o) {
+    uint8_t *z = ops_ptr + (size_t)o * op_bytes + (size_t)(3 * m) * 128;   // whole rows: 128 B each, swizzle-neutral
+    const uint32_t nbytes = (uint32_t)(op_rows - 3 * m) * 128u;
+    for (uint32_t off = threadIdx.x * 16; off < nbytes; off += kThreads * 16)
+      *reinterpret_cast<uint4 *>(z + off) = make_uint4(0, 0, 0, 0);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_sh)), "r"(512u) : "memory");   // two accumulators of 256 columns
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = tmem_base_sh;
+  cdg_grid_dep_wait();            // r is written by the launch before this one
+  const long long deadline = clock64() + kCdgWaitCycles;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      const int nbox = rows8 >> 3;
+      const uint32_t box_bytes = 8u * scols * 4u;
+      int issued = 0;
+      bool ok = true;
+      int s = 0;
+      uint32_t turn = 0;
+      for (int it = 0; it < n_iter; ++it) {
+        if (turn > 0) ok = mbar_wait(smem_u32(&bar_empty[s]), (turn - 1) & 1, deadline);
+        if (!ok) break;
+        const int col = (int)((blk_lo + (long long)it * p.nsub) * kBlockCols);   // a multiple of 64 floats
+        const uint32_t full = smem_u32(&bar_full[s]);
+        const uint32_t dst = stages_base + (uint32_t)s * stage_bytes;
+        mbar_expect_tx(full, stage_bytes);
+        for (int q = 0; q < nbox; ++q) tma_load_2d(dst + q * box_bytes, &tm_g, col, q * 8, full);
+        tma_load_2d(dst + nbox * box_bytes, &tm_r, col, 0, full);
+        issued = it + 1;
+        if (++s == p.stages) { s = 0; ++turn; }
+      }
+      if (!ok) {
+        atomicOr(status, CDG_ST_TIMEOUT);
+        for (int it = max(0, issued - p.stages); it < issued; ++it)
+          mbar_wait(smem_u32(&bar_full[it % p.stages]), (it / p.stages) & 1, clock64() + kCdgWaitCycles);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: the warp loops converged, an elected lane issues ----------------
+    // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = npad
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)p.npad >> 3) << 17) | ((128u >> 4) << 24);
+    bool ok = true;
+    int o = 0, c = 0, in_chunk = 0;
+    uint32_t op_parity = 0;
+    for (int g = 0; g < nsb; ++g) {
+      const int buf = c & 1;
+      const bool chunk_start = in_chunk == 0;
+      if (chunk_start && c >= 2) ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), ((c >> 1) - 1) & 1, deadline);
+      if (ok) ok = mbar_wait(smem_u32(&bar_op_full[o]), op_parity, deadline);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t acc = tmem_acc + (uint32_t)buf * 256u;
+      const uint64_t desc = f32_umma_desc(ops_base + (uint32_t)o * op_bytes);
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const uint64_t dk = desc + (uint64_t)(k4 * 2);     // 16 bf16 = 32 bytes further along K
+        if (f32_elect_one()) f32_umma(acc, dk, dk, idesc, !(chunk_start && k4 == 0));
+      }
+      const bool chunk_end = (in_chunk == p.drain - 1) || (g == nsb - 1);
+      if (f32_elect_one()) {
+        f32_commit(smem_u32(&bar_op_empty[o]));
+        if (chunk_end) f32_commit(smem_u32(&bar_acc_full[buf]));
+      }
+      if (++in_chunk == p.drain) { in_chunk = 0; ++c; }
+      if (++o == p.nops) { o = 0; op_parity ^= 1u; }
+    }
+    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+  } else if (warp < 2 + kConvWarps) {
+    // ---------------- converters: fp32 tile -> differences -> three bf16 terms; b on the side ----------------
+    const int ct = threadIdx.x - 64;                 // 0..191
+    const int q = ct & 15;                           // this thread's float4 of every row it takes
+    const int row0 = ct >> 4;                        // rows row0, row0 + 12, ...
+    // Byte offsets that never change: of the thread's float4 inside a stage (block 0) and of its
+    // 8 bytes of terms inside an operand buffer -- row i, m + i, 2m + i, each 128 B, 16-byte
+    // chunk (q >> 1) at chunk (q >> 1) ^ (row & 7), upper half of the chunk for odd q.
+    uint32_t src[NS], dst_h[NS], dst_m[NS], dst_l[NS];
+    uint32_t vmask = 0;
+#pragma unroll
+    for (int j = 0; j < NS; ++j) {
+      int i = row0 + kConvRows * j;
+      if (i < m) vmask |= 1u << j;
+      else i = m - 1;                                // a slot past the last row loads a valid row and stores nothing
+      const int im = m + i, il = 2 * m + i;
+      src[j] = (uint32_t)(i * scols + q * 4) * 4u;
+      dst_h[j] = (uint32_t)(i * 128 + ((((q >> 1) ^ (i & 7)) << 4) | ((q & 1) << 3)));
+      dst_m[j] = (uint32_t)(im * 128 + ((((q >> 1) ^ (im & 7)) << 4) | ((q & 1) << 3)));
+      dst_l[j] = (uint32_t)(il * 128 + ((((q >> 1) ^ (il & 7)) << 4) | ((q & 1) << 3)));
+    }
+    const uint32_t z2_off = (uint32_t)(m * scols) * 4u;          // from a row of slab 0 to its partner in slab 1
+    float bacc[NS];
+    double bsum[NS];
+#pragma unroll
+    for (int j = 0; j < NS; ++j) { bacc[j] = 0.f; bsum[j] = 0.0; }
+    bool ok = true;
+    int s = 0, o = 0, since_flush = 0;
+    uint32_t full_parity = 0, turn_o = 0;
+    for (int it = 0; it < n_iter && ok; ++it) {
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_full[s]), full_parity, deadline));   // the lanes leave together
+      if (!ok) break;
+      const uint8_t *tile = stages_ptr + (size_t)s * stage_bytes;
+      const float *rt = reinterpret_cast<const float *>(tile) + (size_t)rows8 * scols;
+      const int cnt = min(p.nsub, nsb - it * p.nsub);      // blocks past the range belong to the next CTA
+      for (int sub = 0; sub < cnt; ++sub) {
+        // Straight-line code from here to the stores: every load first, then the split one step
+        // at a time over all slots (each step's 2 NS operations are independent of one another).
+        const float4 rv = *reinterpret_cast<const float4 *>(rt + sub * kBlockCols + q * 4);
+        float c[NS][4];
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+          const float4 za = *reinterpret_cast<const float4 *>(tile + src[j] + sub * (kBlockCols * 4));
+          const float4 zb = *reinterpret_cast<const float4 *>(tile + src[j] + z2_off + sub * (kBlockCols * 4));
+          c[j][0] = za.x - zb.x; c[j][1] = za.y - zb.y; c[j][2] = za.z - zb.z; c[j][3] = za.w - zb.w;
+        }
+        uint32_t hi[NS][2], mid[NS][2], lo[NS][2];
+        float r1[NS][4];
+#pragma unroll
+        for (int j = 0; j < NS; ++j)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) hi[j][h] = pack_bf16x2(c[j][2 * h], c[j][2 * h + 1]);
+#pragma unroll
+        for (int j = 0; j < NS; ++j)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            r1[j][2 * h] = c[j][2 * h] - __uint_as_float(hi[j][h] << 16);
+            r1[j][2 * h + 1] = c[j][2 * h + 1] - __uint_as_float(hi[j][h] & 0xffff0000u);
+          }
+#pragma unroll
+        for (int j = 0; j < NS; ++j)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) mid[j][h] = pack_bf16x2(r1[j][2 * h], r1[j][2 * h + 1]);
+#pragma unroll
+        for (int j = 0; j < NS; ++j)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            r1[j][2 * h] -= __uint_as_float(mid[j][h] << 16);
+            r1[j][2 * h + 1] -= __uint_as_float(mid[j][h] & 0xffff0000u);
+          }
+#pragma unroll
+        for (int j = 0; j < NS; ++j)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) lo[j][h] = pack_bf16x2(r1[j][2 * h], r1[j][2 * h + 1]);
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+          float t = fmaf(rv.x, c[j][0], bacc[j]);
+          t = fmaf(rv.y, c[j][1], t);
+          t = fmaf(rv.z, c[j][2], t);
+          t = fmaf(rv.w, c[j][3], t);
+          bacc[j] = (vmask & (1u << j)) ? t : 0.f;
+        }
+        if (turn_o > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_op_empty[o]), (turn_o - 1) & 1, deadline));
+        if (!ok) break;
+        uint8_t *op = ops_ptr + (size_t)o * op_bytes;
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+          if (vmask & (1u << j)) {
+            *reinterpret_cast<uint2 *>(op + dst_h[j]) = make_uint2(hi[j][0], hi[j][1]);
+            *reinterpret_cast<uint2 *>(op + dst_m[j]) = make_uint2(mid[j][0], mid[j][1]);
+            *reinterpret_cast<uint2 *>(op + dst_l[j]) = make_uint2(lo[j][0], lo[j][1]);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads these bytes through the async proxy
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bar_op_full[o]));
+        if (++o == p.nops) { o = 0; ++turn_o; }
+        if (++since_flush == kFlushBlocks) {
+          since_flush = 0;
+#pragma unroll
+          for (int j = 0; j < NS; ++j) { bsum[j] += (double)bacc[j]; bacc[j] = 0.f; }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
+      if (++s == p.stages) { s = 0; full_parity ^= 1u; }
+    }
+    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+#pragma unroll
+    for (int j = 0; j < NS; ++j) bred[ct * NS + j] = bsum[j] + (double)bacc[j];
+    asm volatile("bar.sync 2, %0;" ::"r"(kConvThreads) : "memory");        // the converter warps only
+    if (ct < m) {
+      // row i was shared by the 16 threads ((i % kConvRows) * 16 + q), slot i / kConvRows: add them in q order
+      double v = 0.0;
+      const int t0 = (ct % kConvRows) * 16, j = ct / kConvRows;
+#pragma unroll
+      for (int qq = 0; qq < 16; ++qq) v += bred[(t0 + qq) * NS + j];
+      bpart[(size_t)blockIdx.x * 64 + ct] = v;
+    }
+  } else {
+    // ---------------- accumulator read-back: TMEM chunks -> fp32 registers -> partial D ----------------
+    const int dw = warp - (2 + kConvWarps);          // 0..7; the first read-back warp's index is a multiple of 4, so warp % 4 == dw % 4
+    const int lg = dw & 3;                           // TMEM lane group this warp may read
+    const int half = dw >> 2;                        // pieces of 16 columns: this warp takes piece 2 pp + half
+    const int row = lg * 32 + lane;
+    const int nchunks = (nsb + p.drain - 1) / p.drain;
+    constexpr int kPieces = kMaxN / 32;              // 6 pieces of 16 columns per warp
+    float accr[kPieces * 16];
+#pragma unroll
+    for (int j = 0; j < kPieces * 16; ++j) accr[j] = 0.f;
+    bool ok = true;
+    for (int c = 0; c < nchunks && ok; ++c) {
+      const int buf = c & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_acc_full[buf]), (c >> 1) & 1, deadline));
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+      for (int pp = 0; pp < kPieces; ++pp) {
+        const int piece = 2 * pp + half;
+        if (piece * 16 < p.npad) {
+          uint32_t v[16];
+          const uint32_t taddr = tmem_acc + (uint32_t)buf * 256u + ((uint32_t)(lg * 32) << 16) + (uint32_t)(piece * 16);
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+              "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+                "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+                "=r"(v[14]), "=r"(v[15])
+              : "r"(taddr) : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 16; ++j) accr[pp * 16 + j] += __uint_as_float(v[j]);
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+    }
+    if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+    if (row < 2 * m) {
+      float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.npad;
+#pragma unroll
+      for (int pp = 0; pp < kPieces; ++pp) {
+        const int piece = 2 * pp + half;
+        if (piece * 16 < p.npad) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4 *>(dst + piece * 16 + j) =
+                make_float4(accr[pp * 16 + j], accr[pp * 16 + j + 1], accr[pp * 16 + j + 2], accr[pp * 16 + j + 3]);
+        }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(512u) : "memory");
+  }
+}
+
+// Sum of the per-CTA partial D over the CTAs, in index order, in fp64: block a adds row a
+// (192 columns x 4 ranges of CTAs, the four range sums then added in range order) and, for
+// a < m, b_a.  The block that takes the last ticket forms G from the summed rows (the eight
+// term products listed at the top of this file), writes (G, b) and takes the step's decisions.
+constexpr int kCombThreads = 768;
+__global__ void __launch_bounds__(kCombThreads)
+umma_f32_combine_kernel(const float *__restrict__ partials, const double *__restrict__ bpart, int ctas, int npad,
+                        int m, double *__restrict__ dsum, double *__restrict__ gram, int *__restrict__ status,
+                        const CdgTail tail) {
+  __shared__ double scan_sh[4 * 64 + 64 * 64];     // m <= 64 on this path
+  __shared__ double part[4][kMaxN];
+  __shared__ int is_last;
+  cdg_grid_dep_wait();            // the partials come from the launch before this one
+  const int a = blockIdx.x;
+  const int col = threadIdx.x % kMaxN, qr = threadIdx.x / kMaxN;
+  if (col < npad) {
+    const int c_lo = ctas * qr / 4, c_hi = ctas * (qr + 1) / 4;
+    const float *P = partials + (size_t)a * npad + col;
+    const size_t cs = (size_t)128 * npad;
+    double v = 0.0;
+    int c = c_lo;
+    for (; c + 8 <= c_hi; c += 8) {
+      float x[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) x[u] = P[(size_t)(c + u) * cs];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v += (double)x[u];
+    }
+    for (; c < c_hi; ++c) v += (double)P[(size_t)c * cs];
+    part[qr][col] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < npad)
+    dsum[(size_t)a * kMaxN + threadIdx.x] =
+        ((part[0][threadIdx.x] + part[1][threadIdx.x]) + part[2][threadIdx.x]) + part[3][threadIdx.x];
+  if (a < m && threadIdx.x >= kCombThreads - 32) {
+    // b_a: lane l adds the CTAs l, l + 32, ... in that order, then a fixed butterfly
+    const int lane = threadIdx.x & 31;
+    double v = 0.0;
+    for (int c = lane; c < ctas; c += 32) v += bpart[(size_t)c * 64 + a];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    if (lane == 0) gram[(size_t)m * m + a] = v;
+  }
+
+  // ---- the block that takes the last ticket has every summed row before it ----
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(tail.ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const ScanSmem S = scan_smem(scan_sh, m);
+  for (int e = threadIdx.x; e < m * m; e += kCombThreads) {
+    const int k = e / m, i = e % m;
+    const double *Dk = dsum + (size_t)k * kMaxN, *Dmk = dsum + (size_t)(m + k) * kMaxN;
+    const double hh = __ldcg(Dk + i), hm = __ldcg(Dk + m + i), hl = __ldcg(Dk + 2 * m + i);
+    const double mh = __ldcg(Dmk + i), mm = __ldcg(Dmk + m + i), ml = __ldcg(Dmk + 2 * m + i);
+    const double lh = __ldcg(dsum + (size_t)i * kMaxN + 2 * m + k), lm = __ldcg(dsum + (size_t)(m + i) * kMaxN + 2 * m + k);
+    // smallest terms first
+    const double v = ((((ml + lm) + (hl + lh)) + mm) + (hm + mh)) + hh;
+    S.g[e] = v;
+    gram[e] = v;
+  }
+  for (int j = threadIdx.x; j < m; j += kCombThreads) S.t[j] = __ldcg(gram + (size_t)m * m + j);
+  if (threadIdx.x == 0) *tail.ticket = 0u;                    // ready for the next launch
+  if (!tail.enabled) return;
+  scan_load_pairs(S, tail.perm_cur, m, tail.n, tail.k);
+  __syncthreads();
+  scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
+                        tail.rule);
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D fp32 map over `rows` rows of d columns, box [box_rows][cols], no swizzle; columns past d read as zeros
+bool encode_f32(CUtensorMap *map, const void *base, long long d, int rows, int box_rows, int cols) {
+  EncodeFn fn = (EncodeFn)cdg_tensor_map_encoder();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)d * 4};
+  cuuint32_t box[2] = {(cuuint32_t)cols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NS>
+cudaError_t f32_launch(cdgrab_ctx *h, const CUtensorMap &tm_g, const F32Params &p, cudaStream_t st) {
+  return cdg_launch_dep(h, gram_umma_f32_kernel<NS>, dim3(h->f32_ctas), dim3(kThreads), h->f32_smem, st, tm_g, h->tm_f32r,
+                        p, h->umma_partials, h->f32_bpart, h->status);
+}
+
+cudaError_t f32_open_limits() {
+  cudaError_t e = cdg_open_smem_limit(gram_umma_f32_kernel<1>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<2>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<3>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<4>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<5>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<6>);
+  return e;
+}
+
+}  // namespace
+
+bool cdg_umma_f32_supported(int m, long long d) {
+  // rows whose pitch is a multiple of 16 bytes; 2m <= 128 rows of hi and mid terms fill the MMA's M
+  return m >= 1 && m <= 64 && d % 4 == 0 && d >= 4096 && d < (1ll << 31) - 512 && cdg_tensor_map_encoder() != nullptr;
+}
+
+int cdg_umma_f32_setup(cdgrab_ctx *h) {
+  const int m = h->m;
+  h->f32_npad = ((3 * m + 15) / 16) * 16;
+  const int rows8 = (2 * m + 7) & ~7;
+  const int op_rows = h->f32_npad > 128 ? h->f32_npad : 128;
+  const size_t op_bytes = (size_t)op_rows * 128;
+  // stage width: 128 columns (512 contiguous bytes per row and copy) while two such stages fit beside
+  // three operand buffers, else 64; CDGRAB_F32_NSUB overrides
+  int nsub = 2, nops = 3;
+  if (const char *e = getenv("CDGRAB_F32_NSUB")) {
+    const int v = atoi(e);
+    if (v == 1 || v == 2 || v == 4) nsub = v;
+  }
+  if (const char *e = getenv("CDGRAB_F32_NOPS")) {
+    const int v = atoi(e);
+    if (v >= 2 && v <= kMaxOps) nops = v;
+  }
+  const size_t budget = (size_t)kCdgMaxDynSmem - 1024 - 12 * 1024;   // static shared memory: barriers and the b sums
+  size_t stage_bytes = (size_t)(rows8 + 1) * nsub * kBlockCols * 4;
+  while (nsub > 1 && budget < nops * op_bytes + 2 * stage_bytes) {
+    nsub >>= 1;
+    stage_bytes = (size_t)(rows8 + 1) * nsub * kBlockCols * 4;
+  }
+  int stages = (int)((budget - nops * op_bytes) / stage_bytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (const char *e = getenv("CDGRAB_F32_STAGES")) {
+    const int v = atoi(e);
+    if (v >= 2 && v < stages) stages = v;
+  }
+  if (stages < 2) return CDGRAB_ERR_INVALID;
+  h->f32_nsub = nsub;
+  h->f32_nops = nops;
+  h->f32_stages = stages;
+  h->f32_smem = 1024 + nops * op_bytes + stages * stage_bytes;
+  // TMEM chunk: about 512 columns (fp32 inputs are held to the 1e-6 sign tolerance); CDGRAB_UMMA_DRAIN overrides
+  h->f32_drain = 512 / kBlockCols;
+  if (const char *e = getenv("CDGRAB_UMMA_DRAIN")) {
+    const int v = atoi(e);
+    if (v >= 1 && v <= (1 << 20)) h->f32_drain = v;
+  }
+  const long long nblk = (h->d + kBlockCols - 1) / kBlockCols;
+  h->f32_ctas = (int)(nblk < h->num_sms ? nblk : h->num_sms);
+  const size_t pbytes = sizeof(float) * 128 * (size_t)h->f32_npad * h->f32_ctas;
+  if (cudaMalloc(&h->umma_partials, pbytes) != cudaSuccess ||
+      cudaMalloc(&h->f32_bpart, sizeof(double) * 64 * (size_t)h->f32_ctas) != cudaSuccess ||
+      cudaMalloc(&h->f32_dsum, sizeof(double) * 128 * kMaxN) != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_NOMEM;
+  }
+  if (cudaMemset(h->umma_partials, 0, pbytes) != cudaSuccess ||
+      cudaMemset(h->f32_bpart, 0, sizeof(double) * 64 * (size_t)h->f32_ctas) != cudaSuccess ||
+      cudaMemset(h->f32_dsum, 0, sizeof(double) * 128 * kMaxN) != cudaSuccess)
+    return CDGRAB_ERR_CUDA;
+  if (!encode_f32(&h->tm_f32r, h->r, h->d, 1, 1, nsub * kBlockCols)) return CDGRAB_ERR_CUDA;
+  if (f32_open_limits() != cudaSuccess) {
+    cudaGetLastError();
+    return CDGRAB_ERR_CUDA;
+  }
+  h->umma_fused = h->shard ? 0 : 1;      // a shard's decisions wait for the sum over shards
+  if (const char *e = getenv("CDGRAB_UMMA_FUSE_TAIL")) {
+    if (atoi(e) == 0) h->umma_fused = 0;
+  }
+  h->umma_f32 = 1;
+  return CDGRAB_OK;
+}
+
+void cdg_umma_f32_teardown(cdgrab_ctx *h) {
+  cudaFree(h->f32_bpart);
+  cudaFree(h->f32_dsum);
+  h->f32_bpart = nullptr;
+  h->f32_dsum = nullptr;
+}
+
+cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  int slot = h->tm_f32g.find(grads);
+  if (slot < 0) {
+    slot = h->tm_f32g.victim();
+    if (!encode_f32(&h->tm_f32g.maps[slot][0], grads, h->d, 2 * h->m, 8, h->f32_nsub * kBlockCols))
+      return cudaErrorInvalidValue;
+    h->tm_f32g.commit(slot, grads);
+  }
+  F32Params p;
+  p.m = h->m;
+  p.npad = h->f32_npad;
+  p.nsub = h->f32_nsub;
+  p.stages = h->f32_stages;
+  p.nops = h->f32_nops;
+  p.drain = h->f32_drain;
+  p.nblk = (h->d + kBlockCols - 1) / kBlockCols;
+  {
+    CdgProfScope ps(h, CDGRAB_K_GRAM, st);
+    const CUtensorMap &tm = h->tm_f32g.maps[slot][0];
+    const int ns = (h->m + kConvRows - 1) / kConvRows;       // rows per converter thread
+    static_assert(kRowSlots <= 6, "one instantiation per slot count");
+    switch (ns) {
+      case 1: f32_launch<1>(h, tm, p, st); break;
+      case 2: f32_launch<2>(h, tm, p, st); break;
+      case 3: f32_launch<3>(h, tm, p, st); break;
+      case 4: f32_launch<4>(h, tm, p, st); break;
+      case 5: f32_launch<5>(h, tm, p, st); break;
+      default: f32_launch<6>(h, tm, p, st); break;
+    }
+  }
+  {
+    CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
+    cdg_launch_dep(h, umma_f32_combine_kernel, dim3(2 * h->m), dim3(kCombThreads), 0, st,
+                   (const float *)h->umma_partials, (const double *)h->f32_bpart, h->f32_ctas, h->f32_npad, h->m,
+                   h->f32_dsum, h->gram, h->status, cdg_tail_of(h, h->umma_fused));
+  }
+  return cudaGetLastError();
+}
