@@ -176,7 +176,11 @@ int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, vo
  * The result is bit-identical to `count` calls of cdgrab_step on the slices (greedy rule of
  * Algorithm 6).  On the single-launch path (small steps) the steps run inside one kernel launch
  * and the running sum never leaves the SM's caches between them; on the other paths the call
- * loops over cdgrab_step.  CDGRAB_ERR_STATE if fewer than `count` steps remain in the epoch
+ * loops over cdgrab_step.  With the environment variable CDGRAB_DEFER=1 at create time, handles
+ * on the two-pass FMA path with long rows (m <= 16, d >= 65536) instead let pass 1 of step j
+ * apply the running-sum update of step j-1 (Algorithm 6's r <- r + s c, deferred by one step):
+ * count + 1 streaming launches and one read of r per step, same bits; measured slower than the
+ * loop, hence off by default.  CDGRAB_ERR_STATE if fewer than `count` steps remain in the epoch
  * (nothing is done then); CDGRAB_ERR_INVALID on a shard handle or count < 1.  Asynchronous on
  * `stream` like cdgrab_step.
  */

@@ -365,6 +365,23 @@ int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream
     h->k += count;
     return CDGRAB_OK;
   }
+  // Deferred update (TMA-fed FMA path): pass 1 of step j also applies the update step j - 1 left
+  // open, so the call takes count + 1 streaming launches instead of 2 count and reads r once per
+  // step; only the last step's update gets a launch of its own.
+  if (count > 1 && h->path == CDGRAB_PATH_FMA && h->fma_tma && h->fma_tma_fused && h->fma_tma_defer &&
+      !h->independent && !h->rule_randomized && !h->mean_out) {
+    cudaStream_t st = (cudaStream_t)stream;
+    const char *g = (const char *)grads_dev;
+    cudaError_t e = cdg_launch_gram_fma_tma(h, g, st);
+    for (int i = 1; i < count && e == cudaSuccess; ++i) {
+      h->k++;                               // the step whose decisions this launch takes
+      e = cdg_launch_gram_fma_tma_deferred(h, g + (size_t)i * step_bytes, g + (size_t)(i - 1) * step_bytes, st);
+    }
+    if (e == cudaSuccess) e = cdg_launch_update(h, g + (size_t)(count - 1) * step_bytes, st);
+    if (e != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+    h->k++;
+    return CDGRAB_OK;
+  }
   for (int i = 0; i < count; ++i) {
     const int rc = cdgrab_step(h, (const char *)grads_dev + (size_t)i * step_bytes, stream);
     if (rc != CDGRAB_OK) return rc;

@@ -787,7 +787,15 @@ struct FtTree {
   unsigned long long *group_ctr;       // [groups] arrivals, monotonic
   unsigned long long *top_ctr;         // [1] finished groups, monotonic
   double *group_partials;              // [groups][NACC]
-  float *r;                            // whole-step mode: the running sum, updated in place
+  float *r;                            // whole-step and deferred-update modes: the running sum, updated in place
+  // Deferred update: this launch first applies the update of the step BEFORE (whose signs are
+  // known by now) to every tile of r it streams -- r <- r + sum_i s_i (z1_i - z2_i) over that
+  // step's rows, which travel in the same stage -- stores the new r, and forms this step's Gram
+  // matrix and b from it.  One read of r per step is saved and pass 2 of all but the last step of a
+  // call needs no launch of its own.
+  int fuse_prev;
+  const int8_t *prev_signs;            // signs of the step before: prev_signs[i * prev_stride]
+  int prev_stride;
 };
 
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long *p) {
@@ -803,9 +811,9 @@ template <> struct FtAcc<float> { typedef double type; };        // fp32 rows: o
 // All 2m values of the column are fetched before the first add, so the only serial part is the
 // chain of m additions.
 template <typename T, int M>
-__device__ __forceinline__ void ft_update_tile(const T *gt, const float *rt, const float *ssh, int m, int col,
-                                               long long gcol, long long d, float *__restrict__ r) {
-  if (gcol >= d) return;
+__device__ __forceinline__ float ft_update_tile(const T *gt, const float *rt, const float *ssh, int m, int col,
+                                                long long gcol, long long d, float *__restrict__ r) {
+  if (gcol >= d) return 0.f;
   float c[M];
 #pragma unroll
   for (int i = 0; i < M; ++i) {
@@ -817,13 +825,15 @@ __device__ __forceinline__ void ft_update_tile(const T *gt, const float *rt, con
 #pragma unroll
   for (int i = 0; i < M; ++i)
     if (i < m) acc += (typename FtAcc<T>::type)c[i];
-  r[gcol] = (float)acc;
+  const float out = (float)acc;
+  r[gcol] = out;
+  return out;
 }
 
 template <typename T, int M>
 __global__ void __launch_bounds__(kFtThreads, 1)
 gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
-                    int m, long long d, int stages, int box_rows, int contiguous,
+                    const __grid_constant__ CUtensorMap tm_p, int m, long long d, int stages, int box_rows, int contiguous,
                     double *__restrict__ partials, int *__restrict__ status, const FtTail tail, const FtTree tree) {
   extern __shared__ uint8_t ft_smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kFtMaxStages];
@@ -844,7 +854,9 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   const int nbox = (2 * m + box_rows - 1) / box_rows;             // row boxes per tile
   const uint32_t box_bytes = (uint32_t)box_rows * kFtCols * (uint32_t)sizeof(T);
   const uint32_t g_bytes = (uint32_t)nbox * box_bytes;            // rows past 2m are zero-filled
-  const uint32_t stage_bytes = g_bytes + kFtCols * (uint32_t)sizeof(float);   // rows, then the r tile
+  const uint32_t r_bytes = kFtCols * (uint32_t)sizeof(float);
+  // rows, then the r tile, then (deferred update) the rows of the step before
+  const uint32_t stage_bytes = g_bytes + r_bytes + (tree.fuse_prev ? g_bytes : 0u);
   const long long ntiles = (d + kFtCols - 1) / kFtCols;
   // tiles of this CTA: a contiguous range, or every gridDim.x-th tile
   const long long t_lo = contiguous ? ntiles * blockIdx.x / gridDim.x : blockIdx.x;
@@ -869,6 +881,10 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   cdg_grid_dep_wait();      // r is written by the launch before this one
   FT_STAMP(threadIdx.x == 0, 1);
   const long long deadline = clock64() + kCdgWaitCycles;
+  if (tree.fuse_prev) {     // the signs the launch before this one decided
+    if (threadIdx.x < m) ssh[threadIdx.x] = (float)tree.prev_signs[(size_t)threadIdx.x * tree.prev_stride];
+    __syncthreads();
+  }
 
   float acc[Split<M>::NLPAD];
 #pragma unroll
@@ -899,6 +915,8 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
         mbar_expect_tx(full, stage_bytes);
         for (int q = 0; q < nbox; ++q) tma_load_2d(dst + q * box_bytes, &tm_g, col, q * box_rows, full);
         tma_load_2d(dst + g_bytes, &tm_r, col, 0, full);
+        if (tree.fuse_prev)
+          for (int q = 0; q < nbox; ++q) tma_load_2d(dst + g_bytes + r_bytes + q * box_bytes, &tm_p, col, q * box_rows, full);
         issued = it + 1;
         if (++s == stages) { s = 0; ++turn; }
       }
@@ -920,7 +938,14 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       if (!ok) break;
       FT_STAMP(threadIdx.x == 0 && it == 0, 2);
       const T *gt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes);
-      const float *rt = reinterpret_cast<const float *>(base_ptr + (size_t)s * stage_bytes + g_bytes);
+      float *rt = reinterpret_cast<float *>(base_ptr + (size_t)s * stage_bytes + g_bytes);
+      if (tree.fuse_prev && group == 1) {
+        // the update the step before left open, on this thread's column; the new value replaces
+        // the old one in the stage so that b below is formed against it
+        const T *pt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes + g_bytes + r_bytes);
+        const long long gcol = (t_lo + (long long)it * t_step) * kFtCols + col;
+        rt[col] = ft_update_tile<T, M>(pt, rt, ssh, m, col, gcol, d, tree.r);
+      }
       if (group == 0) ft_consume<T, M, 0>(gt, rt, m, col, acc);
       else ft_consume<T, M, 1>(gt, rt, m, col, acc);
       __syncwarp();
@@ -1153,6 +1178,20 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
   if (stages < 2) return CDGRAB_ERR_INVALID;
   h->fma_tma_stages = stages;
   h->fma_tma_smem = stages * stage + 128;
+  // deferred update: a stage also carries the rows of the step before
+  const size_t stage2 = stage + (size_t)nbox * box_rows * kFtCols * esz;
+  int stages2 = (int)((200 * 1024) / stage2);
+  if (stages2 > kFtMaxStages) stages2 = kFtMaxStages;
+  h->fma_tma_stages2 = stages2;
+  h->fma_tma_smem2 = stages2 * stage2 + 128;
+  // CDGRAB_DEFER=1: cdgrab_step_many folds pass 2 of a step into pass 1 of the next one.  Off by
+  // default: measured slower than two launches per step at every size tried (the update's loads and
+  // adds land on the threads that also own b, and a stage holds two steps' rows, so the ring is half
+  // as deep): 91 against 63 us per step at m = 16, d = 2^20 fp32; 723 against 439 us at m = 16,
+  // d = 13.5 M bf16.
+  h->fma_tma_defer = 0;
+  if (const char *e = getenv("CDGRAB_DEFER")) h->fma_tma_defer = atoi(e) ? 1 : 0;
+  if (stages2 < 2) h->fma_tma_defer = 0;
   const long long ntiles = (h->d + kFtCols - 1) / kFtCols;
   h->gram_chunks = (int)(ntiles < h->num_sms ? ntiles : h->num_sms);
   if (!ft_encode(&h->tm_fr, h->r, h->d, 1, 1, 4)) return CDGRAB_ERR_CUDA;
@@ -1195,10 +1234,11 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
 }
 
 template <typename T, int M>
-static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g, cudaStream_t st) {
+static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g, const CUtensorMap *tm_prev,
+                                         cudaStream_t st) {
   const FtTail tail = cdg_tail_of(h, h->fma_tma_fused);
   // the whole step in this launch unless something has to happen between the passes' launches
-  const int whole = h->fma_tma_whole && h->fma_tma_fused && !h->mean_out && !h->shard;
+  const int whole = !tm_prev && h->fma_tma_whole && h->fma_tma_fused && !h->mean_out && !h->shard;
   FtTree tree;
   tree.whole = whole;
   tree.gsize = h->ft_gsize;
@@ -1207,12 +1247,18 @@ static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g,
   tree.top_ctr = h->ft_ctr + kFtMaxGroups;
   tree.group_partials = h->ft_group_partials;
   tree.r = h->r;
+  tree.fuse_prev = tm_prev ? 1 : 0;
+  tree.prev_signs = tm_prev ? h->signs + (h->k - 1) : nullptr;
+  tree.prev_stride = h->n / 2;
+  const int stages = tm_prev ? h->fma_tma_stages2 : h->fma_tma_stages;
+  const size_t smem = tm_prev ? h->fma_tma_smem2 : h->fma_tma_smem;
+  const CUtensorMap &tm_p = tm_prev ? *tm_prev : tm_g;
   h->ft_whole_launched = whole;
   {
-    CdgProfScope ps(h, whole ? CDGRAB_K_FUSED : CDGRAB_K_GRAM, st);
+    CdgProfScope ps(h, (whole || tm_prev) ? CDGRAB_K_FUSED : CDGRAB_K_GRAM, st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(h->gram_chunks); cfg.blockDim = dim3(kFtThreads);
-    cfg.dynamicSmemBytes = h->fma_tma_smem; cfg.stream = st;
+    cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute at[2];
     int na = 0;
     if (whole && h->ft_coop) {   // its CTAs wait on one another: all of them must be resident
@@ -1226,14 +1272,14 @@ static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g,
       ++na;
     }
     cfg.attrs = at; cfg.numAttrs = na;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, h->m, h->d, h->fma_tma_stages,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, tm_p, h->m, h->d, stages,
                                        h->fma_tma_boxrows, h->fma_tma_contig, h->partials, h->status, tail, tree);
     if (e != cudaSuccess && whole && h->ft_coop && na == 2) {
       // a driver that does not take both attributes together: cooperative alone from now on
       cudaGetLastError();
       h->ft_coop_no_pdl = 1;
       cfg.numAttrs = 1;
-      e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, h->m, h->d, h->fma_tma_stages,
+      e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, tm_p, h->m, h->d, stages,
                              h->fma_tma_boxrows, h->fma_tma_contig, h->partials, h->status, tail, tree);
     }
     if (e != cudaSuccess) return e;
@@ -1245,22 +1291,46 @@ static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g,
   return cudaGetLastError();
 }
 
-cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+// the tensor map over the 2m rows at `grads` (from the cache of the last few bases, or encoded now)
+static const CUtensorMap *ft_map_of(cdgrab_ctx *h, const void *grads) {
   int slot = h->tm_fg.find(grads);
   if (slot < 0) {
     slot = h->tm_fg.victim();
     if (!ft_encode(&h->tm_fg.maps[slot][0], grads, h->d, 2 * h->m, h->fma_tma_boxrows, h->dtype == CDGRAB_F32 ? 4 : 2))
-      return cudaErrorInvalidValue;
+      return nullptr;
     h->tm_fg.commit(slot, grads);
   }
-  const CUtensorMap &tm = h->tm_fg.maps[slot][0];
+  return &h->tm_fg.maps[slot][0];
+}
+
+// grads_prev != NULL: the launch also applies the update of the step before, whose rows lie there
+static cudaError_t ft_dispatch(cdgrab_ctx *h, const void *grads, const void *grads_prev, cudaStream_t st) {
+  CUtensorMap prev_copy;
+  const CUtensorMap *tp = nullptr;
+  if (grads_prev) {
+    const CUtensorMap *q = ft_map_of(h, grads_prev);
+    if (!q) return cudaErrorInvalidValue;
+    prev_copy = *q;                       // the cache entry may be replaced by the next look-up
+    tp = &prev_copy;
+  }
+  const CUtensorMap *tg = ft_map_of(h, grads);
+  if (!tg) return cudaErrorInvalidValue;
+  const CUtensorMap &tm = *tg;
   const int M = pick_M(h->m);
   if (h->dtype == CDGRAB_F32) {
-    if (M == 4) return launch_gram_fma_tma_t<float, 4>(h, tm, st);
-    if (M == 8) return launch_gram_fma_tma_t<float, 8>(h, tm, st);
-    return launch_gram_fma_tma_t<float, 16>(h, tm, st);
+    if (M == 4) return launch_gram_fma_tma_t<float, 4>(h, tm, tp, st);
+    if (M == 8) return launch_gram_fma_tma_t<float, 8>(h, tm, tp, st);
+    return launch_gram_fma_tma_t<float, 16>(h, tm, tp, st);
   }
-  if (M == 4) return launch_gram_fma_tma_t<__nv_bfloat16, 4>(h, tm, st);
-  if (M == 8) return launch_gram_fma_tma_t<__nv_bfloat16, 8>(h, tm, st);
-  return launch_gram_fma_tma_t<__nv_bfloat16, 16>(h, tm, st);
+  if (M == 4) return launch_gram_fma_tma_t<__nv_bfloat16, 4>(h, tm, tp, st);
+  if (M == 8) return launch_gram_fma_tma_t<__nv_bfloat16, 8>(h, tm, tp, st);
+  return launch_gram_fma_tma_t<__nv_bfloat16, 16>(h, tm, tp, st);
+}
+
+cudaError_t cdg_launch_gram_fma_tma(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  return ft_dispatch(h, grads, nullptr, st);
+}
+
+cudaError_t cdg_launch_gram_fma_tma_deferred(cdgrab_ctx *h, const void *grads, const void *grads_prev, cudaStream_t st) {
+  return ft_dispatch(h, grads, grads_prev, st);
 }

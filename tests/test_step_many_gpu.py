@@ -25,9 +25,18 @@ def epoch(m, n, d, dtype, seed):
     (8, 16, 4096, "f32", "fused"),
     (16, 8, 2048, "bf16", "fused"),
     (3, 10, 516, "f32", "fused"),
-    (8, 6, 200_000, "f32", "fma"),       # two-pass path: the call loops over single steps
+    (8, 6, 200_000, "f32", "fma"),       # two-pass path, TMA-fed pass 1: the call loops over single steps, or
+    (16, 8, 1 << 18, "f32", "fma"),      # (CDGRAB_DEFER=1) the update of a step rides in the next step's pass 1
+    (16, 8, 300_008, "bf16", "fma"),
+    (4, 6, 70_000, "f32", "fma"),
+    (3, 12, 65_540, "bf16", "fma"),
+    (8, 6, 40_000, "f32", "fma"),        # short rows: register-load pass 1, the call loops over single steps
 ])
-def test_many_equals_single_steps_and_oracle(m, n, d, dtype, path):
+@pytest.mark.parametrize("defer", ["0", "1"])
+def test_many_equals_single_steps_and_oracle(m, n, d, dtype, path, defer, monkeypatch):
+    if defer == "1" and (path != "fma" or d < 65536):
+        pytest.skip("the deferred update exists on the TMA-fed two-pass path only")
+    monkeypatch.setenv("CDGRAB_DEFER", defer)
     g = epoch(m, n, d, dtype, 5 + m)
     with binding.CdGrab(m, n, d, dtype) as a, binding.CdGrab(m, n, d, dtype) as b:
         assert a.path == path
@@ -57,6 +66,25 @@ def test_many_equals_single_steps_and_oracle(m, n, d, dtype, path):
         finally:
             cpu.close()
         assert a.status() == binding.OK
+
+
+def test_deferred_update_launch_count_and_switch(monkeypatch):
+    """With CDGRAB_DEFER=1, count steps in one call take count + 1 streaming launches on the TMA-fed
+    path; by default the call loops over single steps (2 launches each).  Same bits either way."""
+    m, n, d = 8, 12, 131_072
+    g = epoch(m, n, d, "f32", 77)
+    out = {}
+    for defer in ("1", "0"):
+        monkeypatch.setenv("CDGRAB_DEFER", defer)
+        with binding.CdGrab(m, n, d, "f32") as h:
+            h.begin_epoch()
+            before = h.launch_count
+            h.step_many(g)
+            out[defer] = (h.launch_count - before, h.signs().clone(), h.r().clone(), h.next_perms().clone())
+            assert h.status() == binding.OK
+    assert out["1"][0] == n // 2 + 1 and out["0"][0] == 2 * (n // 2)
+    for a, b in zip(out["1"][1:], out["0"][1:]):
+        assert torch.equal(a, b)
 
 
 def test_many_rejects_more_steps_than_the_epoch_has():
