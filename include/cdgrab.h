@@ -58,7 +58,8 @@ enum {
   CDGRAB_PATH_FUSED = 1, /* one launch per step, whole step on chip (small d)            */
   CDGRAB_PATH_FMA = 2,   /* two passes, Gram matrix on the fp32 FMA pipe                 */
   CDGRAB_PATH_UMMA = 3,  /* two passes, Gram matrix on tcgen05 tensor cores (bf16)       */
-  CDGRAB_PATH_INDEPENDENT = 4 /* ID-GraB mode: one running sum per worker (see below)     */
+  CDGRAB_PATH_INDEPENDENT = 4, /* ID-GraB mode: one running sum per worker (see below)    */
+  CDGRAB_PATH_LITERAL = 5 /* one launch per step, Algorithm 6 worker by worker (short rows) */
 };
 
 /*
@@ -174,8 +175,8 @@ int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, vo
  * staged ahead (a whole epoch of a small problem): grads_dev is DEVICE memory laid out
  * [count][2][m][d] in the handle's dtype, 16-byte aligned, step j at offset j*2*m*d elements.
  * The result is bit-identical to `count` calls of cdgrab_step on the slices (greedy rule of
- * Algorithm 6).  On the single-launch path (small steps) the steps run inside one kernel launch
- * and the running sum never leaves the SM's caches between them; on the other paths the call
+ * Algorithm 6).  On the single-launch paths (small steps) the steps run inside one kernel launch
+ * and the running sum never leaves the SM between them; on the other paths the call
  * loops over cdgrab_step.  With the environment variable CDGRAB_DEFER=1 at create time, handles
  * on the two-pass FMA path with long rows (m <= 16, d >= 65536) instead let pass 1 of step j
  * apply the running-sum update of step j-1 (Algorithm 6's r <- r + s c, deferred by one step):
@@ -247,7 +248,7 @@ int cdgrab_save_state(cdgrab_t *h, void *host_buf, long long bytes);
 int cdgrab_load_state(cdgrab_t *h, const void *host_buf, long long bytes);
 
 /* Code path the handle uses (CDGRAB_PATH_*).  The environment variable
- * CDGRAB_FORCE_PATH = fused | fma | umma, read at create time, overrides the automatic
+ * CDGRAB_FORCE_PATH = fused | fma | umma | literal, read at create time, overrides the automatic
  * choice when the forced path supports the shape; otherwise create fails with
  * CDGRAB_ERR_INVALID. */
 int cdgrab_path(const cdgrab_t *h);
@@ -296,7 +297,8 @@ int cdgrab_logreg_grads(cdgrab_t *h, const float *X, const float *y, const float
  *   c_i = (sigma(<w,x_p>) - y_p) x_p - (sigma(<w,x_q>) - y_q) x_q,  p, q = perm_cur[i][2k], [2k+1]
  * (each product rounded to fp32 as a stored gradient would be).  Same arguments as
  * cdgrab_logreg_grads minus the output; X and w 16-byte aligned.  Only for fp32 handles small
- * enough for the single-launch path (cdgrab_path == CDGRAB_PATH_FUSED), else CDGRAB_ERR_INVALID.
+ * enough for a single-launch path (cdgrab_path == CDGRAB_PATH_FUSED, or CDGRAB_PATH_LITERAL with
+ * m <= 16), else CDGRAB_ERR_INVALID.
  * Counts as one balancing step.  Asynchronous on `stream`.
  */
 int cdgrab_step_logreg(cdgrab_t *h, const float *X, const float *y, const float *w, void *stream);

@@ -20,7 +20,7 @@ ERR_INVALID, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_NONFINITE, ERR_TIMEOUT, ERR_DEV
 ERR_TOO_LARGE = -8
 PATH_AUTO, PATH_FUSED, PATH_FMA, PATH_UMMA = 0, 1, 2, 3
 KERNEL_KINDS = ("gram", "combine", "scan", "update", "fused", "logreg")
-PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma", 4: "independent"}
+PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma", 4: "independent", 5: "literal"}
 
 # name -> (restype, argtypes); the single list of what include/cdgrab.h declares
 SIGNATURES = {

@@ -52,6 +52,7 @@ int forced_path() {
   if (!strcmp(e, "fused")) return CDGRAB_PATH_FUSED;
   if (!strcmp(e, "fma")) return CDGRAB_PATH_FMA;
   if (!strcmp(e, "umma")) return CDGRAB_PATH_UMMA;
+  if (!strcmp(e, "literal")) return CDGRAB_PATH_LITERAL;
   return -1;
 }
 
@@ -134,14 +135,21 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
   const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);
   const bool fused_ok = cdg_fused_supported(m, d, dtype);
   const bool umma_ok = cdg_umma_supported(m, d, dtype);
+  const bool literal_ok = cdg_literal_supported(m, d, dtype) && !shard && !independent;
   int path;
   if (forced == CDGRAB_PATH_AUTO) {
-    if (fused_ok && step_bytes <= (size_t)768 * 1024 && !shard) path = CDGRAB_PATH_FUSED;
+    // short rows: the literal form (one dot product per worker) beats the Gram form of the
+    // single-launch step up to 1024 columns, and the four launches of the generic two-pass route
+    // for more than 16 workers while m*d stays small (measured; the table is in the design notes)
+    if (literal_ok && ((m <= 16 && d <= 1024) || (m > 16 && d < 4096 && (long long)m * d <= 65536)))
+      path = CDGRAB_PATH_LITERAL;
+    else if (fused_ok && step_bytes <= (size_t)768 * 1024 && !shard) path = CDGRAB_PATH_FUSED;
     else if (umma_ok && !fma_columns_ok(h)) path = CDGRAB_PATH_UMMA;
     else path = CDGRAB_PATH_FMA;
   } else {
     path = forced;
-    if ((path == CDGRAB_PATH_FUSED && (!fused_ok || shard)) || (path == CDGRAB_PATH_UMMA && !umma_ok)) {
+    if ((path == CDGRAB_PATH_FUSED && (!fused_ok || shard)) || (path == CDGRAB_PATH_UMMA && !umma_ok) ||
+        (path == CDGRAB_PATH_LITERAL && !literal_ok)) {
       delete h;
       return CDGRAB_ERR_INVALID;
     }
@@ -338,6 +346,8 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
     e = cdg_launch_indep(h, grads_dev, st);
   } else if (h->path == CDGRAB_PATH_FUSED) {
     e = cdg_launch_fused(h, grads_dev, 1, st);
+  } else if (h->path == CDGRAB_PATH_LITERAL) {
+    e = cdg_launch_literal(h, grads_dev, 1, st);
   } else {
     e = launch_pass1(h, grads_dev, st);
     const bool decided = (h->path == CDGRAB_PATH_UMMA) ? h->umma_fused : (h->fma_tma && h->fma_tma_fused);
@@ -382,6 +392,15 @@ int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream
     h->k++;
     return CDGRAB_OK;
   }
+  if (h->path == CDGRAB_PATH_LITERAL && !h->rule_randomized && !h->mean_out) {
+    if (step_bytes % 16 != 0) return CDGRAB_ERR_INVALID;
+    if (cdg_launch_literal(h, grads_dev, count, (cudaStream_t)stream) != cudaSuccess) {
+      cudaGetLastError();
+      return CDGRAB_ERR_CUDA;
+    }
+    h->k += count;
+    return CDGRAB_OK;
+  }
   for (int i = 0; i < count; ++i) {
     const int rc = cdgrab_step(h, (const char *)grads_dev + (size_t)i * step_bytes, stream);
     if (rc != CDGRAB_OK) return rc;
@@ -391,7 +410,10 @@ int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream
 
 int cdgrab_step_logreg(cdgrab_t *h, const float *X, const float *y, const float *w, void *stream) {
   if (!valid(h) || !X || !y || !w) return CDGRAB_ERR_INVALID;
-  if (h->dtype != CDGRAB_F32 || h->path != CDGRAB_PATH_FUSED) return CDGRAB_ERR_INVALID;
+  // the one-launch step from feature rows serves handles on either single-launch path
+  const bool single = h->path == CDGRAB_PATH_FUSED ||
+                      (h->path == CDGRAB_PATH_LITERAL && cdg_fused_supported(h->m, h->d, h->dtype));
+  if (h->dtype != CDGRAB_F32 || !single) return CDGRAB_ERR_INVALID;
   if ((((uintptr_t)X | (uintptr_t)w) & 15) != 0) return CDGRAB_ERR_INVALID;
   if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;
   if (!h->epoch_open || h->k >= h->n / 2) return CDGRAB_ERR_STATE;
@@ -421,8 +443,8 @@ int cdgrab_step_mean(cdgrab_t *h, const void *grads_dev, float *mean_out_dev, vo
   if (((uintptr_t)mean_out_dev & 15) != 0) return CDGRAB_ERR_INVALID;   // written with 16-byte vector stores
   h->mean_out = mean_out_dev;
   int rc = cdgrab_step(h, grads_dev, stream);
-  if (rc == CDGRAB_OK && h->path == CDGRAB_PATH_FUSED) {
-    // the single-launch step has no separate pass 2 to fold the average into
+  if (rc == CDGRAB_OK && (h->path == CDGRAB_PATH_FUSED || h->path == CDGRAB_PATH_LITERAL)) {
+    // the single-launch steps have no separate pass 2 to fold the average into
     if (cdg_launch_mean(h, grads_dev, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); rc = CDGRAB_ERR_CUDA; }
   }
   h->mean_out = nullptr;

@@ -85,7 +85,8 @@ def test_environment_is_read_at_create_time_only():
     """Launch paths run every few microseconds: knobs are read when a handle is created (create_impl
     and the *_setup / *_supported routines it calls), never per step."""
     csrc = os.path.join(ROOT, "paper_2302_00845_b200", "csrc")
-    allowed = ("create_impl", "forced_path", "cdg_fma_tma_setup", "cdg_umma_setup", "cdg_umma_supported")
+    allowed = ("create_impl", "forced_path", "cdg_fma_tma_setup", "cdg_umma_setup", "cdg_umma_supported",
+               "cdg_umma_f32_setup")
     for f in sorted(os.listdir(csrc)):
         src = open(os.path.join(csrc, f)).read()
         for mt in re.finditer(r"getenv\(", src):

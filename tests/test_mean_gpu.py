@@ -17,7 +17,8 @@ def grads(m, d, dtype, seed):
 
 
 @pytest.mark.parametrize("m,d,dtype,path", [
-    (4, 1024, "f32", "fused"),        # single-launch step: separate averaging kernel
+    (4, 1024, "f32", "literal"),      # single-launch steps: separate averaging kernel
+    (8, 4096, "f32", "fused"),
     (16, 100_000, "f32", "fma"),      # TMA-fed Gram, pass 2 with 256-bit loads
     (5, 1023, "f32", "fma"),          # scalar pass 2
     (12, 70_004, "bf16", "fma"),      # 8-column pass 2 (rows not 32-byte aligned)

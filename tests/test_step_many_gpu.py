@@ -21,10 +21,12 @@ def epoch(m, n, d, dtype, seed):
 
 
 @pytest.mark.parametrize("m,n,d,dtype,path", [
-    (4, 64, 1024, "f32", "fused"),       # the tiny workload: a whole epoch in one launch
+    (4, 64, 1024, "f32", "literal"),     # the tiny workload: a whole epoch in one launch
     (8, 16, 4096, "f32", "fused"),
     (16, 8, 2048, "bf16", "fused"),
-    (3, 10, 516, "f32", "fused"),
+    (3, 10, 516, "f32", "literal"),
+    (6, 10, 1028, "f32", "fused"),
+    (40, 6, 64, "bf16", "literal"),
     (8, 6, 200_000, "f32", "fma"),       # two-pass path, TMA-fed pass 1: the call loops over single steps, or
     (16, 8, 1 << 18, "f32", "fma"),      # (CDGRAB_DEFER=1) the update of a step rides in the next step's pass 1
     (16, 8, 300_008, "bf16", "fma"),
