@@ -47,7 +47,10 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
-    ap.add_argument("--workload", default="gpt2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="gpt2", choices=sorted(synth.WORKLOADS) + ["herding"])
+    ap.add_argument("--herding-total", type=int, default=1_000_000, help="vectors of the herding study (all workers)")
+    ap.add_argument("--herding-epochs", type=int, default=4)
+    ap.add_argument("--herding-seeds", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-events", action="store_true",
@@ -62,7 +65,7 @@ def parse_args():
 
 
 def pick_workload(args) -> synth.Workload:
-    wl = synth.WORKLOADS[args.workload]
+    wl = synth.WORKLOADS["tiny" if args.workload == "herding" else args.workload]
     if args.d:
         wl = wl.scaled(d=args.d, name=f"{wl.name}@d={args.d}")
     if args.m:
@@ -583,6 +586,66 @@ def run_native(args):
         dist.destroy_process_group()
 
 
+def run_herding(args):
+    """The paper's synthetic herding study as a workload: N vectors ~ Unif[0,1)^16, centred and
+    normalised, split over m in {5, 10, 20, 50, 100} workers; a few epochs of coordinated
+    PairBalance orders (each epoch staged in HBM and balanced by one cdgrab_step_many call) against
+    random reshuffling, the parallel herding objective (Eq. 7) evaluated on the device after every
+    epoch.  One JSON line: value = balanced examples per second over all PairBalance epochs."""
+    from paper_2302_00845_b200 import binding, build
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    build.build()
+    N, d, E = args.herding_total, 16, args.herding_epochs
+    table, total_ms, total_examples, launches = [], 0.0, 0, 0
+    for m in (5, 10, 20, 50, 100):
+        n = (N // m) & ~1
+        rows = torch.arange(m, device="cuda")[:, None]
+        for seed in range(args.herding_seeds):
+            z = synth.herding_vectors(m * n, d, seed, "cuda").reshape(m, n, d)
+            cur = synth.random_orders(m, n, 1000 * seed, "cuda")
+            pb = [binding.herding_objective(z, cur)]
+            rr = [pb[0]]
+            out = torch.empty(m, n, dtype=torch.int32, device="cuda")
+            ms = []
+            with binding.CdGrab(m, n, d, "f32") as h:
+                h.set_perms(cur.cpu().numpy())
+                for ep in range(E):
+                    # this epoch's gradients in visiting order, staged as [n/2][2][m][d]
+                    g = z[rows, cur.long()].reshape(m, n // 2, 2, d).permute(1, 2, 0, 3).contiguous()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    before = h.launch_count
+                    torch.cuda.synchronize()
+                    e0.record()
+                    h.begin_epoch()
+                    h.step_many(g)
+                    h.end_epoch(out)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    launches += h.launch_count - before
+                    ms.append(e0.elapsed_time(e1))
+                    cur = out.clone()
+                    pb.append(binding.herding_objective(z, cur))
+                    rr.append(binding.herding_objective(z, synth.random_orders(m, n, 1000 * seed + ep + 1, "cuda")))
+                h.check_status()
+                path = h.path
+            total_ms += sum(ms)
+            total_examples += E * m * n
+            table.append({"m": m, "n": n, "seed": seed, "path": path, "pairbalance": pb, "random_reshuffling": rr,
+                          "ms_per_epoch": sum(ms) / E, "us_per_step": 1e3 * sum(ms) / E / (n // 2)})
+    line = {"metric": METRIC, "value": total_examples / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": E * len(table), "warmup": 0, "ms_per_step": total_ms / (E * len(table)), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "herding", "total_vectors": N, "d": d, "epochs": E, "seeds": args.herding_seeds,
+                       "step": "one epoch of PairBalance orders (cdgrab_begin_epoch, cdgrab_step_many over n/2 staged "
+                               "steps, cdgrab_end_epoch)"},
+            "gpu_launches": launches, "herding": table}
+    print(json.dumps(line), flush=True)
+
+
 def run_e2e(h, wl, dev_buf, state, one_step):
     """Same metric through cdgrab_step_host: every step copies its [2][m][d] input from pinned host
     memory and reads the sign table back."""
@@ -626,6 +689,8 @@ def main():
     args = parse_args()
     if args.oracle_child:
         oracle_child(args.oracle_child, args.cpu_seconds)
+    elif args.workload == "herding" and args.impl == "native":
+        run_herding(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

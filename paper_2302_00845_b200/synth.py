@@ -164,6 +164,21 @@ class LogregProblem:
         self.w = torch.randn(wl.d, generator=g0, device=dev) * 0.1
 
 
+def herding_vectors(total: int, d: int = 16, seed: int = 0, device="cpu") -> torch.Tensor:
+    """The vectors of the paper's synthetic herding study (experiment-details appendix, simulated
+    ablation): `total` points uniform in [0,1)^d, zero-centred, then scaled to unit Euclidean norm."""
+    g = _gen(torch.device(device), seed, 0xD44, total, d)
+    z = torch.rand(total, d, generator=g, device=device)
+    z = z - z.mean(dim=0)
+    return (z / z.norm(dim=1, keepdim=True)).contiguous()
+
+
+def random_orders(m: int, n: int, seed: int, device="cpu") -> torch.Tensor:
+    """m independent uniformly random permutations of [0, n) as int32 [m][n] (random reshuffling)."""
+    g = _gen(torch.device(device), seed, 0xE55, m, n)
+    return torch.argsort(torch.rand(m, n, generator=g, device=device), dim=1).to(torch.int32).contiguous()
+
+
 def bf16_bits(t: torch.Tensor):
     """Host numpy view of a bf16 tensor as uint16 bit patterns (what the oracle reads)."""
     import numpy as np

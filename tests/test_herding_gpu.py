@@ -6,7 +6,8 @@ import pytest
 import torch
 
 import oracle
-from paper_2302_00845_b200 import binding
+from paper_2302_00845_b200 import binding, synth
+from parity import Pair
 from test_oracle_pins import load_herding_cases
 
 pytestmark = pytest.mark.gpu
@@ -76,3 +77,55 @@ def test_pairbalance_orders_shrink_the_bound():
     assert history[-1] < 0.25 * start
     want = oracle.herding_objective(z.cpu().numpy(), cur.cpu().numpy())
     assert abs(history[-1] - want) <= 1e-9 * max(1.0, want)
+
+
+def _staged_epoch(z, cur):
+    m, n, d = z.shape
+    rows = torch.arange(m, device="cuda")[:, None]
+    return z[rows, cur.long()].reshape(m, n // 2, 2, d).permute(1, 2, 0, 3).contiguous()
+
+
+@pytest.mark.parametrize("m", [5, 10, 20, 50, 100])
+def test_herding_study_reduced_beats_random_reshuffling(m):
+    """The synthetic study at reduced size (20 000 vectors in R^16): after four epochs the bound of
+    the library's coordinated orders is below that of every random-reshuffling order drawn."""
+    n, d = (20_000 // m) & ~1, 16
+    z = synth.herding_vectors(m * n, d, 7, "cuda").reshape(m, n, d)
+    cur = synth.random_orders(m, n, 70, "cuda")
+    rr = [binding.herding_objective(z, synth.random_orders(m, n, 71 + e, "cuda")) for e in range(4)]
+    out = torch.empty(m, n, dtype=torch.int32, device="cuda")
+    hist = [binding.herding_objective(z, cur)]
+    with binding.CdGrab(m, n, d, "f32") as h:
+        h.set_perms(cur.cpu().numpy())
+        for _ in range(4):
+            h.begin_epoch()
+            h.step_many(_staged_epoch(z, cur))
+            h.end_epoch(out)
+            torch.cuda.synchronize()
+            cur = out.clone()
+            hist.append(binding.herding_objective(z, cur))
+        assert h.status() == binding.OK
+    print(f"m={m}: PairBalance {[round(v, 2) for v in hist]}  random reshuffling {[round(v, 2) for v in rr]}")
+    assert hist[-1] < min(rr)
+    assert hist[-1] < 0.5 * hist[0]
+
+
+def test_herding_study_largest_worker_count_against_the_oracle():
+    """m = 100 workers, short rows: signs, permutations and Eq. (7) of one epoch against the oracle."""
+    m, n, d = 100, 60, 16
+    z = synth.herding_vectors(m * n, d, 3, "cuda").reshape(m, n, d)
+    cur = synth.random_orders(m, n, 30, "cuda")
+    g = _staged_epoch(z, cur)
+    pr = Pair(m, n, d, "f32", perms0=cur.cpu().numpy())
+    try:
+        pr.begin()
+        for k in range(n // 2):
+            pr.step(g[k])
+        rep = pr.end()
+        assert rep.raw_agreement == 1.0
+        got = pr.gpu.perms()
+        want = oracle.herding_objective(z.cpu().numpy(), got.cpu().numpy())
+        dev = binding.herding_objective(z, got)
+        assert abs(dev - want) <= 1e-9 * max(1.0, want)
+    finally:
+        pr.close()
