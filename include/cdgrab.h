@@ -49,7 +49,9 @@ enum {
   CDGRAB_ERR_NONFINITE = -5, /* NaN/Inf met in a reduction (device status word)          */
   CDGRAB_ERR_TIMEOUT = -6,   /* a bounded device-side wait expired (device status word)  */
   CDGRAB_ERR_DEVICE = -7,    /* no usable sm_100 device                                  */
-  CDGRAB_ERR_TOO_LARGE = -8  /* size beyond the fixed scratch of cdgrab_step_noalloc        */
+  CDGRAB_ERR_TOO_LARGE = -8, /* size beyond the fixed scratch of cdgrab_step_noalloc        */
+  CDGRAB_ERR_CORRUPT = -9    /* debug build only: guard bytes around library memory were
+                                overwritten, or an index check in a kernel failed            */
 };
 
 /* Which code path a handle uses (cdgrab_path / CDGRAB_FORCE_PATH). */

@@ -18,6 +18,7 @@ F32, BF16 = 0, 1
 OK = 0
 ERR_INVALID, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_NONFINITE, ERR_TIMEOUT, ERR_DEVICE = -1, -2, -3, -4, -5, -6, -7
 ERR_TOO_LARGE = -8
+ERR_CORRUPT = -9
 PATH_AUTO, PATH_FUSED, PATH_FMA, PATH_UMMA = 0, 1, 2, 3
 KERNEL_KINDS = ("gram", "combine", "scan", "update", "fused", "logreg")
 PATH_NAMES = {PATH_FUSED: "fused", PATH_FMA: "fma", PATH_UMMA: "umma", 4: "independent", 5: "literal"}

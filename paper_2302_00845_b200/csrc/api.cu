@@ -31,13 +31,13 @@ __global__ void iota_perm_kernel(int32_t *p, int m, int n) {
 
 void free_all(cdgrab_ctx *h) {
   cdg_umma_teardown(h);
-  cudaFree(h->r); cudaFree(h->perm_cur); cudaFree(h->perm_next); cudaFree(h->signs);
-  cudaFree(h->margins); cudaFree(h->rnorm2); cudaFree(h->status); cudaFree(h->gram);
-  cudaFree(h->partials);
-  cudaFree(h->ticket);
-  cudaFree(h->ft_ctr);
-  cudaFree(h->ft_group_partials);
-  cudaFree(h->oob);
+  cdg_free(h->r); cdg_free(h->perm_cur); cdg_free(h->perm_next); cdg_free(h->signs);
+  cdg_free(h->margins); cdg_free(h->rnorm2); cdg_free(h->status); cdg_free(h->gram);
+  cdg_free(h->partials);
+  cdg_free(h->ticket);
+  cdg_free(h->ft_ctr);
+  cdg_free(h->ft_group_partials);
+  cdg_free(h->oob);
   if (h->prof_ev) {
     for (int i = 0; i < 2 * h->prof_cap; ++i) if (h->prof_ev[i]) cudaEventDestroy(h->prof_ev[i]);
     free(h->prof_ev);
@@ -69,6 +69,39 @@ int copy_out(void *dst, const void *src, size_t bytes, void *stream) {
 
 }  // namespace
 
+int cdg_first_broken_guard(const cdgrab_ctx *h) {
+#ifdef CDGRAB_DEBUG
+  unsigned char buf[2 * kCdgGuardBytes];
+  for (int g = 0; g < h->nguards; ++g) {
+    const CdgGuardRec &rec = h->guards[g];
+    if (cudaMemcpy(buf, rec.base, kCdgGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(buf + kCdgGuardBytes, rec.base + kCdgGuardBytes + rec.bytes, kCdgGuardBytes,
+                   cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaGetLastError();
+      return g;
+    }
+    for (size_t i = 0; i < 2 * kCdgGuardBytes; ++i)
+      if (buf[i] != kCdgGuardPattern) return g;
+  }
+#else
+  (void)h;
+#endif
+  return -1;
+}
+
+#ifdef CDGRAB_DEBUG
+// Debug build only: how many guarded allocations the handle has, and a HOST-side overwrite of one
+// guard byte of allocation `which` (behind it when tail != 0), for the test of the guard check.
+extern "C" int cdgrab_debug_guard_count(cdgrab_t *h) { return valid(h) ? h->nguards : CDGRAB_ERR_INVALID; }
+extern "C" int cdgrab_debug_poke_guard(cdgrab_t *h, int which, int tail) {
+  if (!valid(h) || which < 0 || which >= h->nguards) return CDGRAB_ERR_INVALID;
+  const CdgGuardRec &rec = h->guards[which];
+  unsigned char *p = tail ? rec.base + kCdgGuardBytes + rec.bytes : rec.base + kCdgGuardBytes - 1;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemset(p, 0, 1) != cudaSuccess) { cudaGetLastError(); return CDGRAB_ERR_CUDA; }
+  return CDGRAB_OK;
+}
+#endif
+
 extern "C" {
 
 const char *cdgrab_strerror(int code) {
@@ -82,6 +115,7 @@ const char *cdgrab_strerror(int code) {
     case CDGRAB_ERR_TIMEOUT: return "bounded device-side wait expired";
     case CDGRAB_ERR_DEVICE: return "no usable sm_100 CUDA device";
     case CDGRAB_ERR_TOO_LARGE: return "size beyond the fixed scratch of the no-allocation entry point";
+    case CDGRAB_ERR_CORRUPT: return "guard bytes around library memory overwritten, or an index check failed (debug build)";
     default: return "unknown error";
   }
 }
@@ -161,22 +195,22 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
   const size_t np = (size_t)m * (size_t)(n / 2);
   bool ok = true;
   const size_t r_elems = (size_t)d * (independent ? (size_t)m : 1);
-  ok = ok && cudaMalloc(&h->r, sizeof(float) * r_elems) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->perm_cur, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->perm_next, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->signs, np) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->margins, sizeof(float) * np) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->rnorm2, sizeof(double)) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->status, sizeof(int)) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->gram, sizeof(double) * ((size_t)m * m + m)) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->oob, sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->r, sizeof(float) * r_elems) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->perm_cur, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->perm_next, sizeof(int32_t) * (size_t)m * n) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->signs, np) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->margins, sizeof(float) * np) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->rnorm2, sizeof(double)) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->status, sizeof(int)) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->gram, sizeof(double) * ((size_t)m * m + m)) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->oob, sizeof(unsigned long long)) == cudaSuccess;
   ok = ok && cudaMemset(h->oob, 0, sizeof(unsigned long long)) == cudaSuccess;
-  ok = ok && cudaMalloc(&h->ticket, sizeof(unsigned)) == cudaSuccess;
+  ok = ok && cdg_alloc(h, &h->ticket, sizeof(unsigned)) == cudaSuccess;
   ok = ok && cudaMemset(h->ticket, 0, sizeof(unsigned)) == cudaSuccess;
   if (ok && independent) {
     h->gram_chunks = cdg_indep_chunks(h);
     h->partials_bytes = sizeof(double) * 3 * (size_t)m * (size_t)h->gram_chunks;
-    ok = ok && cudaMalloc(&h->partials, h->partials_bytes) == cudaSuccess;
+    ok = ok && cdg_alloc(h, &h->partials, h->partials_bytes) == cudaSuccess;
   }
   if (ok && path == CDGRAB_PATH_FMA) {
     if (fma_columns_ok(h)) {
@@ -202,7 +236,7 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
       h->gram_chunks = (int)chunks;
       h->partials_bytes = sizeof(double) * CDG_TILE_ENTRIES * (size_t)npairs * (size_t)chunks;
     }
-    ok = ok && cudaMalloc(&h->partials, h->partials_bytes) == cudaSuccess;
+    ok = ok && cdg_alloc(h, &h->partials, h->partials_bytes) == cudaSuccess;
   }
   if (!ok) {
     cudaGetLastError();
@@ -246,10 +280,11 @@ int cdgrab_destroy(cdgrab_t *h) {
   if (!h) return CDGRAB_OK;
   if (!valid(h)) return CDGRAB_ERR_INVALID;
   cudaDeviceSynchronize();
+  const int rc = cdg_first_broken_guard(h) >= 0 ? CDGRAB_ERR_CORRUPT : CDGRAB_OK;   // debug build only
   free_all(h);
   h->magic = 0;
   delete h;
-  return CDGRAB_OK;
+  return rc;
 }
 
 int cdgrab_set_perms(cdgrab_t *h, const int32_t *perms_in) {
@@ -505,6 +540,8 @@ int cdgrab_status(cdgrab_t *h) {
     cudaGetLastError();
     return CDGRAB_ERR_CUDA;
   }
+  if (st & CDG_ST_BOUNDS) return CDGRAB_ERR_CORRUPT;
+  if (cdg_first_broken_guard(h) >= 0) return CDGRAB_ERR_CORRUPT;
   if (st & CDG_ST_TIMEOUT) return CDGRAB_ERR_TIMEOUT;
   if (st & CDG_ST_NONFINITE) return CDGRAB_ERR_NONFINITE;
   return CDGRAB_OK;

@@ -13,6 +13,21 @@
 // bits of the device status word
 #define CDG_ST_NONFINITE 1
 #define CDG_ST_TIMEOUT 2
+#define CDG_ST_BOUNDS 4       // debug build: an index check failed (the write was skipped)
+
+// Debug build (-DCDGRAB_DEBUG, python -m paper_2302_00845_b200.build --debug): index checks in
+// front of the writes of the decision routines, and every handle-owned allocation wrapped in two
+// guard blocks whose pattern cdgrab_status and cdgrab_destroy verify.  A failed check raises
+// CDG_ST_BOUNDS and skips the write; nothing traps.
+#ifdef CDGRAB_DEBUG
+#define CDG_IDX_OK(cond, status) ((cond) ? true : (atomicOr((status), CDG_ST_BOUNDS), false))
+#else
+#define CDG_IDX_OK(cond, status) true
+#endif
+constexpr size_t kCdgGuardBytes = 256;
+constexpr int kCdgMaxGuards = 32;
+constexpr int kCdgGuardPattern = 0xA5;
+struct CdgGuardRec { unsigned char *base; size_t bytes; };   // base: start of the head guard
 
 // register tile edge of the generic FMA Gram kernel
 #define CDG_TM 8
@@ -40,6 +55,8 @@ struct CdgMapCache {
 
 struct cdgrab_ctx {
   uint32_t magic;
+  int nguards;                          // debug build: guarded allocations of this handle
+  CdgGuardRec guards[kCdgMaxGuards];
   int m, n;
   long long d;
   int dtype;
@@ -136,6 +153,40 @@ struct cdgrab_ctx {
   CUtensorMap tm_f32r;     // 2-D map over r (one row)
   CdgMapCache<1> tm_f32g;  // 2-D maps over the gradient rows of the last few buffers
 };
+
+// Handle-owned device memory.  Release build: cudaMalloc / cudaFree.  Debug build: 256 guard bytes
+// in front and behind, recorded in the handle.
+template <typename P>
+inline cudaError_t cdg_alloc(cdgrab_ctx *h, P **out, size_t bytes) {
+#ifdef CDGRAB_DEBUG
+  *out = nullptr;
+  if (h->nguards >= kCdgMaxGuards) return cudaErrorMemoryAllocation;
+  unsigned char *base = nullptr;
+  cudaError_t e = cudaMalloc(&base, bytes + 2 * kCdgGuardBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaMemset(base, kCdgGuardPattern, kCdgGuardBytes);
+  if (e == cudaSuccess) e = cudaMemset(base + kCdgGuardBytes + bytes, kCdgGuardPattern, kCdgGuardBytes);
+  if (e != cudaSuccess) { cudaFree(base); return e; }
+  h->guards[h->nguards].base = base;
+  h->guards[h->nguards].bytes = bytes;
+  h->nguards++;
+  *out = reinterpret_cast<P *>(base + kCdgGuardBytes);
+  return cudaSuccess;
+#else
+  (void)h;
+  return cudaMalloc(out, bytes);
+#endif
+}
+inline void cdg_free(void *p) {
+#ifdef CDGRAB_DEBUG
+  if (p) cudaFree(static_cast<unsigned char *>(p) - kCdgGuardBytes);
+#else
+  cudaFree(p);
+#endif
+}
+// index of the first allocation whose guard blocks no longer hold the pattern, -1 if all intact
+// (always -1 in the release build); synchronous
+int cdg_first_broken_guard(const cdgrab_ctx *h);
 
 template <typename T>
 __device__ __forceinline__ float cdg_ld(const T *p);

@@ -1210,7 +1210,7 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
   while ((h->gram_chunks + h->ft_gsize - 1) / h->ft_gsize > kFtMaxGroups) ++h->ft_gsize;
   const size_t ctr_bytes = sizeof(unsigned long long) * (kFtMaxGroups + 1);
   const size_t gp_bytes = sizeof(double) * 152 * kFtMaxGroups;
-  if (cudaMalloc(&h->ft_ctr, ctr_bytes) != cudaSuccess || cudaMalloc(&h->ft_group_partials, gp_bytes) != cudaSuccess) {
+  if (cdg_alloc(h, &h->ft_ctr, ctr_bytes) != cudaSuccess || cdg_alloc(h, &h->ft_group_partials, gp_bytes) != cudaSuccess) {
     cudaGetLastError();
     return CDGRAB_ERR_NOMEM;
   }

@@ -142,7 +142,7 @@ literal_step_kernel(const T *__restrict__ g, int count, float *__restrict__ r_gl
         for (int j = 0; j < CH; ++j)
 #pragma unroll
           for (int q = 0; q < 4; ++q) r[j][q] += sd * (double)c[j][q];
-        if (tid == 0) {
+        if (tid == 0 && CDG_IDX_OK(k >= 0 && k < half && i < m, status)) {
           const size_t pos = (size_t)i * half + k;
           tail.signs[pos] = (int8_t)s;
           // |t| / (||r|| ||c||) in fp32: a double square root and division would sit in the chain of decisions

@@ -538,8 +538,8 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     h->umma_ctas = (int)(units < h->num_sms ? (units > 0 ? units : 1) : h->num_sms);
   }
   h->d_pad = total_sub * kSubCols;
-  if (cudaMalloc(&h->r_split, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
-      cudaMalloc(&h->umma_partials, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess) {
+  if (cdg_alloc(h, &h->r_split, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
+      cdg_alloc(h, &h->umma_partials, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess) {
     cudaGetLastError();
     return CDGRAB_ERR_NOMEM;
   }
@@ -569,8 +569,8 @@ int cdg_umma_setup(cdgrab_ctx *h) {
 
 void cdg_umma_teardown(cdgrab_ctx *h) {
   cdg_umma_f32_teardown(h);
-  cudaFree(h->r_split);
-  cudaFree(h->umma_partials);
+  cdg_free(h->r_split);
+  cdg_free(h->umma_partials);
   h->r_split = nullptr;
   h->umma_partials = nullptr;
 }

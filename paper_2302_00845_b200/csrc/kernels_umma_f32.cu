@@ -555,9 +555,9 @@ int cdg_umma_f32_setup(cdgrab_ctx *h) {
   const long long nblk = (h->d + kBlockCols - 1) / kBlockCols;
   h->f32_ctas = (int)(nblk < h->num_sms ? nblk : h->num_sms);
   const size_t pbytes = sizeof(float) * 128 * (size_t)h->f32_npad * h->f32_ctas;
-  if (cudaMalloc(&h->umma_partials, pbytes) != cudaSuccess ||
-      cudaMalloc(&h->f32_bpart, sizeof(double) * 64 * (size_t)h->f32_ctas) != cudaSuccess ||
-      cudaMalloc(&h->f32_dsum, sizeof(double) * 128 * kMaxN) != cudaSuccess) {
+  if (cdg_alloc(h, &h->umma_partials, pbytes) != cudaSuccess ||
+      cdg_alloc(h, &h->f32_bpart, sizeof(double) * 64 * (size_t)h->f32_ctas) != cudaSuccess ||
+      cdg_alloc(h, &h->f32_dsum, sizeof(double) * 128 * kMaxN) != cudaSuccess) {
     cudaGetLastError();
     return CDGRAB_ERR_NOMEM;
   }
@@ -579,8 +579,8 @@ int cdg_umma_f32_setup(cdgrab_ctx *h) {
 }
 
 void cdg_umma_f32_teardown(cdgrab_ctx *h) {
-  cudaFree(h->f32_bpart);
-  cudaFree(h->f32_dsum);
+  cdg_free(h->f32_bpart);
+  cdg_free(h->f32_dsum);
   h->f32_bpart = nullptr;
   h->f32_dsum = nullptr;
 }

@@ -174,6 +174,7 @@ __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const d
   if (!write_out) return;       // a replica of the decisions: S.s is all the caller needs
   const int half = n >> 1;
   for (int i = tid; i < m; i += blockDim.x) {
+    if (!CDG_IDX_OK(k >= 0 && k < half, status)) continue;     // slots k and n-1-k of a row of n
     const int s = S.s[i];
     const size_t pos = (size_t)i * half + k;
     signs[pos] = (int8_t)s;
