@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--no-side-workloads", action="store_true",
                     help="skip the brief runs of the other configurations after the headline one")
     ap.add_argument("--oracle-child", default="", help=argparse.SUPPRESS)
+    ap.add_argument("--independent", action="store_true",
+                    help="ID-GraB (PairBal) mode: one running sum per worker (the uncoordinated baseline)")
     ap.add_argument("--d", type=int, default=0, help="override d (smaller cases for profiler captures)")
     ap.add_argument("--m", type=int, default=0, help="override m")
     return ap.parse_args()
@@ -171,14 +173,14 @@ def source_hash(files=None) -> str:
 # captured with ncu --set full (profiles/*.md); gpt2 figures were taken at d = 8,000,000 and are
 # scaled by d to a full-size launch (traffic grows in proportion to d)
 NCU_TRAFFIC.update({
-    ("gram", "gpt2"): {"bytes": 2.108741e9 * 15.5, "files": ["kernels_umma.cu", "ptx.cuh"], "source": "bd355a8289fade27"},
-    ("update", "gpt2"): {"bytes": 2.156232e9 * 15.5, "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
+    ("gram", "gpt2"): {"bytes": 2.106419e9 * 15.5, "files": ["kernels_umma.cu", "ptx.cuh"], "source": "c889f8e27a23db29"},
+    ("update", "gpt2"): {"bytes": 2.156359e9 * 15.5, "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
     # lstm: captured at d = 4,194,304, scaled by d
-    ("gram", "lstm"): {"bytes": 566.473e6 * (13_500_000 / 4_194_304), "files": ["kernels_umma.cu", "ptx.cuh"], "source": "bd355a8289fade27"},
-    ("update", "lstm"): {"bytes": 582.696e6 * (13_500_000 / 4_194_304), "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
-    # mid, pass 2: bytes of a cold launch (ncu flushes L2 between replays); live, a part of the rows
-    # is still in L2 from pass 1 (128 MiB of inputs against 126 MB of L2)
-    ("update", "mid"): {"bytes": 142.587e6, "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
+    ("gram", "lstm"): {"bytes": 566.966e6 * (13_500_000 / 4_194_304), "files": ["kernels_umma.cu", "ptx.cuh"], "source": "c889f8e27a23db29"},
+    ("update", "lstm"): {"bytes": 585.676e6 * (13_500_000 / 4_194_304), "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
+    # mid, at full size.  Pass 2: bytes of a cold launch (ncu flushes L2 between replays)
+    ("gram", "mid"): {"bytes": 145.620e6, "files": ["kernels_fma.cu", "ptx.cuh"], "source": "0d7b4d20e422bd9e"},
+    ("update", "mid"): {"bytes": 142.614e6, "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
 })
 
 
@@ -263,8 +265,9 @@ def run_reference(args):
 class Run:
     """One workload set up on the current device: handle, input buffers, the step closure."""
 
-    def __init__(self, wl, local: int):
+    def __init__(self, wl, local: int, independent: bool = False):
         from paper_2302_00845_b200 import binding
+        self.independent = independent
         self.wl = wl
         m, n, d = wl.m, wl.n, wl.d
         self.step_bytes = 2 * m * d * wl.elem_bytes
@@ -283,7 +286,7 @@ class Run:
             self.bufs = [gs.step(k) for k in range(self.nbuf)]
         self.flush = (torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
                       if self.flush_mode != "inputs_larger_than_l2" else None)
-        self.h = binding.CdGrab(m, n, d, wl.dtype)
+        self.h = binding.CdGrab(m, n, d, wl.dtype, independent=independent)
         self.stream = torch.cuda.current_stream()
         self.state = {"step": 0}
 
@@ -358,9 +361,11 @@ class Run:
         return {"ms": ms, "launches": launches, "prof": prof, "kernel_events": kernel_events, "wall": (t0, t1)}
 
     def model_bytes(self) -> float:
+        if self.independent:     # every worker has its own running sum: read twice, written once
+            return 2.0 * self.step_bytes + 12.0 * self.wl.m * self.wl.d
         b2 = 2.0 * self.step_bytes + 12.0 * self.wl.d
         b1 = 1.0 * self.step_bytes + 8.0 * self.wl.d
-        return b1 if self.h.path == "fused" else b2
+        return b1 if self.h.path in ("fused", "literal") else b2
 
     def close(self):
         self.h.destroy()
@@ -534,7 +539,7 @@ def run_native(args):
 
     wl = pick_workload(args)
     m, n, d = wl.m, wl.n, wl.d
-    run = Run(wl, local)
+    run = Run(wl, local, independent=args.independent)
     h = run.h
     sampler = ClockSampler(local) if rank == 0 else None
     res = run.measure(args.steps, args.warmup, barrier, not args.no_kernel_events)
@@ -561,7 +566,7 @@ def run_native(args):
 
     # ---- the other configurations of the metric, briefly, after the headline one ---------------
     side = None
-    if rank == 0 and world == 1 and not args.no_side_workloads and not args.d and not args.m:
+    if rank == 0 and world == 1 and not args.no_side_workloads and not args.d and not args.m and not args.independent:
         side = side_workloads(wl.name, local, barrier, peak, with_oracle)
         if with_oracle:
             cpu["one_thread"] = [one_thread_oracle(name, 3.0) for name in ("tiny", "logreg", "mid")]
@@ -575,6 +580,7 @@ def run_native(args):
                        "path": path, "step_input_bytes": step_bytes, "input_buffers": nbuf,
                        "cache": flush_mode, "kernel_events": res["kernel_events"],
                        "parallelism": "replicas" if world > 1 else "single",
+                       "order": "independent" if args.independent else "coordinated",
                        "step_model_bytes": model, "step_model_gbs": step_gbs,
                        "step_model_frac_of_peak": step_gbs / peak,
                        "step_model_frac_of_nominal": step_gbs / NOMINAL_HBM_GBS},

@@ -158,6 +158,19 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream);
  */
 int cdgrab_step_randomized(cdgrab_t *h, const void *grads_dev, const float *u_dev, double w, void *stream);
 
+/*
+ * The same rule with the draws made by the library, so that a randomized epoch can be repeated
+ * from (seed, epoch) alone: u_i for worker i at the handle's current pair index k is the top 24
+ * bits, times 2^-24, of the first output word of Philox4x32-10 (Salmon et al., SC 2011) with the
+ * key (low, high half of seed) and the counter (i, k, epoch, 0).  The caller says which epoch it
+ * is in.  cdgrab_randomized_uniforms writes the m draws of (seed, epoch, k) to u_out_dev (DEVICE
+ * float [m]) without touching a handle.  Errors as for cdgrab_step_randomized.
+ */
+int cdgrab_step_randomized_seeded(cdgrab_t *h, const void *grads_dev, unsigned long long seed, unsigned epoch,
+                                  double w, void *stream);
+int cdgrab_randomized_uniforms(unsigned long long seed, unsigned epoch, unsigned k, int m, float *u_out_dev,
+                               void *stream);
+
 /* Synchronise the device and return how many positions of the current/last epoch had
  * |<r,c>| > w under the randomized rule (negative CDGRAB_ERR_* on error). */
 long long cdgrab_out_of_bound(cdgrab_t *h);

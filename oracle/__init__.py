@@ -67,6 +67,10 @@ def _load():
         lib.cdo_mismatches.argtypes = [C.c_void_p]
         lib.cdo_pairs_done.argtypes = [C.c_void_p]
         lib.cdo_threads.restype = C.c_int
+        lib.cdo_philox4x32_10.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.cdo_philox4x32_10.restype = None
+        lib.cdo_uniform.argtypes = [C.c_ulonglong, C.c_uint, C.c_uint, C.c_uint]
+        lib.cdo_uniform.restype = C.c_double
         _lib = lib
     return _lib
 
@@ -216,6 +220,21 @@ class PairBalanceOracle:
 def threads() -> int:
     """Number of OpenMP threads the C oracle will use."""
     return int(_load().cdo_threads())
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """Philox4x32-10 block: counter of four and key of two 32-bit words -> four 32-bit words."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.empty(4, dtype=np.uint32)
+    assert c.shape == (4,) and k.shape == (2,)
+    _load().cdo_philox4x32_10(c.ctypes.data, k.ctypes.data, out.ctypes.data)
+    return out
+
+
+def uniform(seed: int, epoch: int, k: int, i: int) -> float:
+    """The draw RandomizedBalance uses for worker i at pair index k of an epoch, u in [0,1)."""
+    return float(_load().cdo_uniform(int(seed), int(epoch), int(k), int(i)))
 
 
 def logistic_grad(x: np.ndarray, y: float, w: np.ndarray) -> np.ndarray:

@@ -232,6 +232,38 @@ int cdo_balance_one_randomized(cdo_t *s, int i, const void *g_prev, const void *
 }
 
 /*
+ * The uniform draw of RandomizedBalance ("with probability p", Algorithm 2's subroutine) as a
+ * function of (seed, epoch, pair index k, worker i), so that a randomized epoch can be repeated:
+ * Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3",
+ * SC 2011, section on Philox), written from the published definition.  One round maps the
+ * counter (c0,c1,c2,c3) under the key (k0,k1) to
+ *   (hi(M1*c2) ^ c1 ^ k0,  lo(M1*c2),  hi(M0*c0) ^ c3 ^ k1,  lo(M0*c0))
+ * with M0 = 0xD2511F53, M1 = 0xCD9E8D57; after each round the key advances by the Weyl constants
+ * (0x9E3779B9, 0xBB67AE85).  Ten rounds.  Pinned by the known-answer vectors published with the
+ * generator (tests/golden/philox4x32_10_kat.txt).
+ */
+void cdo_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* u in [0,1) for (seed, epoch, k, i): counter (i, k, epoch, 0), key = the two halves of the seed,
+ * the top 24 bits of the first output word times 2^-24 (exact in single precision). */
+double cdo_uniform(unsigned long long seed, unsigned epoch, unsigned k, unsigned i) {
+  const uint32_t ctr[4] = {i, k, epoch, 0u}, key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t out[4];
+  cdo_philox4x32_10(ctr, key, out);
+  return (double)(out[0] >> 8) * (1.0 / 16777216.0);
+}
+
+/*
  * One whole step: grads is [2][m][d] (slab 0 = earlier position of each pair, slab 1
  * = later), replay is NULL or m signs.
  */

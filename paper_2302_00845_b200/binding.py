@@ -37,6 +37,8 @@ SIGNATURES = {
     "cdgrab_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_step_randomized": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p]),
     "cdgrab_out_of_bound": (C.c_longlong, [C.c_void_p]),
+    "cdgrab_step_randomized_seeded": (C.c_int, [C.c_void_p, C.c_void_p, C.c_ulonglong, C.c_uint, C.c_double, C.c_void_p]),
+    "cdgrab_randomized_uniforms": (C.c_int, [C.c_ulonglong, C.c_uint, C.c_uint, C.c_int, C.c_void_p, C.c_void_p]),
     "cdgrab_step_mean": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_end_epoch": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "cdgrab_get_signs": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -164,6 +166,11 @@ class CdGrab:
         _check(lib().cdgrab_step_randomized(self._h, _ptr(grads), _ptr(u), float(w), _stream_ptr(stream)),
                "cdgrab_step_randomized")
 
+    def step_randomized_seeded(self, grads, seed: int, epoch: int, w: float, stream=None):
+        """step() under the randomized rule with the library's own counter-based draws."""
+        _check(lib().cdgrab_step_randomized_seeded(self._h, _ptr(grads), int(seed), int(epoch), float(w),
+                                                   _stream_ptr(stream)), "cdgrab_step_randomized_seeded")
+
     @property
     def out_of_bound(self) -> int:
         return int(lib().cdgrab_out_of_bound(self._h))
@@ -288,6 +295,15 @@ def step_noalloc(grads, r, signs_out, stream=None):
     code = F32 if grads.dtype == torch.float32 else BF16
     _check(lib().cdgrab_step_noalloc(m, d, code, _ptr(grads), _ptr(r), _ptr(signs_out), _stream_ptr(stream)),
            "cdgrab_step_noalloc")
+
+
+def randomized_uniforms(seed: int, epoch: int, k: int, m: int, stream=None):
+    """The m draws of (seed, epoch, k) as a CUDA float32 tensor."""
+    import torch
+    out = torch.empty(m, dtype=torch.float32, device="cuda")
+    _check(lib().cdgrab_randomized_uniforms(int(seed), int(epoch), int(k), m, _ptr(out), _stream_ptr(stream)),
+           "cdgrab_randomized_uniforms")
+    return out
 
 
 def noalloc_status() -> int:

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "scan.cuh"
 
 namespace {
 
@@ -463,6 +464,30 @@ int cdgrab_step_randomized(cdgrab_t *h, const void *grads_dev, const float *u_de
   const int rc = cdgrab_step(h, grads_dev, stream);
   h->rule_randomized = 0; h->rule_u = nullptr; h->rule_w = 0.0;
   return rc;
+}
+
+int cdgrab_step_randomized_seeded(cdgrab_t *h, const void *grads_dev, unsigned long long seed, unsigned epoch,
+                                  double w, void *stream) {
+  if (!valid(h) || !(w > 0.0)) return CDGRAB_ERR_INVALID;
+  h->rule_randomized = 1; h->rule_u = nullptr; h->rule_w = w; h->rule_seed = seed; h->rule_epoch = epoch;
+  const int rc = cdgrab_step(h, grads_dev, stream);
+  h->rule_randomized = 0; h->rule_w = 0.0;
+  return rc;
+}
+
+namespace {
+__global__ void seeded_uniforms_kernel(unsigned long long seed, unsigned epoch, unsigned k, int m, float *out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < m) out[i] = cdg_seeded_uniform(seed, epoch, k, (unsigned)i);
+}
+}  // namespace
+
+int cdgrab_randomized_uniforms(unsigned long long seed, unsigned epoch, unsigned k, int m, float *u_out_dev,
+                               void *stream) {
+  if (m < 1 || !u_out_dev) return CDGRAB_ERR_INVALID;
+  seeded_uniforms_kernel<<<(m + 127) / 128, 128, 0, (cudaStream_t)stream>>>(seed, epoch, k, m, u_out_dev);
+  if (cudaGetLastError() != cudaSuccess) return CDGRAB_ERR_CUDA;
+  return CDGRAB_OK;
 }
 
 long long cdgrab_out_of_bound(cdgrab_t *h) {

@@ -80,7 +80,9 @@ struct cdgrab_ctx {
   int shard_pending;     // step_begin issued, step_finish outstanding
   int independent;       // 1: ID-GraB mode, r is [m][d] (one running sum per worker)
   int rule_randomized;   // balance rule of the step being enqueued (0: greedy)
-  const float *rule_u;   // [m] uniforms for the randomized rule
+  const float *rule_u;   // [m] uniforms for the randomized rule (NULL: seeded draws)
+  unsigned long long rule_seed;
+  unsigned rule_epoch;
   double rule_w;
   unsigned long long *oob;  // [1] positions with |<r,c>| > w seen by the randomized rule this epoch
   float *mean_out;       // [2][d] destination of the averaged gather buffers for the step being enqueued, or NULL

@@ -42,6 +42,12 @@ literal_step_kernel(const T *__restrict__ g, int count, float *__restrict__ r_gl
                     const CdgTail tail, int *__restrict__ status) {
   __shared__ double red[2][32][2];         // [slot][warp][t, ||c||^2]
   __shared__ int32_t pairs[2 * kLitMaxM];
+  // what the step's write-out needs about worker i, left there by the chain of decisions:
+  // <r,c>, ||c||^2 (fp32 is enough for the reported margin) and the sign
+  __shared__ double t_sh[kLitMaxM];
+  __shared__ float cc_sh[kLitMaxM];
+  __shared__ signed char s_sh[kLitMaxM];
+  __shared__ double rn2_step;               // ||r||^2 at the start of the step
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nth = blockDim.x, nwarps = nth >> 5;
   const int nvec = (int)(d / 4);
@@ -98,9 +104,9 @@ literal_step_kernel(const T *__restrict__ g, int count, float *__restrict__ r_gl
     for (int u = 0; u < PF; ++u) {
       if (w0 + u < total) {
         if (i == 0) {
-          __syncthreads();                 // the pairs of the step before have been used
+          __syncthreads();                 // the write-out of the step before is over
           for (int j = tid; j < 2 * m; j += nth) pairs[j] = tail.perm_cur[(size_t)(j >> 1) * tail.n + 2 * k + (j & 1)];
-          __syncthreads();
+          if (tid == 0) rn2_step = rn2;
         }
         float c[CH][4];
 #pragma unroll
@@ -142,27 +148,52 @@ literal_step_kernel(const T *__restrict__ g, int count, float *__restrict__ r_gl
         for (int j = 0; j < CH; ++j)
 #pragma unroll
           for (int q = 0; q < 4; ++q) r[j][q] += sd * (double)c[j][q];
-        if (tid == 0 && CDG_IDX_OK(k >= 0 && k < half && i < m, status)) {
-          const size_t pos = (size_t)i * half + k;
-          tail.signs[pos] = (int8_t)s;
-          // |t| / (||r|| ||c||) in fp32: a double square root and division would sit in the chain of decisions
-          const float den = sqrtf((float)rn2) * sqrtf((float)cc);
-          tail.margins[pos] = (den > 0.f) ? (float)fabs(t) / den : 0.f;
-          // Algorithm 7: the item that received +1 goes to the front slot, the other to the back
-          const int32_t first = pairs[2 * i], second = pairs[2 * i + 1];
-          tail.perm_next[(size_t)i * tail.n + k] = (s == 1) ? first : second;
-          tail.perm_next[(size_t)i * tail.n + (tail.n - 1 - k)] = (s == 1) ? second : first;
-        }
+        if (tid == 0) { t_sh[i] = t; cc_sh[i] = (float)cc; s_sh[i] = (signed char)s; }
         rn2 += 2.0 * sd * t + cc;
         if (rn2 < 0.0) rn2 = 0.0;
         if (++i == m) {
           // end of a step: r takes the fp32 value a launch per step would have stored, so that a
           // staged call gives the bits of the same steps taken one by one
-          i = 0; ++k;
+          i = 0;
 #pragma unroll
           for (int j = 0; j < CH; ++j)
 #pragma unroll
             for (int q = 0; q < 4; ++q) r[j][q] = (double)(float)r[j][q];
+          // The step's write-out, off the chain of decisions and by all threads: signs, margins
+          // |t| / (||r|| ||c||) with ||r||^2 rebuilt worker by worker from the step's start, and
+          // Algorithm 7's slots: the item that received +1 to the front slot k, the other to n-1-k.
+          __syncthreads();
+          if (CDG_IDX_OK(k >= 0 && k < half, status)) {
+            for (int w = tid; w < m; w += nth) {
+              const int sw = s_sh[w];
+              const size_t pos = (size_t)w * half + k;
+              tail.signs[pos] = (int8_t)sw;
+              const int32_t first = pairs[2 * w], second = pairs[2 * w + 1];
+              tail.perm_next[(size_t)w * tail.n + k] = (sw == 1) ? first : second;
+              tail.perm_next[(size_t)w * tail.n + (tail.n - 1 - k)] = (sw == 1) ? second : first;
+            }
+            if (warp == 0) {
+              // ||r||^2 seen by worker w = start + sum_{v<w} (2 s_v t_v + ||c_v||^2): a running sum, 32 workers at a time
+              double base = rn2_step;
+              for (int w0 = 0; w0 < m; w0 += 32) {
+                const int w = w0 + lane;
+                const double inc = (w < m) ? 2.0 * (double)s_sh[w] * t_sh[w] + (double)cc_sh[w] : 0.0;
+                double pre = inc;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                  const double up = __shfl_up_sync(0xffffffffu, pre, off);
+                  if (lane >= off) pre += up;
+                }
+                if (w < m) {
+                  const double before = base + (pre - inc);
+                  const float den = sqrtf(before > 0.0 ? (float)before : 0.f) * sqrtf(cc_sh[w]);
+                  tail.margins[(size_t)w * half + k] = (den > 0.f) ? (float)fabs(t_sh[w]) / den : 0.f;
+                }
+                base += __shfl_sync(0xffffffffu, pre, 31);
+              }
+            }
+          }
+          ++k;
         }
       }
     }

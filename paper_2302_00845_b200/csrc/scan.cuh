@@ -13,16 +13,39 @@
 // (where Algorithm 5 would stop) are counted in *oob.
 struct CdgRule {
   int randomized;
-  const float *u;             // [m] uniforms in [0,1), device
+  const float *u;             // [m] uniforms in [0,1), device; NULL: drawn from (seed, epoch, k, i)
   double w;
   unsigned long long *oob;    // device counter
+  unsigned long long seed;    // seeded draws: Philox4x32-10 keyed by the seed, counter (i, k, epoch, 0)
+  unsigned epoch, k;
 };
+
+// Philox4x32-10 (Salmon et al., SC 2011): ten rounds of
+//   (c0, c1, c2, c3) <- (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)),
+// the key advancing by the Weyl constants after each round.  Returns the first output word.
+__host__ __device__ inline uint32_t cdg_philox4x32_10_first(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                            uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const unsigned long long p0 = 0xD2511F53ull * c0, p1 = 0xCD9E8D57ull * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    c1 = (uint32_t)p1; c3 = (uint32_t)p0; c0 = n0; c2 = n2;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+// the draw of worker i at pair index k of an epoch: top 24 bits of the word, times 2^-24
+__host__ __device__ inline float cdg_seeded_uniform(unsigned long long seed, unsigned epoch, unsigned k, unsigned i) {
+  const uint32_t x = cdg_philox4x32_10_first(i, k, epoch, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+  return (float)(x >> 8) * (1.0f / 16777216.0f);
+}
 
 __device__ __forceinline__ int cdg_decide(const CdgRule &rule, int i, double ti, int &oob_local) {
   if (!rule.randomized) return (ti < 0.0) ? 1 : -1;   // a tie gives -1
   const double p = 0.5 - ti / (2.0 * rule.w);
   if (fabs(ti) > rule.w) ++oob_local;
-  return ((double)rule.u[i] < p) ? 1 : -1;
+  const float u = rule.u ? rule.u[i] : cdg_seeded_uniform(rule.seed, rule.epoch, rule.k, (unsigned)i);
+  return ((double)u < p) ? 1 : -1;
 }
 
 inline CdgRule cdg_rule_of(const cdgrab_ctx *h) {
@@ -31,6 +54,9 @@ inline CdgRule cdg_rule_of(const cdgrab_ctx *h) {
   r.u = h->rule_u;
   r.w = h->rule_w;
   r.oob = h->oob;
+  r.seed = h->rule_seed;
+  r.epoch = h->rule_epoch;
+  r.k = (unsigned)h->k;
   return r;
 }
 

@@ -525,3 +525,45 @@ def test_randomized_replay_band():
     o3, z3, _, _ = _rand_state(5)
     s = o3.balance_one_randomized(0, z3[0, 2], z3[0, 3], p + 2.0 * band, w, replay=+1, tau=tau)
     assert s == -1 and o3.mismatches == 1                              # outside: own sign kept
+
+
+# ---- the seeded draws of RandomizedBalance: Philox4x32-10 -----------------------------------------
+def test_philox_known_answer_vectors():
+    """The generator's published known-answer vectors (tests/golden/philox4x32_10_kat.txt)."""
+    rows = [l for l in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for line in rows:
+        ctr, key, want = [[int(w, 16) for w in part.split()] for part in line.split("|")]
+        assert oracle.philox4x32_10(ctr, key).tolist() == want
+
+
+def test_philox_reduced_rounds_would_not_pass_and_words_are_not_swapped():
+    """A dropped round, swapped multipliers or a swapped key word all change the first vector."""
+    M0, M1, W0, W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
+
+    def ref(ctr, key, rounds=10, m0=M0, m1=M1):
+        c, k = list(ctr), list(key)
+        for _ in range(rounds):
+            p0, p1 = m0 * c[0], m1 * c[2]
+            c = [(p1 >> 32) ^ c[1] ^ k[0], p1 & 0xFFFFFFFF, (p0 >> 32) ^ c[3] ^ k[1], p0 & 0xFFFFFFFF]
+            k = [(k[0] + W0) & 0xFFFFFFFF, (k[1] + W1) & 0xFFFFFFFF]
+        return c
+    ctr, key = [1, 2, 3, 4], [5, 6]
+    good = oracle.philox4x32_10(ctr, key).tolist()
+    assert good == ref(ctr, key)
+    assert good != ref(ctr, key, rounds=9) and good != ref(ctr, key, m0=M1, m1=M0) and good != ref(ctr, [6, 5])
+
+
+def test_seeded_uniform_is_a_24_bit_fraction_of_the_first_word():
+    for seed, epoch, k, i in [(0, 0, 0, 0), (12345678901234567, 3, 17, 99), (2**64 - 1, 2**32 - 1, 7, 1023)]:
+        x0 = int(oracle.philox4x32_10([i, k, epoch, 0], [seed & 0xFFFFFFFF, seed >> 32])[0])
+        u = oracle.uniform(seed, epoch, k, i)
+        assert u == (x0 >> 8) / 2.0**24 and 0.0 <= u < 1.0
+
+
+def test_seeded_uniforms_look_uniform():
+    u = np.array([oracle.uniform(42, 1, k, i) for k in range(200) for i in range(100)])
+    assert abs(u.mean() - 0.5) < 0.01 and abs(u.var() - 1 / 12) < 0.005
+    hist, _ = np.histogram(u, bins=10, range=(0, 1))
+    assert hist.min() > 1800 and hist.max() < 2200
+    assert len(np.unique(u)) > 19_900                       # distinct counters give distinct draws
