@@ -56,7 +56,7 @@ def main():
           f"single-launch form only): {(t[:, 10].min() - t[:, 11].max()) / 1e3:.2f} us")
     for slot, name in NAMES:
         col = (t[:, slot] - t0) / 1e3
-        col = col[t[:, slot] > 0]
+        col = col[t[:, slot] >= t[:, 10]]        # stamped during the last launch (not a leftover of an earlier one)
         if col.size:
             print(f"{name:38s} min {col.min():8.2f}  median {np.median(col):8.2f}  max {col.max():8.2f} us"
                   f"   ({col.size} CTAs)")
