@@ -173,14 +173,14 @@ def source_hash(files=None) -> str:
 # captured with ncu --set full (profiles/*.md); gpt2 figures were taken at d = 8,000,000 and are
 # scaled by d to a full-size launch (traffic grows in proportion to d)
 NCU_TRAFFIC.update({
-    ("gram", "gpt2"): {"bytes": 2.106419e9 * 15.5, "files": ["kernels_umma.cu", "ptx.cuh"], "source": "c889f8e27a23db29"},
-    ("update", "gpt2"): {"bytes": 2.156359e9 * 15.5, "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
+    ("gram", "gpt2"): {"bytes": 2.105560e+09 * 15.5, "files": ["kernels_umma.cu", "ptx.cuh"], "source": "c889f8e27a23db29"},
+    ("update", "gpt2"): {"bytes": 2.155899e+09 * 15.5, "files": ["kernels_generic.cu"], "source": "1cffb536a83d70ae"},
     # lstm: captured at d = 4,194,304, scaled by d
-    ("gram", "lstm"): {"bytes": 566.966e6 * (13_500_000 / 4_194_304), "files": ["kernels_umma.cu", "ptx.cuh"], "source": "c889f8e27a23db29"},
-    ("update", "lstm"): {"bytes": 585.676e6 * (13_500_000 / 4_194_304), "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
+    ("gram", "lstm"): {"bytes": 5.664448e+08 * (13_500_000 / 4_194_304), "files": ["kernels_umma.cu", "ptx.cuh"], "source": "c889f8e27a23db29"},
+    ("update", "lstm"): {"bytes": 5.820989e+08 * (13_500_000 / 4_194_304), "files": ["kernels_generic.cu"], "source": "1cffb536a83d70ae"},
     # mid, at full size.  Pass 2: bytes of a cold launch (ncu flushes L2 between replays)
-    ("gram", "mid"): {"bytes": 145.620e6, "files": ["kernels_fma.cu", "ptx.cuh"], "source": "0d7b4d20e422bd9e"},
-    ("update", "mid"): {"bytes": 142.614e6, "files": ["kernels_generic.cu"], "source": "16428dad55e58a5c"},
+    ("gram", "mid"): {"bytes": 1.445571e+08, "files": ["kernels_fma.cu", "ptx.cuh"], "source": "0d7b4d20e422bd9e"},
+    ("update", "mid"): {"bytes": 1.417111e+08, "files": ["kernels_generic.cu"], "source": "1cffb536a83d70ae"},
 })
 
 

@@ -165,11 +165,21 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
   h->pdl = 1;                      // CDGRAB_PDL=0: plain stream order between the launches of a step
   if (const char *e = getenv("CDGRAB_PDL")) h->pdl = atoi(e) ? 1 : 0;
   if (const char *e = getenv("CDGRAB_CLUSTER")) h->cluster_off = atoi(e) ? 0 : 1;
+  // Pass 2 is the last reader of a step's rows.  Where a step is about the size of L2 (workload 3:
+  // 128 MiB against 126 MB) reading them with the evict-first priority keeps them from pushing r
+  // and the next step's first rows out: pass 2 took 24.8 instead of 30 us on a box where it paid
+  // most; on steps many times L2 the hint cost 1-4 %, so it is tied to the step's size.
+  // CDGRAB_UPD_EF=0/1 overrides.
+  h->upd_evict_first = (2 * (size_t)m * (size_t)d * elem_size(dtype) <= ((size_t)192 << 20)) ? 1 : 0;
+  if (const char *e = getenv("CDGRAB_UPD_EF")) h->upd_evict_first = atoi(e) ? 1 : 0;
 
   // ---- choose the path ------------------------------------------------------------
   const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);
   const bool fused_ok = cdg_fused_supported(m, d, dtype);
-  const bool umma_ok = cdg_umma_supported(m, d, dtype);
+  // bf16 with 65..128 workers: the term-splitting tensor-core kernel (CDGRAB_UMMA_BF16_WIDE=0: not used)
+  const char *wide_env = getenv("CDGRAB_UMMA_BF16_WIDE");
+  const bool umma_wide = dtype == CDGRAB_BF16 && cdg_umma_terms_bf16_supported(m, d) && !(wide_env && atoi(wide_env) == 0);
+  const bool umma_ok = cdg_umma_supported(m, d, dtype) || umma_wide;
   const bool literal_ok = cdg_literal_supported(m, d, dtype) && !shard && !independent;
   int path;
   if (forced == CDGRAB_PATH_AUTO) {
@@ -246,7 +256,7 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
     return CDGRAB_ERR_NOMEM;
   }
   if (path == CDGRAB_PATH_UMMA) {
-    const int rc = cdg_umma_setup(h);
+    const int rc = umma_wide ? cdg_umma_f32_setup(h) : cdg_umma_setup(h);
     if (rc != CDGRAB_OK) { free_all(h); delete h; return rc; }
   }
   if (path == CDGRAB_PATH_FMA && fma_columns_ok(h) && cdg_fma_tma_supported(m, d, dtype)) {
@@ -332,6 +342,7 @@ int cdgrab_begin_epoch(cdgrab_t *h, void *stream) {
 }
 
 static cudaError_t launch_pass1(cdgrab_ctx *h, const void *grads_dev, cudaStream_t st) {
+  if (h->path == CDGRAB_PATH_UMMA && h->umma_f32) return cdg_launch_gram_umma_f32(h, grads_dev, st);
   if (h->path == CDGRAB_PATH_UMMA) return cdg_launch_gram_umma(h, grads_dev, st);
   if (h->fma_tma) return cdg_launch_gram_fma_tma(h, grads_dev, st);
   if (fma_columns_ok(h)) return cdg_launch_gram_fma(h, grads_dev, st);

@@ -95,6 +95,7 @@ struct cdgrab_ctx {
   int fma_tma_stages;
   int fma_tma_boxrows;     // rows per bulk-tensor copy
   int fma_tma_contig;      // 1: each CTA owns a contiguous range of tiles
+  int upd_evict_first;     // pass 2 reads the rows with the L2 evict-first priority (256-bit loads)
   int pdl;                 // 1: dependent launches start early and wait on the device for their predecessor
   int cluster_off;         // 1: the one-launch step never spreads over a thread-block cluster (CDGRAB_CLUSTER=0)
   int fma_tma_fused;       // 1: the last CTA of pass 1 also combines and decides (no scan launch)
@@ -143,15 +144,16 @@ struct cdgrab_ctx {
 
   // tcgen05 path for fp32 gradients with the bf16 terms formed inside the kernel
   int umma_f32;            // 1: that kernel serves pass 1
-  int f32_npad;            // MMA N: 3m rounded up to 16
+  int f32_nt;              // bf16 terms per difference: 3 (fp32 gradients) or 2 (bf16 gradients, m > 64)
+  int f32_npad;            // MMA N: terms x m rounded up to 16
   int f32_nsub;            // 64-column blocks per stage
   int f32_nops;            // operand buffers
   int f32_stages;
   int f32_drain;           // 64-column blocks per TMEM accumulation chunk
   int f32_ctas;
   size_t f32_smem;
-  double *f32_bpart;       // [ctas][64] per-CTA partial b
-  double *f32_dsum;        // [128][192] the partial D summed over the CTAs
+  double *f32_bpart;       // [ctas][128] per-CTA partial b
+  double *f32_dsum;        // [128][256] the partial D summed over the CTAs
   CUtensorMap tm_f32r;     // 2-D map over r (one row)
   CdgMapCache<1> tm_f32g;  // 2-D maps over the gradient rows of the last few buffers
 };
@@ -302,6 +304,7 @@ void cdg_umma_teardown(cdgrab_ctx *h);
 cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t st);
 // ... for fp32 gradients, terms formed in the kernel (17 <= m <= 64)
 bool cdg_umma_f32_supported(int m, long long d);
+bool cdg_umma_terms_bf16_supported(int m, long long d);   // the same kernel for bf16 gradients, 65 <= m <= 128
 int cdg_umma_f32_setup(cdgrab_ctx *h);
 void cdg_umma_f32_teardown(cdgrab_ctx *h);
 cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStream_t st);

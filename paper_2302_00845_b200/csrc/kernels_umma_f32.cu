@@ -1,4 +1,6 @@
-// Pass 1 on the tensor cores (tcgen05) for fp32 gradients, 17 <= m <= 64.
+// Pass 1 on the tensor cores (tcgen05) with the pair differences split into bf16 terms inside the
+// kernel: fp32 gradients with 17 <= m <= 64 (three terms), and bf16 gradients with 65 <= m <= 128
+// (two terms; their 2m raw rows no longer fit one 128-row MMA tile).  The fp32 case first:
 //
 // The pair differences c_i = z1_i - z2_i (rounded to fp32, as every other path forms them) are
 // written as three bf16 terms hi + mid + lo = c exactly (3 x 8 significand bits).  Products of
@@ -24,6 +26,14 @@
 // go to global memory, a second kernel adds the CTAs in index order in fp64, forms G and takes
 // the step's decisions.  Every wait is bounded: on expiry the CTA raises the time-out bit of the
 // status word, lets its copies land, frees its TMEM and returns.
+//
+// bf16 gradients, 65 <= m <= 128 (NT = 2): c = z1 - z2 in fp32, then c = hi + lo with a residual
+// below 2^-17 |c| (the tolerance for bf16 inputs is 1e-3).  B = [hi_0.. | lo_0..] (N = 2m <= 256),
+// A = the first 128 rows (all of hi), and  G_ki = D[k][i] + D[k][m+i] + D[i][m+k]  (hi x hi,
+// hi x lo and its transpose; lo x lo, below 2^-16 of the product, is left out).  The converter
+// threads take the rows in two passes to bound their registers, and the read-back warps add
+// each chunk (4096 columns) to the CTA's partial D in global memory (it stays in L2) instead of
+// holding 256 columns of accumulators in registers.
 #include <cudaTypedefs.h>
 #include <stdlib.h>
 
@@ -46,7 +56,8 @@ constexpr int kMaxOps = 4;                           // operand buffers (one 64-
 constexpr int kRowSlots = (64 + kConvRows - 1) / kConvRows;   // rows per converter thread at m = 64
 constexpr int kBlockCols = 64;                       // columns per MMA block = one 128-byte swizzle row of bf16
 constexpr int kFlushBlocks = 32;                     // blocks between two moves of the fp32 b sums into fp64
-constexpr int kMaxN = 192;                           // 3 m at m = 64
+constexpr int kMaxN = 256;                           // row pitch of the summed D: 3 m at m = 64, 2 m at m = 128
+constexpr int kMaxM = 128;
 
 struct F32Params {
   int m;
@@ -56,6 +67,25 @@ struct F32Params {
   int nops;            // operand buffers
   int drain;           // blocks accumulated in TMEM before the sum is read back
   long long nblk;      // ceil(d / 64)
+  int pass_rows;       // rows per converter pass (a multiple of 8; = m rounded up when there is one pass)
+};
+
+template <typename T>
+struct TermIn;
+template <>
+struct TermIn<float> {                     // 4 columns = 16 bytes
+  static __device__ __forceinline__ void ld(const uint8_t *p, float (&v)[4]) {
+    const float4 f = *reinterpret_cast<const float4 *>(p);
+    v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+  }
+};
+template <>
+struct TermIn<__nv_bfloat16> {             // 4 columns = 8 bytes, widened exactly
+  static __device__ __forceinline__ void ld(const uint8_t *p, float (&v)[4]) {
+    const uint2 w = *reinterpret_cast<const uint2 *>(p);
+    v[0] = __uint_as_float(w.x << 16); v[1] = __uint_as_float(w.x & 0xffff0000u);
+    v[2] = __uint_as_float(w.y << 16); v[3] = __uint_as_float(w.y & 0xffff0000u);
+  }
 };
 
 __device__ __forceinline__ uint64_t f32_umma_desc(uint32_t saddr) {
@@ -88,9 +118,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float x, float y) {
   return *reinterpret_cast<const uint32_t *>(&h);
 }
 
-// NS: rows each converter thread takes = ceil(m / kConvRows), a compile-time count so that the
-// NS x 2 split chains of a block sit in one basic block and the scheduler can interleave them.
-template <int NS>
+// T: element type of the gradients; NT: bf16 terms per difference; NP: passes the converter
+// threads make over the rows of a block; NS: rows each converter thread takes per pass, a
+// compile-time count so that the NS x 2 split chains sit in one basic block and the scheduler
+// can interleave them.
+template <typename T, int NT, int NS, int NP>
 __global__ void __launch_bounds__(kThreads, 1)
 gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
                      const F32Params p, float *__restrict__ partials, double *__restrict__ bpart,
@@ -103,13 +135,14 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
   __shared__ __align__(8) uint64_t bar_acc_full[2];
   __shared__ __align__(8) uint64_t bar_acc_empty[2];
   __shared__ uint32_t tmem_base_sh;
-  __shared__ double bred[kConvThreads * NS];
+  constexpr uint32_t ES = (uint32_t)sizeof(T);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m = p.m;
   const int scols = p.nsub * kBlockCols;
   const int rows8 = (2 * m + 7) & ~7;                                      // rows a stage holds (8-row boxes)
-  const uint32_t stage_bytes = (uint32_t)(rows8 + 1) * scols * 4u;         // the rows, then the piece of r
+  const uint32_t rows_bytes = (uint32_t)rows8 * scols * ES;
+  const uint32_t stage_bytes = rows_bytes + (uint32_t)scols * 4u;          // the rows, then the piece of r (fp32)
   const int op_rows = p.npad > 128 ? p.npad : 128;                         // operand A spans 128 rows
   const uint32_t op_bytes = (uint32_t)op_rows * 128u;
   const uint32_t ops_base = (smem_u32(smem_raw) + 1023u) & ~1023u;         // swizzle atoms need 1024-B alignment
@@ -139,10 +172,10 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_g) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_r) : "memory");
   }
-  // operand rows no converter ever writes (past the 3m term rows) are zeroed once
+  // operand rows no converter ever writes (past the NT m term rows) are zeroed once
   for (int o = 0; o < p.nops; ++o) {
-    uint8_t *z = ops_ptr + (size_t)o * op_bytes + (size_t)(3 * m) * 128;   // whole rows: 128 B each, swizzle-neutral
-    const uint32_t nbytes = (uint32_t)(op_rows - 3 * m) * 128u;
+    uint8_t *z = ops_ptr + (size_t)o * op_bytes + (size_t)(NT * m) * 128;   // whole rows: 128 B each, swizzle-neutral
+    const uint32_t nbytes = (uint32_t)(op_rows - NT * m) * 128u;
     for (uint32_t off = threadIdx.x * 16; off < nbytes; off += kThreads * 16)
       *reinterpret_cast<uint4 *>(z + off) = make_uint4(0, 0, 0, 0);
   }
@@ -163,7 +196,7 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       const int nbox = rows8 >> 3;
-      const uint32_t box_bytes = 8u * scols * 4u;
+      const uint32_t box_bytes = 8u * scols * ES;
       int issued = 0;
       bool ok = true;
       int s = 0;
@@ -218,31 +251,33 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     }
     if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
   } else if (warp < 2 + kConvWarps) {
-    // ---------------- converters: fp32 tile -> differences -> three bf16 terms; b on the side ----------------
+    // ---------------- converters: tile -> differences -> NT bf16 terms; b on the side ----------------
     const int ct = threadIdx.x - 64;                 // 0..191
-    const int q = ct & 15;                           // this thread's float4 of every row it takes
-    const int row0 = ct >> 4;                        // rows row0, row0 + 12, ...
-    // Byte offsets that never change: of the thread's float4 inside a stage (block 0) and of its
-    // 8 bytes of terms inside an operand buffer -- row i, m + i, 2m + i, each 128 B, 16-byte
-    // chunk (q >> 1) at chunk (q >> 1) ^ (row & 7), upper half of the chunk for odd q.
-    uint32_t src[NS], dst_h[NS], dst_m[NS], dst_l[NS];
-    uint32_t vmask = 0;
+    const int q = ct & 15;                           // this thread's 4 columns of every row it takes
+    const int row0 = ct >> 4;                        // rows row0, row0 + 12, ... of a pass
+    // Byte offsets that never change (pass 0): of the thread's 4 columns inside a stage (block 0)
+    // and of its 8 bytes of term t inside an operand buffer -- row t m + i, 128 B per row, 16-byte
+    // chunk (q >> 1) at chunk (q >> 1) ^ (row & 7), upper half of the chunk for odd q.  A further
+    // pass lies pass_rows rows on: a multiple of 8, so the swizzle phase of every row is the same.
+    uint32_t src[NS], dst[NT][NS];
 #pragma unroll
     for (int j = 0; j < NS; ++j) {
-      int i = row0 + kConvRows * j;
-      if (i < m) vmask |= 1u << j;
-      else i = m - 1;                                // a slot past the last row loads a valid row and stores nothing
-      const int im = m + i, il = 2 * m + i;
-      src[j] = (uint32_t)(i * scols + q * 4) * 4u;
-      dst_h[j] = (uint32_t)(i * 128 + ((((q >> 1) ^ (i & 7)) << 4) | ((q & 1) << 3)));
-      dst_m[j] = (uint32_t)(im * 128 + ((((q >> 1) ^ (im & 7)) << 4) | ((q & 1) << 3)));
-      dst_l[j] = (uint32_t)(il * 128 + ((((q >> 1) ^ (il & 7)) << 4) | ((q & 1) << 3)));
-    }
-    const uint32_t z2_off = (uint32_t)(m * scols) * 4u;          // from a row of slab 0 to its partner in slab 1
-    float bacc[NS];
-    double bsum[NS];
+      const int i = row0 + kConvRows * j;
+      src[j] = (uint32_t)(i * scols + q * 4) * ES;
 #pragma unroll
-    for (int j = 0; j < NS; ++j) { bacc[j] = 0.f; bsum[j] = 0.0; }
+      for (int t = 0; t < NT; ++t) {
+        const int row = t * m + i;
+        dst[t][j] = (uint32_t)(row * 128 + ((((q >> 1) ^ (row & 7)) << 4) | ((q & 1) << 3)));
+      }
+    }
+    const uint32_t z2_off = (uint32_t)(m * scols) * ES;          // from a row of slab 0 to its partner in slab 1
+    const uint32_t pass_src = (uint32_t)(p.pass_rows * scols) * ES, pass_dst = (uint32_t)p.pass_rows * 128u;
+    float bacc[NP][NS];
+    double bsum[NP][NS];
+#pragma unroll
+    for (int hp = 0; hp < NP; ++hp)
+#pragma unroll
+      for (int j = 0; j < NS; ++j) { bacc[hp][j] = 0.f; bsum[hp][j] = 0.0; }
     bool ok = true;
     int s = 0, o = 0, since_flush = 0;
     uint32_t full_parity = 0, turn_o = 0;
@@ -250,64 +285,69 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_full[s]), full_parity, deadline));   // the lanes leave together
       if (!ok) break;
       const uint8_t *tile = stages_ptr + (size_t)s * stage_bytes;
-      const float *rt = reinterpret_cast<const float *>(tile) + (size_t)rows8 * scols;
+      const float *rt = reinterpret_cast<const float *>(tile + rows_bytes);
       const int cnt = min(p.nsub, nsb - it * p.nsub);      // blocks past the range belong to the next CTA
       for (int sub = 0; sub < cnt; ++sub) {
-        // Straight-line code from here to the stores: every load first, then the split one step
-        // at a time over all slots (each step's 2 NS operations are independent of one another).
-        const float4 rv = *reinterpret_cast<const float4 *>(rt + sub * kBlockCols + q * 4);
-        float c[NS][4];
-#pragma unroll
-        for (int j = 0; j < NS; ++j) {
-          const float4 za = *reinterpret_cast<const float4 *>(tile + src[j] + sub * (kBlockCols * 4));
-          const float4 zb = *reinterpret_cast<const float4 *>(tile + src[j] + z2_off + sub * (kBlockCols * 4));
-          c[j][0] = za.x - zb.x; c[j][1] = za.y - zb.y; c[j][2] = za.z - zb.z; c[j][3] = za.w - zb.w;
-        }
-        uint32_t hi[NS][2], mid[NS][2], lo[NS][2];
-        float r1[NS][4];
-#pragma unroll
-        for (int j = 0; j < NS; ++j)
-#pragma unroll
-          for (int h = 0; h < 2; ++h) hi[j][h] = pack_bf16x2(c[j][2 * h], c[j][2 * h + 1]);
-#pragma unroll
-        for (int j = 0; j < NS; ++j)
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            r1[j][2 * h] = c[j][2 * h] - __uint_as_float(hi[j][h] << 16);
-            r1[j][2 * h + 1] = c[j][2 * h + 1] - __uint_as_float(hi[j][h] & 0xffff0000u);
-          }
-#pragma unroll
-        for (int j = 0; j < NS; ++j)
-#pragma unroll
-          for (int h = 0; h < 2; ++h) mid[j][h] = pack_bf16x2(r1[j][2 * h], r1[j][2 * h + 1]);
-#pragma unroll
-        for (int j = 0; j < NS; ++j)
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            r1[j][2 * h] -= __uint_as_float(mid[j][h] << 16);
-            r1[j][2 * h + 1] -= __uint_as_float(mid[j][h] & 0xffff0000u);
-          }
-#pragma unroll
-        for (int j = 0; j < NS; ++j)
-#pragma unroll
-          for (int h = 0; h < 2; ++h) lo[j][h] = pack_bf16x2(r1[j][2 * h], r1[j][2 * h + 1]);
-#pragma unroll
-        for (int j = 0; j < NS; ++j) {
-          float t = fmaf(rv.x, c[j][0], bacc[j]);
-          t = fmaf(rv.y, c[j][1], t);
-          t = fmaf(rv.z, c[j][2], t);
-          t = fmaf(rv.w, c[j][3], t);
-          bacc[j] = (vmask & (1u << j)) ? t : 0.f;
-        }
         if (turn_o > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_op_empty[o]), (turn_o - 1) & 1, deadline));
         if (!ok) break;
         uint8_t *op = ops_ptr + (size_t)o * op_bytes;
+        const float4 rv = *reinterpret_cast<const float4 *>(rt + sub * kBlockCols + q * 4);
 #pragma unroll
-        for (int j = 0; j < NS; ++j) {
-          if (vmask & (1u << j)) {
-            *reinterpret_cast<uint2 *>(op + dst_h[j]) = make_uint2(hi[j][0], hi[j][1]);
-            *reinterpret_cast<uint2 *>(op + dst_m[j]) = make_uint2(mid[j][0], mid[j][1]);
-            *reinterpret_cast<uint2 *>(op + dst_l[j]) = make_uint2(lo[j][0], lo[j][1]);
+        for (int hp = 0; hp < NP; ++hp) {
+          // Straight-line code from the loads to the stores: every load first, then the split one
+          // step at a time over all slots (each step's 2 NS operations are independent of one another).
+          uint32_t vmask = 0;
+          float c[NS][4];
+#pragma unroll
+          for (int j = 0; j < NS; ++j) {
+            int i = hp * p.pass_rows + row0 + kConvRows * j;
+            const bool in_pass = row0 + kConvRows * j < p.pass_rows;
+            if (i < m && in_pass) vmask |= 1u << j;
+            // a slot past the last row loads a valid row (row 0 of the pass) and stores nothing
+            const uint32_t so = (i < m && in_pass) ? src[j] : (uint32_t)(q * 4) * ES;
+            float za[4], zb[4];
+            TermIn<T>::ld(tile + hp * pass_src + so + sub * (kBlockCols * ES), za);
+            TermIn<T>::ld(tile + hp * pass_src + so + z2_off + sub * (kBlockCols * ES), zb);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) c[j][e] = za[e] - zb[e];
+          }
+          uint32_t term[NT][NS][2];
+          float r1[NS][4];
+#pragma unroll
+          for (int j = 0; j < NS; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) r1[j][e] = c[j][e];
+#pragma unroll
+          for (int t = 0; t < NT; ++t) {
+#pragma unroll
+            for (int j = 0; j < NS; ++j)
+#pragma unroll
+              for (int h = 0; h < 2; ++h) term[t][j][h] = pack_bf16x2(r1[j][2 * h], r1[j][2 * h + 1]);
+            if (t + 1 < NT) {
+#pragma unroll
+              for (int j = 0; j < NS; ++j)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                  r1[j][2 * h] -= __uint_as_float(term[t][j][h] << 16);
+                  r1[j][2 * h + 1] -= __uint_as_float(term[t][j][h] & 0xffff0000u);
+                }
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < NS; ++j) {
+            float t = fmaf(rv.x, c[j][0], bacc[hp][j]);
+            t = fmaf(rv.y, c[j][1], t);
+            t = fmaf(rv.z, c[j][2], t);
+            t = fmaf(rv.w, c[j][3], t);
+            bacc[hp][j] = (vmask & (1u << j)) ? t : 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < NS; ++j) {
+            if (vmask & (1u << j)) {
+#pragma unroll
+              for (int t = 0; t < NT; ++t)
+                *reinterpret_cast<uint2 *>(op + hp * pass_dst + dst[t][j]) = make_uint2(term[t][j][0], term[t][j][1]);
+            }
           }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads these bytes through the async proxy
@@ -317,7 +357,9 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
         if (++since_flush == kFlushBlocks) {
           since_flush = 0;
 #pragma unroll
-          for (int j = 0; j < NS; ++j) { bsum[j] += (double)bacc[j]; bacc[j] = 0.f; }
+          for (int hp = 0; hp < NP; ++hp)
+#pragma unroll
+            for (int j = 0; j < NS; ++j) { bsum[hp][j] += (double)bacc[hp][j]; bacc[hp][j] = 0.f; }
         }
       }
       __syncwarp();
@@ -325,28 +367,42 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
       if (++s == p.stages) { s = 0; full_parity ^= 1u; }
     }
     if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
-#pragma unroll
-    for (int j = 0; j < NS; ++j) bred[ct * NS + j] = bsum[j] + (double)bacc[j];
+    // the ring of stages is idle now (every tile has landed and been converted): it holds the
+    // per-thread sums of b while the 16 threads that shared a row are added up, in q order
     asm volatile("bar.sync 2, %0;" ::"r"(kConvThreads) : "memory");        // the converter warps only
-    if (ct < m) {
-      // row i was shared by the 16 threads ((i % kConvRows) * 16 + q), slot i / kConvRows: add them in q order
-      double v = 0.0;
-      const int t0 = (ct % kConvRows) * 16, j = ct / kConvRows;
+    double *bred = reinterpret_cast<double *>(stages_ptr);
+    if (ok) {
 #pragma unroll
-      for (int qq = 0; qq < 16; ++qq) v += bred[(t0 + qq) * NS + j];
-      bpart[(size_t)blockIdx.x * 64 + ct] = v;
+      for (int hp = 0; hp < NP; ++hp)
+#pragma unroll
+        for (int j = 0; j < NS; ++j) bred[(ct * NP + hp) * NS + j] = bsum[hp][j] + (double)bacc[hp][j];
+    }
+    asm volatile("bar.sync 2, %0;" ::"r"(kConvThreads) : "memory");
+    if (ct < m && ok) {
+      const int hp = ct / p.pass_rows, within = ct % p.pass_rows;
+      const int t0 = (within % kConvRows) * 16, j = within / kConvRows;
+      double v = 0.0;
+#pragma unroll
+      for (int qq = 0; qq < 16; ++qq) v += bred[((t0 + qq) * NP + hp) * NS + j];
+      bpart[(size_t)blockIdx.x * kMaxM + ct] = v;
     }
   } else {
-    // ---------------- accumulator read-back: TMEM chunks -> fp32 registers -> partial D ----------------
+    // ---------------- accumulator read-back: TMEM chunks -> partial D ----------------
     const int dw = warp - (2 + kConvWarps);          // 0..7; the first read-back warp's index is a multiple of 4, so warp % 4 == dw % 4
     const int lg = dw & 3;                           // TMEM lane group this warp may read
     const int half = dw >> 2;                        // pieces of 16 columns: this warp takes piece 2 pp + half
     const int row = lg * 32 + lane;
     const int nchunks = (nsb + p.drain - 1) / p.drain;
-    constexpr int kPieces = kMaxN / 32;              // 6 pieces of 16 columns per warp
-    float accr[kPieces * 16];
+    const int rows_needed = (NT == 3) ? 2 * m : m;   // rows of D the combine reads
+    float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.npad;
+    // NT == 3 (N <= 192): the chunks are added in fp32 registers and stored once.  NT == 2
+    // (N <= 256): each chunk is added to the partial in global memory (first chunk: stored).
+    constexpr int kPieces = (NT == 3) ? 6 : 8;       // pieces of 16 columns per warp
+    float accr[(NT == 3) ? kPieces * 16 : 1];
+    if constexpr (NT == 3) {
 #pragma unroll
-    for (int j = 0; j < kPieces * 16; ++j) accr[j] = 0.f;
+      for (int j = 0; j < kPieces * 16; ++j) accr[j] = 0.f;
+    }
     bool ok = true;
     for (int c = 0; c < nchunks && ok; ++c) {
       const int buf = c & 1;
@@ -367,8 +423,19 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
                 "=r"(v[14]), "=r"(v[15])
               : "r"(taddr) : "memory");
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if constexpr (NT == 3) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) accr[pp * 16 + j] += __uint_as_float(v[j]);
+            for (int j = 0; j < 16; ++j) accr[pp * 16 + j] += __uint_as_float(v[j]);
+          } else if (row < rows_needed) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) {
+              float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (c > 0) acc4 = *reinterpret_cast<const float4 *>(dst + piece * 16 + j);   // this thread's own earlier store
+              acc4.x += __uint_as_float(v[j]); acc4.y += __uint_as_float(v[j + 1]);
+              acc4.z += __uint_as_float(v[j + 2]); acc4.w += __uint_as_float(v[j + 3]);
+              *reinterpret_cast<float4 *>(dst + piece * 16 + j) = acc4;
+            }
+          }
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -376,16 +443,17 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
       if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
     }
     if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
-    if (row < 2 * m) {
-      float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.npad;
+    if constexpr (NT == 3) {
+      if (row < rows_needed) {
 #pragma unroll
-      for (int pp = 0; pp < kPieces; ++pp) {
-        const int piece = 2 * pp + half;
-        if (piece * 16 < p.npad) {
+        for (int pp = 0; pp < kPieces; ++pp) {
+          const int piece = 2 * pp + half;
+          if (piece * 16 < p.npad) {
 #pragma unroll
-          for (int j = 0; j < 16; j += 4)
-            *reinterpret_cast<float4 *>(dst + piece * 16 + j) =
-                make_float4(accr[pp * 16 + j], accr[pp * 16 + j + 1], accr[pp * 16 + j + 2], accr[pp * 16 + j + 3]);
+            for (int j = 0; j < 16; j += 4)
+              *reinterpret_cast<float4 *>(dst + piece * 16 + j) =
+                  make_float4(accr[pp * 16 + j], accr[pp * 16 + j + 1], accr[pp * 16 + j + 2], accr[pp * 16 + j + 3]);
+          }
         }
       }
     }
@@ -400,22 +468,23 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
 }
 
 // Sum of the per-CTA partial D over the CTAs, in index order, in fp64: block a adds row a
-// (192 columns x 4 ranges of CTAs, the four range sums then added in range order) and, for
-// a < m, b_a.  The block that takes the last ticket forms G from the summed rows (the eight
-// term products listed at the top of this file), writes (G, b) and takes the step's decisions.
+// (its columns x 3 ranges of CTAs, the range sums then added in range order) and, for a < m,
+// b_a.  The block that takes the last ticket forms G from the summed rows (the term products
+// listed at the top of this file), writes (G, b) and takes the step's decisions.
 constexpr int kCombThreads = 768;
+constexpr int kCombRanges = kCombThreads / kMaxN;    // 3
 __global__ void __launch_bounds__(kCombThreads)
 umma_f32_combine_kernel(const float *__restrict__ partials, const double *__restrict__ bpart, int ctas, int npad,
-                        int m, double *__restrict__ dsum, double *__restrict__ gram, int *__restrict__ status,
+                        int m, int nt, double *__restrict__ dsum, double *__restrict__ gram, int *__restrict__ status,
                         const CdgTail tail) {
-  __shared__ double scan_sh[4 * 64 + 64 * 64];     // m <= 64 on this path
-  __shared__ double part[4][kMaxN];
+  extern __shared__ double scan_sh[];              // (4m + m*m) doubles: the scan's arrays and G
+  __shared__ double part[kCombRanges][kMaxN];
   __shared__ int is_last;
   cdg_grid_dep_wait();            // the partials come from the launch before this one
   const int a = blockIdx.x;
   const int col = threadIdx.x % kMaxN, qr = threadIdx.x / kMaxN;
   if (col < npad) {
-    const int c_lo = ctas * qr / 4, c_hi = ctas * (qr + 1) / 4;
+    const int c_lo = ctas * qr / kCombRanges, c_hi = ctas * (qr + 1) / kCombRanges;
     const float *P = partials + (size_t)a * npad + col;
     const size_t cs = (size_t)128 * npad;
     double v = 0.0;
@@ -432,13 +501,12 @@ umma_f32_combine_kernel(const float *__restrict__ partials, const double *__rest
   }
   __syncthreads();
   if (threadIdx.x < npad)
-    dsum[(size_t)a * kMaxN + threadIdx.x] =
-        ((part[0][threadIdx.x] + part[1][threadIdx.x]) + part[2][threadIdx.x]) + part[3][threadIdx.x];
+    dsum[(size_t)a * kMaxN + threadIdx.x] = (part[0][threadIdx.x] + part[1][threadIdx.x]) + part[2][threadIdx.x];
   if (a < m && threadIdx.x >= kCombThreads - 32) {
     // b_a: lane l adds the CTAs l, l + 32, ... in that order, then a fixed butterfly
     const int lane = threadIdx.x & 31;
     double v = 0.0;
-    for (int c = lane; c < ctas; c += 32) v += bpart[(size_t)c * 64 + a];
+    for (int c = lane; c < ctas; c += 32) v += bpart[(size_t)c * kMaxM + a];
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
     if (lane == 0) gram[(size_t)m * m + a] = v;
@@ -454,12 +522,18 @@ umma_f32_combine_kernel(const float *__restrict__ partials, const double *__rest
   const ScanSmem S = scan_smem(scan_sh, m);
   for (int e = threadIdx.x; e < m * m; e += kCombThreads) {
     const int k = e / m, i = e % m;
-    const double *Dk = dsum + (size_t)k * kMaxN, *Dmk = dsum + (size_t)(m + k) * kMaxN;
-    const double hh = __ldcg(Dk + i), hm = __ldcg(Dk + m + i), hl = __ldcg(Dk + 2 * m + i);
-    const double mh = __ldcg(Dmk + i), mm = __ldcg(Dmk + m + i), ml = __ldcg(Dmk + 2 * m + i);
-    const double lh = __ldcg(dsum + (size_t)i * kMaxN + 2 * m + k), lm = __ldcg(dsum + (size_t)(m + i) * kMaxN + 2 * m + k);
-    // smallest terms first
-    const double v = ((((ml + lm) + (hl + lh)) + mm) + (hm + mh)) + hh;
+    const double *Dk = dsum + (size_t)k * kMaxN;
+    double v;
+    if (nt == 3) {
+      const double *Dmk = dsum + (size_t)(m + k) * kMaxN;
+      const double hh = __ldcg(Dk + i), hm = __ldcg(Dk + m + i), hl = __ldcg(Dk + 2 * m + i);
+      const double mh = __ldcg(Dmk + i), mm = __ldcg(Dmk + m + i), ml = __ldcg(Dmk + 2 * m + i);
+      const double lh = __ldcg(dsum + (size_t)i * kMaxN + 2 * m + k), lm = __ldcg(dsum + (size_t)(m + i) * kMaxN + 2 * m + k);
+      v = ((((ml + lm) + (hl + lh)) + mm) + (hm + mh)) + hh;     // smallest terms first
+    } else {
+      const double hh = __ldcg(Dk + i), hl = __ldcg(Dk + m + i), lh = __ldcg(dsum + (size_t)i * kMaxN + m + k);
+      v = (hl + lh) + hh;
+    }
     S.g[e] = v;
     gram[e] = v;
   }
@@ -476,65 +550,86 @@ typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, voi
                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 2-D fp32 map over `rows` rows of d columns, box [box_rows][cols], no swizzle; columns past d read as zeros
-bool encode_f32(CUtensorMap *map, const void *base, long long d, int rows, int box_rows, int cols) {
+// 2-D map over `rows` rows of d columns of fp32 or bf16, box [box_rows][cols], no swizzle; columns
+// past d read as zeros
+bool encode_rows(CUtensorMap *map, const void *base, long long d, int rows, int box_rows, int cols, int elem_bytes) {
   EncodeFn fn = (EncodeFn)cdg_tensor_map_encoder();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)d * 4};
+  cuuint64_t strides[1] = {(cuuint64_t)d * elem_bytes};
   cuuint32_t box[2] = {(cuuint32_t)cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  return fn(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NS>
-cudaError_t f32_launch(cdgrab_ctx *h, const CUtensorMap &tm_g, const F32Params &p, cudaStream_t st) {
-  return cdg_launch_dep(h, gram_umma_f32_kernel<NS>, dim3(h->f32_ctas), dim3(kThreads), h->f32_smem, st, tm_g, h->tm_f32r,
-                        p, h->umma_partials, h->f32_bpart, h->status);
+template <typename T, int NT, int NS, int NP>
+cudaError_t terms_launch(cdgrab_ctx *h, const CUtensorMap &tm_g, const F32Params &p, cudaStream_t st) {
+  return cdg_launch_dep(h, gram_umma_f32_kernel<T, NT, NS, NP>, dim3(h->f32_ctas), dim3(kThreads), h->f32_smem, st, tm_g,
+                        h->tm_f32r, p, h->umma_partials, h->f32_bpart, h->status);
 }
 
-cudaError_t f32_open_limits() {
-  cudaError_t e = cdg_open_smem_limit(gram_umma_f32_kernel<1>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<2>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<3>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<4>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<5>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<6>);
+cudaError_t terms_open_limits() {
+  cudaError_t e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 1, 1>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 2, 1>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 3, 1>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 4, 1>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 5, 1>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 6, 1>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 4, 2>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 5, 2>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 6, 2>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(umma_f32_combine_kernel);
   return e;
 }
 
+// bf16 gradients: 65..128 workers take two converter passes of pass_rows rows each
+inline int bf16_pass_rows(int m) { return (((m + 1) / 2) + 7) & ~7; }
+
 }  // namespace
 
+// fp32: rows whose pitch is a multiple of 16 bytes; 2m <= 128 rows of hi and mid terms fill the MMA's M.
+// bf16: 65 <= m <= 128 (up to 64 workers the raw rows go through the MMA as they lie in HBM).
 bool cdg_umma_f32_supported(int m, long long d) {
-  // rows whose pitch is a multiple of 16 bytes; 2m <= 128 rows of hi and mid terms fill the MMA's M
   return m >= 1 && m <= 64 && d % 4 == 0 && d >= 4096 && d < (1ll << 31) - 512 && cdg_tensor_map_encoder() != nullptr;
+}
+bool cdg_umma_terms_bf16_supported(int m, long long d) {
+  return m > 64 && m <= kMaxM && d % 8 == 0 && d >= 4096 && d < (1ll << 31) - 512 && cdg_tensor_map_encoder() != nullptr;
 }
 
 int cdg_umma_f32_setup(cdgrab_ctx *h) {
   const int m = h->m;
-  h->f32_npad = ((3 * m + 15) / 16) * 16;
+  const int nt = (h->dtype == CDGRAB_F32) ? 3 : 2;
+  const size_t es = (h->dtype == CDGRAB_F32) ? 4 : 2;
+  h->f32_nt = nt;
+  h->f32_npad = ((nt * m + 15) / 16) * 16;
   const int rows8 = (2 * m + 7) & ~7;
   const int op_rows = h->f32_npad > 128 ? h->f32_npad : 128;
   const size_t op_bytes = (size_t)op_rows * 128;
-  // stage width: 128 columns (512 contiguous bytes per row and copy) while two such stages fit beside
-  // three operand buffers, else 64; CDGRAB_F32_NSUB overrides
+  // stage width: 128 columns (512 or 256 contiguous bytes per row and copy) while two such stages fit
+  // beside the operand buffers (three, or two when three leave no room), else 64;
+  // CDGRAB_F32_NSUB / CDGRAB_F32_NOPS override
   int nsub = 2, nops = 3;
+  bool nops_forced = false;
   if (const char *e = getenv("CDGRAB_F32_NSUB")) {
     const int v = atoi(e);
     if (v == 1 || v == 2 || v == 4) nsub = v;
   }
   if (const char *e = getenv("CDGRAB_F32_NOPS")) {
     const int v = atoi(e);
-    if (v >= 2 && v <= kMaxOps) nops = v;
+    if (v >= 2 && v <= kMaxOps) { nops = v; nops_forced = true; }
   }
-  const size_t budget = (size_t)kCdgMaxDynSmem - 1024 - 12 * 1024;   // static shared memory: barriers and the b sums
-  size_t stage_bytes = (size_t)(rows8 + 1) * nsub * kBlockCols * 4;
+  const size_t budget = (size_t)kCdgMaxDynSmem - 1024 - 4 * 1024;   // static shared memory: the barriers
+  auto stage_of = [&](int ns) { return (size_t)rows8 * ns * kBlockCols * es + (size_t)ns * kBlockCols * 4; };
+  size_t stage_bytes = stage_of(nsub);
+  if (!nops_forced && nops > 2 && budget < nops * op_bytes + 2 * stage_bytes) nops = 2;
   while (nsub > 1 && budget < nops * op_bytes + 2 * stage_bytes) {
     nsub >>= 1;
-    stage_bytes = (size_t)(rows8 + 1) * nsub * kBlockCols * 4;
+    stage_bytes = stage_of(nsub);
   }
+  if (budget < nops * op_bytes + 2 * stage_bytes) return CDGRAB_ERR_INVALID;
   int stages = (int)((budget - nops * op_bytes) / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (const char *e = getenv("CDGRAB_F32_STAGES")) {
@@ -546,8 +641,9 @@ int cdg_umma_f32_setup(cdgrab_ctx *h) {
   h->f32_nops = nops;
   h->f32_stages = stages;
   h->f32_smem = 1024 + nops * op_bytes + stages * stage_bytes;
-  // TMEM chunk: about 512 columns (fp32 inputs are held to the 1e-6 sign tolerance); CDGRAB_UMMA_DRAIN overrides
-  h->f32_drain = 512 / kBlockCols;
+  // TMEM chunk: about 512 columns for fp32 inputs (held to the 1e-6 sign tolerance), 4096 for bf16;
+  // CDGRAB_UMMA_DRAIN overrides
+  h->f32_drain = (nt == 3 ? 512 : 4096) / kBlockCols;
   if (const char *e = getenv("CDGRAB_UMMA_DRAIN")) {
     const int v = atoi(e);
     if (v >= 1 && v <= (1 << 20)) h->f32_drain = v;
@@ -556,17 +652,17 @@ int cdg_umma_f32_setup(cdgrab_ctx *h) {
   h->f32_ctas = (int)(nblk < h->num_sms ? nblk : h->num_sms);
   const size_t pbytes = sizeof(float) * 128 * (size_t)h->f32_npad * h->f32_ctas;
   if (cdg_alloc(h, &h->umma_partials, pbytes) != cudaSuccess ||
-      cdg_alloc(h, &h->f32_bpart, sizeof(double) * 64 * (size_t)h->f32_ctas) != cudaSuccess ||
+      cdg_alloc(h, &h->f32_bpart, sizeof(double) * kMaxM * (size_t)h->f32_ctas) != cudaSuccess ||
       cdg_alloc(h, &h->f32_dsum, sizeof(double) * 128 * kMaxN) != cudaSuccess) {
     cudaGetLastError();
     return CDGRAB_ERR_NOMEM;
   }
   if (cudaMemset(h->umma_partials, 0, pbytes) != cudaSuccess ||
-      cudaMemset(h->f32_bpart, 0, sizeof(double) * 64 * (size_t)h->f32_ctas) != cudaSuccess ||
+      cudaMemset(h->f32_bpart, 0, sizeof(double) * kMaxM * (size_t)h->f32_ctas) != cudaSuccess ||
       cudaMemset(h->f32_dsum, 0, sizeof(double) * 128 * kMaxN) != cudaSuccess)
     return CDGRAB_ERR_CUDA;
-  if (!encode_f32(&h->tm_f32r, h->r, h->d, 1, 1, nsub * kBlockCols)) return CDGRAB_ERR_CUDA;
-  if (f32_open_limits() != cudaSuccess) {
+  if (!encode_rows(&h->tm_f32r, h->r, h->d, 1, 1, nsub * kBlockCols, 4)) return CDGRAB_ERR_CUDA;
+  if (terms_open_limits() != cudaSuccess) {
     cudaGetLastError();
     return CDGRAB_ERR_CUDA;
   }
@@ -586,10 +682,11 @@ void cdg_umma_f32_teardown(cdgrab_ctx *h) {
 }
 
 cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStream_t st) {
+  const int es = (h->dtype == CDGRAB_F32) ? 4 : 2;
   int slot = h->tm_f32g.find(grads);
   if (slot < 0) {
     slot = h->tm_f32g.victim();
-    if (!encode_f32(&h->tm_f32g.maps[slot][0], grads, h->d, 2 * h->m, 8, h->f32_nsub * kBlockCols))
+    if (!encode_rows(&h->tm_f32g.maps[slot][0], grads, h->d, 2 * h->m, 8, h->f32_nsub * kBlockCols, es))
       return cudaErrorInvalidValue;
     h->tm_f32g.commit(slot, grads);
   }
@@ -604,22 +701,34 @@ cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStrea
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     const CUtensorMap &tm = h->tm_f32g.maps[slot][0];
-    const int ns = (h->m + kConvRows - 1) / kConvRows;       // rows per converter thread
     static_assert(kRowSlots <= 6, "one instantiation per slot count");
-    switch (ns) {
-      case 1: f32_launch<1>(h, tm, p, st); break;
-      case 2: f32_launch<2>(h, tm, p, st); break;
-      case 3: f32_launch<3>(h, tm, p, st); break;
-      case 4: f32_launch<4>(h, tm, p, st); break;
-      case 5: f32_launch<5>(h, tm, p, st); break;
-      default: f32_launch<6>(h, tm, p, st); break;
+    if (h->f32_nt == 3) {
+      p.pass_rows = (h->m + 7) & ~7;
+      const int ns = (h->m + kConvRows - 1) / kConvRows;       // rows per converter thread
+      switch (ns) {
+        case 1: terms_launch<float, 3, 1, 1>(h, tm, p, st); break;
+        case 2: terms_launch<float, 3, 2, 1>(h, tm, p, st); break;
+        case 3: terms_launch<float, 3, 3, 1>(h, tm, p, st); break;
+        case 4: terms_launch<float, 3, 4, 1>(h, tm, p, st); break;
+        case 5: terms_launch<float, 3, 5, 1>(h, tm, p, st); break;
+        default: terms_launch<float, 3, 6, 1>(h, tm, p, st); break;
+      }
+    } else {
+      p.pass_rows = bf16_pass_rows(h->m);                      // 40..64
+      const int ns = (p.pass_rows + kConvRows - 1) / kConvRows;
+      switch (ns) {
+        case 4: terms_launch<__nv_bfloat16, 2, 4, 2>(h, tm, p, st); break;
+        case 5: terms_launch<__nv_bfloat16, 2, 5, 2>(h, tm, p, st); break;
+        default: terms_launch<__nv_bfloat16, 2, 6, 2>(h, tm, p, st); break;
+      }
     }
   }
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
-    cdg_launch_dep(h, umma_f32_combine_kernel, dim3(2 * h->m), dim3(kCombThreads), 0, st,
+    const int rows = (h->f32_nt == 3) ? 2 * h->m : h->m;
+    cdg_launch_dep(h, umma_f32_combine_kernel, dim3(rows), dim3(kCombThreads), scan_smem_bytes(h->m, true), st,
                    (const float *)h->umma_partials, (const double *)h->f32_bpart, h->f32_ctas, h->f32_npad, h->m,
-                   h->f32_dsum, h->gram, h->status, cdg_tail_of(h, h->umma_fused));
+                   h->f32_nt, h->f32_dsum, h->gram, h->status, cdg_tail_of(h, h->umma_fused));
   }
   return cudaGetLastError();
 }

@@ -117,3 +117,37 @@ def test_umma_long_rows_with_common_mean(mean, scale, monkeypatch):
         assert rep.raw_agreement == 1.0
     finally:
         pr.close()
+
+
+@pytest.mark.parametrize("m,n,d", [
+    (65, 4, 8192),            # first m past one 128-row tile of raw rows; fewer blocks than SMs
+    (72, 4, 100_000),         # passes of 40 rows
+    (73, 4, 70_008),          # ragged last block (d a multiple of 8 only)
+    (100, 4, 300_000),
+    (128, 4, 64 * 148 * 2 + 8),   # the largest m: N = 256, both TMEM buffers full width
+    (128, 6, 1_000_000),      # several accumulator chunks per CTA
+])
+def test_bf16_more_than_64_workers_on_the_tensor_cores(m, n, d):
+    """bf16 gradients with 65..128 workers: the differences go through the MMA as two bf16 terms
+    each, formed inside the kernel; the bf16 sign tolerance (1e-3) applies."""
+    rep = run(m, n, d, seed=m + d % 5)
+    print(f"umma bf16 wide m={m} n={n} d={d}:", rep)
+    assert rep.raw_agreement > 0.9
+
+
+def test_bf16_wide_matches_the_fma_route(monkeypatch):
+    """Same steps with the term-splitting kernel and with the blocked FMA Gram: same signs, same r."""
+    m, n, d = 96, 6, 131_072
+    out = {}
+    for wide in ("1", "0"):
+        monkeypatch.setenv("CDGRAB_UMMA_BF16_WIDE", wide)
+        with binding.CdGrab(m, n, d, "bf16") as h:
+            assert h.path == ("umma" if wide == "1" else "fma")
+            h.begin_epoch()
+            for k in range(n // 2):
+                h.step(grads(m, d, 900 + k, mean=0.2))
+            out[wide] = (h.signs().cpu(), h.r().cpu(), h.margins().cpu())
+            assert h.status() == binding.OK
+    assert torch.equal(out["1"][0], out["0"][0])
+    assert torch.equal(out["1"][1], out["0"][1])
+    np.testing.assert_allclose(out["1"][2].numpy(), out["0"][2].numpy(), rtol=2e-3, atol=1e-5)
