@@ -830,7 +830,9 @@ __device__ __forceinline__ float ft_update_tile(const T *gt, const float *rt, co
   return out;
 }
 
-template <typename T, int M>
+// FUSE: the launch also applies the update the step before left open (see FtTree); a separate
+// instantiation, so that the plain pass 1 carries none of it.
+template <typename T, int M, bool FUSE>
 __global__ void __launch_bounds__(kFtThreads, 1)
 gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
                     const __grid_constant__ CUtensorMap tm_p, int m, long long d, int stages, int box_rows, int contiguous,
@@ -856,7 +858,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   const uint32_t g_bytes = (uint32_t)nbox * box_bytes;            // rows past 2m are zero-filled
   const uint32_t r_bytes = kFtCols * (uint32_t)sizeof(float);
   // rows, then the r tile, then (deferred update) the rows of the step before
-  const uint32_t stage_bytes = g_bytes + r_bytes + (tree.fuse_prev ? g_bytes : 0u);
+  const uint32_t stage_bytes = g_bytes + r_bytes + (FUSE ? g_bytes : 0u);
   const long long ntiles = (d + kFtCols - 1) / kFtCols;
   // tiles of this CTA: a contiguous range, or every gridDim.x-th tile
   const long long t_lo = contiguous ? ntiles * blockIdx.x / gridDim.x : blockIdx.x;
@@ -881,7 +883,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
   cdg_grid_dep_wait();      // r is written by the launch before this one
   FT_STAMP(threadIdx.x == 0, 1);
   const long long deadline = clock64() + kCdgWaitCycles;
-  if (tree.fuse_prev) {     // the signs the launch before this one decided
+  if constexpr (FUSE) {     // the signs the launch before this one decided
     if (threadIdx.x < m) ssh[threadIdx.x] = (float)tree.prev_signs[(size_t)threadIdx.x * tree.prev_stride];
     __syncthreads();
   }
@@ -915,7 +917,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
         mbar_expect_tx(full, stage_bytes);
         for (int q = 0; q < nbox; ++q) tma_load_2d(dst + q * box_bytes, &tm_g, col, q * box_rows, full);
         tma_load_2d(dst + g_bytes, &tm_r, col, 0, full);
-        if (tree.fuse_prev)
+        if constexpr (FUSE)
           for (int q = 0; q < nbox; ++q) tma_load_2d(dst + g_bytes + r_bytes + q * box_bytes, &tm_p, col, q * box_rows, full);
         issued = it + 1;
         if (++s == stages) { s = 0; ++turn; }
@@ -939,7 +941,7 @@ gram_fma_tma_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
       FT_STAMP(threadIdx.x == 0 && it == 0, 2);
       const T *gt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes);
       float *rt = reinterpret_cast<float *>(base_ptr + (size_t)s * stage_bytes + g_bytes);
-      if (tree.fuse_prev && group == 1) {
+      if (FUSE && group == 1) {
         // the update the step before left open, on this thread's column; the new value replaces
         // the old one in the stage so that b below is formed against it
         const T *pt = reinterpret_cast<const T *>(base_ptr + (size_t)s * stage_bytes + g_bytes + r_bytes);
@@ -1152,7 +1154,8 @@ static bool ft_encode(CUtensorMap *map, const void *base, long long d, int rows,
 
 template <typename T, int M>
 static cudaError_t ft_set_smem(size_t smem) {
-  return cdg_open_smem_limit(gram_fma_tma_kernel<T, M>);
+  const cudaError_t e = cdg_open_smem_limit(gram_fma_tma_kernel<T, M, false>);
+  return e != cudaSuccess ? e : cdg_open_smem_limit(gram_fma_tma_kernel<T, M, true>);
 }
 
 int cdg_fma_tma_setup(cdgrab_ctx *h) {
@@ -1272,14 +1275,15 @@ static cudaError_t launch_gram_fma_tma_t(cdgrab_ctx *h, const CUtensorMap &tm_g,
       ++na;
     }
     cfg.attrs = at; cfg.numAttrs = na;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, tm_p, h->m, h->d, stages,
+    auto kernel = tm_prev ? gram_fma_tma_kernel<T, M, true> : gram_fma_tma_kernel<T, M, false>;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tm_g, h->tm_fr, tm_p, h->m, h->d, stages,
                                        h->fma_tma_boxrows, h->fma_tma_contig, h->partials, h->status, tail, tree);
     if (e != cudaSuccess && whole && h->ft_coop && na == 2) {
       // a driver that does not take both attributes together: cooperative alone from now on
       cudaGetLastError();
       h->ft_coop_no_pdl = 1;
       cfg.numAttrs = 1;
-      e = cudaLaunchKernelEx(&cfg, gram_fma_tma_kernel<T, M>, tm_g, h->tm_fr, tm_p, h->m, h->d, stages,
+      e = cudaLaunchKernelEx(&cfg, kernel, tm_g, h->tm_fr, tm_p, h->m, h->d, stages,
                              h->fma_tma_boxrows, h->fma_tma_contig, h->partials, h->status, tail, tree);
     }
     if (e != cudaSuccess) return e;

@@ -520,30 +520,46 @@ umma_f32_combine_kernel(const float *__restrict__ partials, const double *__rest
   if (!is_last) return;
   __threadfence();
   const ScanSmem S = scan_smem(scan_sh, m);
-  for (int e = threadIdx.x; e < m * m; e += kCombThreads) {
-    const int k = e / m, i = e % m;
-    const double *Dk = dsum + (size_t)k * kMaxN;
-    double v;
-    if (nt == 3) {
-      const double *Dmk = dsum + (size_t)(m + k) * kMaxN;
-      const double hh = __ldcg(Dk + i), hm = __ldcg(Dk + m + i), hl = __ldcg(Dk + 2 * m + i);
-      const double mh = __ldcg(Dmk + i), mm = __ldcg(Dmk + m + i), ml = __ldcg(Dmk + 2 * m + i);
-      const double lh = __ldcg(dsum + (size_t)i * kMaxN + 2 * m + k), lm = __ldcg(dsum + (size_t)(m + i) * kMaxN + 2 * m + k);
-      v = ((((ml + lm) + (hl + lh)) + mm) + (hm + mh)) + hh;     // smallest terms first
-    } else {
-      const double hh = __ldcg(Dk + i), hl = __ldcg(Dk + m + i), lh = __ldcg(dsum + (size_t)i * kMaxN + m + k);
-      v = (hl + lh) + hh;
+  // four entries per thread and round, every load of the round in flight before the first sum
+  for (int e0 = threadIdx.x; e0 < m * m; e0 += 4 * kCombThreads) {
+    double x[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * kCombThreads;
+      if (e < m * m) {
+        const int k = e / m, i = e % m;
+        const double *Dk = dsum + (size_t)k * kMaxN;
+        if (nt == 3) {
+          const double *Dmk = dsum + (size_t)(m + k) * kMaxN;
+          x[u][0] = __ldcg(Dk + i); x[u][1] = __ldcg(Dk + m + i); x[u][2] = __ldcg(Dk + 2 * m + i);      // hh hm hl
+          x[u][3] = __ldcg(Dmk + i); x[u][4] = __ldcg(Dmk + m + i); x[u][5] = __ldcg(Dmk + 2 * m + i);   // mh mm ml
+          x[u][6] = __ldcg(dsum + (size_t)i * kMaxN + 2 * m + k);                                        // lh
+          x[u][7] = __ldcg(dsum + (size_t)(m + i) * kMaxN + 2 * m + k);                                  // lm
+        } else {
+          x[u][0] = __ldcg(Dk + i); x[u][1] = __ldcg(Dk + m + i);                                        // hh hl
+          x[u][2] = __ldcg(dsum + (size_t)i * kMaxN + m + k);                                            // lh
+        }
+      }
     }
-    S.g[e] = v;
-    gram[e] = v;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u * kCombThreads;
+      if (e < m * m) {
+        // smallest terms first
+        const double v = (nt == 3) ? ((((x[u][5] + x[u][7]) + (x[u][2] + x[u][6])) + x[u][4]) + (x[u][1] + x[u][3])) + x[u][0]
+                                   : (x[u][1] + x[u][2]) + x[u][0];
+        S.g[e] = v;
+        gram[e] = v;
+      }
+    }
   }
   for (int j = threadIdx.x; j < m; j += kCombThreads) S.t[j] = __ldcg(gram + (size_t)m * m + j);
   if (threadIdx.x == 0) *tail.ticket = 0u;                    // ready for the next launch
   if (!tail.enabled) return;
   scan_load_pairs(S, tail.perm_cur, m, tail.n, tail.k);
   __syncthreads();
-  scan_decide_and_write(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
-                        tail.rule);
+  scan_decide_and_write<4>(S, S.g, m, tail.n, tail.k, tail.perm_next, tail.signs, tail.margins, tail.rnorm2, status,
+                           tail.rule);
 }
 
 typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,

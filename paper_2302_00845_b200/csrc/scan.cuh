@@ -115,11 +115,75 @@ __device__ __forceinline__ void scan_load_pairs(const ScanSmem &S, const int32_t
   }
 }
 
+// The chain of decisions in registers for m <= 32 Q: lane j holds t_j, t_{j+32}, ...; row i of G is
+// fetched one decision ahead.  Only what the next decision depends on sits in the loop (broadcast
+// t_i, decide, one multiply-add per held entry); signs, norms and the non-finite check follow from
+// the final t_j of every lane afterwards, in parallel.  Warp 0 only; rn2 = ||r||^2 before the
+// step on entry, after it on return.
+template <int Q>
+__device__ __forceinline__ void scan_chain_regs(const ScanSmem &S, const double *G, int m, const CdgRule &rule,
+                                                double &rn2, bool &bad, int &oob, int lane) {
+  bool h[Q];
+  double t[Q], g[Q], dg[Q];
+#pragma unroll
+  for (int q = 0; q < Q; ++q) {
+    const int j = lane + 32 * q;
+    h[q] = j < m;
+    t[q] = h[q] ? S.t[j] : 0.0;
+    g[q] = h[q] ? G[j] : 0.0;
+    dg[q] = h[q] ? G[(size_t)j * m + j] : 0.0;
+  }
+#pragma unroll
+  for (int seg = 0; seg < Q; ++seg) {
+    const int i_hi = (m < 32 * (seg + 1)) ? m : 32 * (seg + 1);
+    for (int i = 32 * seg; i < i_hi; ++i) {
+      double nx[Q];
+#pragma unroll
+      for (int q = 0; q < Q; ++q) nx[q] = (i + 1 < m && h[q]) ? G[(size_t)(i + 1) * m + lane + 32 * q] : 0.0;
+      const double ti = __shfl_sync(0xffffffffu, t[seg], i & 31);
+      // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0 (or the randomized rule)
+      int dummy = 0;
+      const double sd = rule.randomized ? (double)cdg_decide(rule, i, ti, dummy) : ((ti < 0.0) ? 1.0 : -1.0);
+      // every later t_j gains s_i G_ij, summed in the order i = 0, 1, ...
+#pragma unroll
+      for (int q = 0; q < Q; ++q) {
+        if (lane + 32 * q > i) t[q] = fma(sd, g[q], t[q]);
+        g[q] = nx[q];
+      }
+    }
+  }
+  // lane j now holds t_j = <r_{j-1}, c_j> (and t_{j+32}, ...); its sign follows from it alone.
+  // ||r||^2 seen by worker j: ||r_0||^2 + sum_{i<j} (2 s_i t_i + G_ii), an exclusive prefix sum over
+  // the lanes, 32 workers after 32 workers
+#pragma unroll
+  for (int q = 0; q < Q; ++q) {
+    const int j = lane + 32 * q;
+    const int sj = h[q] ? cdg_decide(rule, j, t[q], oob) : 0;
+    bad = bad || (h[q] && !(isfinite(t[q]) && isfinite(dg[q])));
+    const double inc = h[q] ? 2.0 * (double)sj * t[q] + dg[q] : 0.0;
+    double pre = inc;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const double up = __shfl_up_sync(0xffffffffu, pre, off);
+      if (lane >= off) pre += up;
+    }
+    const double before = rn2 + (pre - inc);
+    if (h[q]) { S.s[j] = sj; S.rn[j] = before > 0.0 ? before : 0.0; S.t[j] = t[q]; }
+    rn2 += __shfl_sync(0xffffffffu, pre, 31);
+  }
+  if (rn2 < 0.0) rn2 = 0.0;
+  bad = __any_sync(0xffffffffu, bad);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) oob += __shfl_xor_sync(0xffffffffu, oob, off);
+}
+
 // S.t = b, S.p = pairs and G (shared or global, row-major [m][m]) must be ready and visible
 // to the block (barrier before the call).  Warp 0 decides, the block writes out.
 // rn2_in: ||r||^2 before the step when the caller fetched it ahead of time, else negative
 // (the routine then reads *rnorm2 itself).  write_out = false: decide only (signs in S.s),
-// nothing is written to global memory.
+// nothing is written to global memory.  QMAX: lanes hold up to QMAX entries of the chain in
+// registers (m <= 32 QMAX); beyond that the chain runs through shared memory.
+template <int QMAX = 2>
 __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const double *G, int m, int n, int k,
                                                       int32_t *__restrict__ perm_next, int8_t *__restrict__ signs,
                                                       float *__restrict__ margins, double *__restrict__ rnorm2,
@@ -131,52 +195,18 @@ __device__ __forceinline__ void scan_decide_and_write(const ScanSmem &S, const d
     double rn2 = (rn2_in >= 0.0) ? rn2_in : *rnorm2;
     bool bad = false;
     int oob = 0;
+    bool in_regs = false;
     if (m <= 64) {
-      // The chain stays in registers: lane j holds t_j and t_{j+32}; row i of G is fetched one
-      // decision ahead.  Only what the next decision depends on sits in the loop (broadcast t_i,
-      // decide, one multiply-add per lane); signs, norms and the non-finite check follow from the
-      // final t_j of every lane afterwards, in parallel.
-      const bool h0 = lane < m, h1 = lane + 32 < m;
-      double t0 = h0 ? S.t[lane] : 0.0, t1 = h1 ? S.t[lane + 32] : 0.0;
-      double g0 = h0 ? G[lane] : 0.0, g1 = h1 ? G[lane + 32] : 0.0;
-      const double d0 = h0 ? G[(size_t)lane * m + lane] : 0.0, d1 = h1 ? G[(size_t)(lane + 32) * m + lane + 32] : 0.0;
-      for (int i = 0; i < m; ++i) {
-        double n0 = 0.0, n1 = 0.0;
-        if (i + 1 < m) {
-          if (h0) n0 = G[(size_t)(i + 1) * m + lane];
-          if (h1) n1 = G[(size_t)(i + 1) * m + lane + 32];
-        }
-        const double ti = __shfl_sync(0xffffffffu, (i < 32) ? t0 : t1, i & 31);
-        // Algorithm 6: +1 iff ||r + c|| < ||r - c||  <=>  <r,c> < 0 (or the randomized rule)
-        int dummy = 0;
-        const double sd = rule.randomized ? (double)cdg_decide(rule, i, ti, dummy) : ((ti < 0.0) ? 1.0 : -1.0);
-        // every later t_j gains s_i G_ij, summed in the order i = 0, 1, ...
-        if (lane > i) t0 = fma(sd, g0, t0);
-        if (lane + 32 > i) t1 = fma(sd, g1, t1);
-        g0 = n0; g1 = n1;
+      scan_chain_regs<2>(S, G, m, rule, rn2, bad, oob, lane);
+      in_regs = true;
+    }
+    if constexpr (QMAX >= 4) {
+      if (!in_regs && m <= 128) {
+        scan_chain_regs<4>(S, G, m, rule, rn2, bad, oob, lane);
+        in_regs = true;
       }
-      // lane j now holds t_j = <r_{j-1}, c_j> (and t_{j+32}); its sign follows from it alone
-      const int s0 = h0 ? cdg_decide(rule, lane, t0, oob) : 0, s1 = h1 ? cdg_decide(rule, lane + 32, t1, oob) : 0;
-      bad = (h0 && !(isfinite(t0) && isfinite(d0))) || (h1 && !(isfinite(t1) && isfinite(d1)));
-      // ||r||^2 seen by worker j: ||r_0||^2 + sum_{i<j} (2 s_i t_i + G_ii), an exclusive prefix sum
-      // over the lanes (first the lower 32 workers, then the upper ones)
-      double inc0 = h0 ? 2.0 * (double)s0 * t0 + d0 : 0.0, inc1 = h1 ? 2.0 * (double)s1 * t1 + d1 : 0.0;
-      double p0 = inc0, p1 = inc1;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const double u0 = __shfl_up_sync(0xffffffffu, p0, off), u1 = __shfl_up_sync(0xffffffffu, p1, off);
-        if (lane >= off) { p0 += u0; p1 += u1; }
-      }
-      const double tot0 = __shfl_sync(0xffffffffu, p0, 31);
-      const double before0 = rn2 + (p0 - inc0), before1 = rn2 + tot0 + (p1 - inc1);
-      if (h0) { S.s[lane] = s0; S.rn[lane] = before0 > 0.0 ? before0 : 0.0; S.t[lane] = t0; }
-      if (h1) { S.s[lane + 32] = s1; S.rn[lane + 32] = before1 > 0.0 ? before1 : 0.0; S.t[lane + 32] = t1; }
-      rn2 = rn2 + tot0 + __shfl_sync(0xffffffffu, p1, 31);
-      if (rn2 < 0.0) rn2 = 0.0;
-      bad = __any_sync(0xffffffffu, bad);
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) oob += __shfl_xor_sync(0xffffffffu, oob, off);
-    } else {
+    }
+    if (!in_regs) {
       for (int i = 0; i < m; ++i) {
         const double ti = S.t[i];
         const double gii = G[(size_t)i * m + i];
