@@ -179,7 +179,7 @@ NCU_TRAFFIC.update({
     ("gram", "lstm"): {"bytes": 5.664448e+08 * (13_500_000 / 4_194_304), "files": ["kernels_umma.cu", "ptx.cuh"], "source": "c889f8e27a23db29"},
     ("update", "lstm"): {"bytes": 5.820989e+08 * (13_500_000 / 4_194_304), "files": ["kernels_generic.cu"], "source": "1cffb536a83d70ae"},
     # mid, at full size.  Pass 2: bytes of a cold launch (ncu flushes L2 between replays)
-    ("gram", "mid"): {"bytes": 1.445166e+08, "files": ["kernels_fma.cu", "ptx.cuh"], "source": "93237938826dd79f"},
+    ("gram", "mid"): {"bytes": 1.445166e+08, "files": ["kernels_fma.cu", "ptx.cuh"], "source": "76d0347672d85fa9"},
     ("update", "mid"): {"bytes": 1.415913e+08, "files": ["kernels_generic.cu"], "source": "1cffb536a83d70ae"},
 })
 

@@ -1190,7 +1190,7 @@ int cdg_fma_tma_setup(cdgrab_ctx *h) {
   // CDGRAB_DEFER=1: cdgrab_step_many folds pass 2 of a step into pass 1 of the next one.  Off by
   // default: measured slower than two launches per step at every size tried (the update's loads and
   // adds land on the threads that also own b, and a stage holds two steps' rows, so the ring is half
-  // as deep): 91 against 63 us per step at m = 16, d = 2^20 fp32; 723 against 439 us at m = 16,
+  // as deep): 91 against 52 us per step at m = 16, d = 2^20 fp32; 773 against 436 us at m = 16,
   // d = 13.5 M bf16.
   h->fma_tma_defer = 0;
   if (const char *e = getenv("CDGRAB_DEFER")) h->fma_tma_defer = atoi(e) ? 1 : 0;
