@@ -14,7 +14,7 @@ LIB = os.path.join(HERE, "libcdgrab.so")
 #   --stamp  -DCDGRAB_STAMP  kernels record phase time stamps (libcdgrab_stamp.so)
 #   --debug  -DCDGRAB_DEBUG  index checks and guard words around scratch (libcdgrab_debug.so)
 VARIANTS = {"stamp": ("-DCDGRAB_STAMP", "libcdgrab_stamp.so"), "debug": ("-DCDGRAB_DEBUG", "libcdgrab_debug.so")}
-SOURCES = ["api.cu", "kernels_generic.cu", "kernels_fma.cu", "kernels_umma.cu", "kernels_umma_f32.cu", "noalloc.cu", "herding.cu", "kernels_indep.cu", "kernels_block.cu", "kernels_literal.cu"]
+SOURCES = ["api.cu", "kernels_generic.cu", "kernels_fma.cu", "kernels_umma.cu", "kernels_umma_f32.cu", "noalloc.cu", "herding.cu", "kernels_indep.cu", "kernels_block.cu", "kernels_literal.cu", "kernels_small.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",

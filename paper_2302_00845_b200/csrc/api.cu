@@ -175,7 +175,7 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
 
   // ---- choose the path ------------------------------------------------------------
   const size_t step_bytes = 2 * (size_t)m * (size_t)d * elem_size(dtype);
-  const bool fused_ok = cdg_fused_supported(m, d, dtype);
+  const bool fused_ok = cdg_fused_supported(m, d, dtype) || cdg_small_supported(m, d, dtype);
   // bf16 with 65..128 workers: the term-splitting tensor-core kernel (CDGRAB_UMMA_BF16_WIDE=0: not used)
   const char *wide_env = getenv("CDGRAB_UMMA_BF16_WIDE");
   const bool umma_wide = dtype == CDGRAB_BF16 && cdg_umma_terms_bf16_supported(m, d) && !(wide_env && atoi(wide_env) == 0);
@@ -187,9 +187,16 @@ static int create_impl(int m, int n, long long d, int dtype, int mode, cdgrab_t 
     // single-launch step up to 1024 columns, and the four launches of the generic two-pass route
     // for more than 16 workers while m*d stays small (measured per step with cold caches: 10.2 against
     // 12.5 us at m = 4, d = 1024; 29.5 against 60.5 us at m = 32, d = 1024; 70 against 57 us at m = 64, d = 2048)
-    if (literal_ok && ((m <= 16 && d <= 1024) || (m > 16 && d < 4096 && (long long)m * d <= 65536)))
+    // More than 16 workers with rows of at most 64 columns (the synthetic herding study: 16) take
+    // the Gram form in one CTA instead: every dot product in parallel rather than one block-wide
+    // reduction per worker (12.8 / 18.6 / 34.9 against 17.2 / 35.0 / 62.1 us per step at m = 20 /
+    // 50 / 100, d = 16); with longer rows its one thread per entry loses to the literal form
+    // (76 against 31 us at m = 32, d = 1024).
+    const bool small_auto = cdg_small_supported(m, d, dtype) && d <= 64 && !shard;
+    if (literal_ok && !small_auto && ((m <= 16 && d <= 1024) || (m > 16 && d < 4096 && (long long)m * d <= 65536)))
       path = CDGRAB_PATH_LITERAL;
-    else if (fused_ok && step_bytes <= (size_t)768 * 1024 && !shard) path = CDGRAB_PATH_FUSED;
+    else if (small_auto || (cdg_fused_supported(m, d, dtype) && step_bytes <= (size_t)768 * 1024 && !shard))
+      path = CDGRAB_PATH_FUSED;
     else if (umma_ok && !fma_columns_ok(h)) path = CDGRAB_PATH_UMMA;
     else path = CDGRAB_PATH_FMA;
   } else {
@@ -393,7 +400,7 @@ int cdgrab_step(cdgrab_t *h, const void *grads_dev, void *stream) {
     if (h->rule_randomized || h->mean_out) return CDGRAB_ERR_INVALID;  // greedy rule only in this mode
     e = cdg_launch_indep(h, grads_dev, st);
   } else if (h->path == CDGRAB_PATH_FUSED) {
-    e = cdg_launch_fused(h, grads_dev, 1, st);
+    e = h->m > 16 ? cdg_launch_small(h, grads_dev, 1, st) : cdg_launch_fused(h, grads_dev, 1, st);
   } else if (h->path == CDGRAB_PATH_LITERAL) {
     e = cdg_launch_literal(h, grads_dev, 1, st);
   } else {
@@ -416,7 +423,9 @@ int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream
   const size_t step_bytes = 2 * (size_t)h->m * (size_t)h->d * (h->dtype == CDGRAB_F32 ? 4 : 2);
   if (h->path == CDGRAB_PATH_FUSED && !h->independent && !h->rule_randomized && !h->mean_out) {
     if (step_bytes % 16 != 0) return CDGRAB_ERR_INVALID;
-    if (cdg_launch_fused(h, grads_dev, count, (cudaStream_t)stream) != cudaSuccess) {
+    const cudaError_t e = h->m > 16 ? cdg_launch_small(h, grads_dev, count, (cudaStream_t)stream)
+                                    : cdg_launch_fused(h, grads_dev, count, (cudaStream_t)stream);
+    if (e != cudaSuccess) {
       cudaGetLastError();
       return CDGRAB_ERR_CUDA;
     }
@@ -459,8 +468,8 @@ int cdgrab_step_many(cdgrab_t *h, const void *grads_dev, int count, void *stream
 int cdgrab_step_logreg(cdgrab_t *h, const float *X, const float *y, const float *w, void *stream) {
   if (!valid(h) || !X || !y || !w) return CDGRAB_ERR_INVALID;
   // the one-launch step from feature rows serves handles on either single-launch path
-  const bool single = h->path == CDGRAB_PATH_FUSED ||
-                      (h->path == CDGRAB_PATH_LITERAL && cdg_fused_supported(h->m, h->d, h->dtype));
+  const bool single = (h->path == CDGRAB_PATH_FUSED || h->path == CDGRAB_PATH_LITERAL) &&
+                      cdg_fused_supported(h->m, h->d, h->dtype);
   if (h->dtype != CDGRAB_F32 || !single) return CDGRAB_ERR_INVALID;
   if ((((uintptr_t)X | (uintptr_t)w) & 15) != 0) return CDGRAB_ERR_INVALID;
   if (!on_own_device(h)) return CDGRAB_ERR_DEVICE;

@@ -277,6 +277,9 @@ cudaError_t cdg_launch_fused_logreg(cdgrab_ctx *h, const float *X, const float *
 cudaError_t cdg_launch_logreg(cdgrab_ctx *h, const float *X, const float *y, const float *w,
                               float *out, cudaStream_t st);
 bool cdg_fused_supported(int m, long long d, int dtype);
+// the same single-launch Gram form for 17 <= m <= 128 workers whose step fits shared memory
+bool cdg_small_supported(int m, long long d, int dtype);
+cudaError_t cdg_launch_small(cdgrab_ctx *h, const void *grads, int count, cudaStream_t st);
 // the literal form: one CTA, Algorithm 6 worker by worker, count steps per launch (short rows, any m <= 1024)
 bool cdg_literal_supported(int m, long long d, int dtype);
 cudaError_t cdg_launch_literal(cdgrab_ctx *h, const void *grads, int count, cudaStream_t st);

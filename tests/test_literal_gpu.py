@@ -42,9 +42,11 @@ def test_literal_path_matches_oracle(m, n, d, dtype, monkeypatch):
         pr.close()
 
 
-def test_many_workers_with_short_rows_take_the_literal_path_by_default():
+def test_default_paths_for_short_rows():
     with binding.CdGrab(100, 4, 16, "f32") as h:
-        assert h.path == "literal"
+        assert h.path == "fused"         # many workers, differences fit shared memory: Gram form in one CTA
+    with binding.CdGrab(1024, 4, 64, "f32") as h:
+        assert h.path == "literal"       # more workers than that form holds
     with binding.CdGrab(8, 4, 1024, "f32") as h:
         assert h.path == "literal"
     with binding.CdGrab(8, 4, 2048, "f32") as h:

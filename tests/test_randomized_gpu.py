@@ -22,7 +22,8 @@ def grads(m, d, dtype, seed):
 @pytest.mark.parametrize("m,d,dtype,path", [
     (4, 4096, "f32", "fused"),
     (4, 1024, "f32", "literal"),      # Algorithm 6 worker by worker in one CTA
-    (40, 64, "bf16", "literal"),
+    (40, 128, "bf16", "literal"),
+    (40, 64, "bf16", "fused"),        # many workers, short rows: the Gram form in one CTA
     (8, 16_384, "bf16", "fused"),
     (16, 100_000, "f32", "fma"),      # decisions taken in the tail of the TMA-fed Gram kernel
     (5, 3_001, "f32", "fma"),         # generic tiles + stand-alone scan

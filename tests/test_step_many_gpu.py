@@ -26,7 +26,8 @@ def epoch(m, n, d, dtype, seed):
     (16, 8, 2048, "bf16", "fused"),
     (3, 10, 516, "f32", "literal"),
     (6, 10, 1028, "f32", "fused"),
-    (40, 6, 64, "bf16", "literal"),
+    (40, 6, 128, "bf16", "literal"),
+    (40, 6, 64, "bf16", "fused"),        # many workers, short rows: the Gram form in one CTA
     (8, 6, 200_000, "f32", "fma"),       # two-pass path, TMA-fed pass 1: the call loops over single steps, or
     (16, 8, 1 << 18, "f32", "fma"),      # (CDGRAB_DEFER=1) the update of a step rides in the next step's pass 1
     (16, 8, 300_008, "bf16", "fma"),

@@ -1,4 +1,6 @@
 """Parity of the tensor-core (tcgen05) Gram path against the CPU oracle, bf16 inputs."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -130,6 +132,8 @@ def test_umma_long_rows_with_common_mean(mean, scale, monkeypatch):
 def test_bf16_more_than_64_workers_on_the_tensor_cores(m, n, d):
     """bf16 gradients with 65..128 workers: the differences go through the MMA as two bf16 terms
     each, formed inside the kernel; the bf16 sign tolerance (1e-3) applies."""
+    if os.environ.get("CDGRAB_UMMA_BF16_WIDE") == "0":
+        pytest.skip("the knob under test keeps these shapes off the tensor cores")
     rep = run(m, n, d, seed=m + d % 5)
     print(f"umma bf16 wide m={m} n={n} d={d}:", rep)
     assert rep.raw_agreement > 0.9
