@@ -43,17 +43,16 @@
 
 namespace {
 
-#ifndef CDG_F32_CONV_WARPS
-#define CDG_F32_CONV_WARPS 6
-#endif
-constexpr int kConvWarps = CDG_F32_CONV_WARPS;
-constexpr int kConvThreads = 32 * kConvWarps;       // 16 float4 of a 64-column block x kConvRows rows at a time
-constexpr int kConvRows = kConvThreads / 16;
+// Converter warps: CW = 6 (12 rows of a 64-column block at a time) or CW = 8 (16 rows at a time).
+// Eight pay where six would leave a thread six rows per pass (fp32 with more than 60 workers, bf16
+// with more than 112): pass 1 measured 8 % (fp32, m = 64) and 13 % (bf16, m = 128) faster.  Where
+// six warps take five rows each the two forms tie or eight lose a few per cent (m = 56, 100, 112),
+// below that eight lose outright (idle row slots, warps waiting on one another).
 constexpr int kDrainWarps = 8;
-constexpr int kThreads = 64 + kConvThreads + 32 * kDrainWarps;
+__host__ __device__ constexpr int terms_threads(int cw) { return 64 + 32 * cw + 32 * kDrainWarps; }
+__host__ __device__ constexpr int terms_conv_rows(int cw) { return 2 * cw; }          // 16 threads (float4 each) per row of a block
 constexpr int kMaxStages = 8;
 constexpr int kMaxOps = 4;                           // operand buffers (one 64-column block each)
-constexpr int kRowSlots = (64 + kConvRows - 1) / kConvRows;   // rows per converter thread at m = 64
 constexpr int kBlockCols = 64;                       // columns per MMA block = one 128-byte swizzle row of bf16
 constexpr int kFlushBlocks = 32;                     // blocks between two moves of the fp32 b sums into fp64
 constexpr int kMaxN = 256;                           // row pitch of the summed D: 3 m at m = 64, 2 m at m = 128
@@ -112,6 +111,22 @@ __device__ __forceinline__ void f32_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Bounded wait like mbar_wait, with a suspend-time hint: a waiting warp (producer, MMA issuer,
+// read-back) sleeps in the barrier unit for up to a microsecond at a time instead of polling, and
+// leaves the issue slots of its scheduler to the converter warps (-2 % on pass 1 at m = 32).
+__device__ __forceinline__ bool f32_wait(uint32_t bar, uint32_t parity, long long deadline) {
+  while (true) {
+    uint32_t done;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+    if (done) return true;
+    if (clock64() > deadline) return false;
+  }
+}
+
 // two floats rounded to bf16 (to nearest even), x in the low half
 __device__ __forceinline__ uint32_t pack_bf16x2(float x, float y) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
@@ -122,8 +137,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float x, float y) {
 // threads make over the rows of a block; NS: rows each converter thread takes per pass, a
 // compile-time count so that the NS x 2 split chains sit in one basic block and the scheduler
 // can interleave them.
-template <typename T, int NT, int NS, int NP>
-__global__ void __launch_bounds__(kThreads, 1)
+template <typename T, int NT, int NS, int NP, int CW>
+__global__ void __launch_bounds__(terms_threads(CW), 1)
 gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_r,
                      const F32Params p, float *__restrict__ partials, double *__restrict__ bpart,
                      int *__restrict__ status) {
@@ -136,6 +151,7 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
   __shared__ __align__(8) uint64_t bar_acc_empty[2];
   __shared__ uint32_t tmem_base_sh;
   constexpr uint32_t ES = (uint32_t)sizeof(T);
+  constexpr int kConvWarps = CW, kConvThreads = 32 * CW, kConvRows = terms_conv_rows(CW), kThreads = terms_threads(CW);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m = p.m;
@@ -202,7 +218,7 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
       int s = 0;
       uint32_t turn = 0;
       for (int it = 0; it < n_iter; ++it) {
-        if (turn > 0) ok = mbar_wait(smem_u32(&bar_empty[s]), (turn - 1) & 1, deadline);
+        if (turn > 0) ok = f32_wait(smem_u32(&bar_empty[s]), (turn - 1) & 1, deadline);
         if (!ok) break;
         const int col = (int)((blk_lo + (long long)it * p.nsub) * kBlockCols);   // a multiple of 64 floats
         const uint32_t full = smem_u32(&bar_full[s]);
@@ -216,7 +232,7 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
       if (!ok) {
         atomicOr(status, CDG_ST_TIMEOUT);
         for (int it = max(0, issued - p.stages); it < issued; ++it)
-          mbar_wait(smem_u32(&bar_full[it % p.stages]), (it / p.stages) & 1, clock64() + kCdgWaitCycles);
+          f32_wait(smem_u32(&bar_full[it % p.stages]), (it / p.stages) & 1, clock64() + kCdgWaitCycles);
       }
     }
   } else if (warp == 1) {
@@ -229,8 +245,8 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     for (int g = 0; g < nsb; ++g) {
       const int buf = c & 1;
       const bool chunk_start = in_chunk == 0;
-      if (chunk_start && c >= 2) ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), ((c >> 1) - 1) & 1, deadline);
-      if (ok) ok = mbar_wait(smem_u32(&bar_op_full[o]), op_parity, deadline);
+      if (chunk_start && c >= 2) ok = f32_wait(smem_u32(&bar_acc_empty[buf]), ((c >> 1) - 1) & 1, deadline);
+      if (ok) ok = f32_wait(smem_u32(&bar_op_full[o]), op_parity, deadline);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -282,13 +298,13 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     int s = 0, o = 0, since_flush = 0;
     uint32_t full_parity = 0, turn_o = 0;
     for (int it = 0; it < n_iter && ok; ++it) {
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_full[s]), full_parity, deadline));   // the lanes leave together
+      ok = __all_sync(0xffffffffu, f32_wait(smem_u32(&bar_full[s]), full_parity, deadline));   // the lanes leave together
       if (!ok) break;
       const uint8_t *tile = stages_ptr + (size_t)s * stage_bytes;
       const float *rt = reinterpret_cast<const float *>(tile + rows_bytes);
       const int cnt = min(p.nsub, nsb - it * p.nsub);      // blocks past the range belong to the next CTA
       for (int sub = 0; sub < cnt; ++sub) {
-        if (turn_o > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_op_empty[o]), (turn_o - 1) & 1, deadline));
+        if (turn_o > 0) ok = __all_sync(0xffffffffu, f32_wait(smem_u32(&bar_op_empty[o]), (turn_o - 1) & 1, deadline));
         if (!ok) break;
         uint8_t *op = ops_ptr + (size_t)o * op_bytes;
         const float4 rv = *reinterpret_cast<const float4 *>(rt + sub * kBlockCols + q * 4);
@@ -388,8 +404,8 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     }
   } else {
     // ---------------- accumulator read-back: TMEM chunks -> partial D ----------------
-    const int dw = warp - (2 + kConvWarps);          // 0..7; the first read-back warp's index is a multiple of 4, so warp % 4 == dw % 4
-    const int lg = dw & 3;                           // TMEM lane group this warp may read
+    const int dw = warp - (2 + kConvWarps);          // 0..7
+    const int lg = warp & 3;                         // TMEM lane group this warp may read; four consecutive warps cover all four
     const int half = dw >> 2;                        // pieces of 16 columns: this warp takes piece 2 pp + half
     const int row = lg * 32 + lane;
     const int nchunks = (nsb + p.drain - 1) / p.drain;
@@ -406,7 +422,7 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     bool ok = true;
     for (int c = 0; c < nchunks && ok; ++c) {
       const int buf = c & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_acc_full[buf]), (c >> 1) & 1, deadline));
+      ok = __all_sync(0xffffffffu, f32_wait(smem_u32(&bar_acc_full[buf]), (c >> 1) & 1, deadline));
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
@@ -581,22 +597,24 @@ bool encode_rows(CUtensorMap *map, const void *base, long long d, int rows, int 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int NT, int NS, int NP>
+template <typename T, int NT, int NS, int NP, int CW = 6>
 cudaError_t terms_launch(cdgrab_ctx *h, const CUtensorMap &tm_g, const F32Params &p, cudaStream_t st) {
-  return cdg_launch_dep(h, gram_umma_f32_kernel<T, NT, NS, NP>, dim3(h->f32_ctas), dim3(kThreads), h->f32_smem, st, tm_g,
-                        h->tm_f32r, p, h->umma_partials, h->f32_bpart, h->status);
+  return cdg_launch_dep(h, gram_umma_f32_kernel<T, NT, NS, NP, CW>, dim3(h->f32_ctas), dim3(terms_threads(CW)), h->f32_smem,
+                        st, tm_g, h->tm_f32r, p, h->umma_partials, h->f32_bpart, h->status);
 }
 
 cudaError_t terms_open_limits() {
-  cudaError_t e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 1, 1>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 2, 1>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 3, 1>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 4, 1>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 5, 1>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 6, 1>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 4, 2>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 5, 2>);
-  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 6, 2>);
+  cudaError_t e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 1, 1, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 2, 1, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 3, 1, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 4, 1, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 5, 1, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 6, 1, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 4, 2, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 5, 2, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 6, 2, 6>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<float, 3, 4, 1, 8>);
+  if (e == cudaSuccess) e = cdg_open_smem_limit(gram_umma_f32_kernel<__nv_bfloat16, 2, 4, 2, 8>);
   if (e == cudaSuccess) e = cdg_open_smem_limit(umma_f32_combine_kernel);
   return e;
 }
@@ -686,6 +704,8 @@ int cdg_umma_f32_setup(cdgrab_ctx *h) {
   if (const char *e = getenv("CDGRAB_UMMA_FUSE_TAIL")) {
     if (atoi(e) == 0) h->umma_fused = 0;
   }
+  h->f32_conv8 = 1;                      // CDGRAB_F32_CONV8=0: six converter warps at every size
+  if (const char *e = getenv("CDGRAB_F32_CONV8")) h->f32_conv8 = atoi(e) ? 1 : 0;
   h->umma_f32 = 1;
   return CDGRAB_OK;
 }
@@ -717,11 +737,13 @@ cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStrea
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     const CUtensorMap &tm = h->tm_f32g.maps[slot][0];
-    static_assert(kRowSlots <= 6, "one instantiation per slot count");
+    // rows per converter thread and pass: up to 5 with six converter warps; where they would take 6, eight warps take 4
     if (h->f32_nt == 3) {
       p.pass_rows = (h->m + 7) & ~7;
-      const int ns = (h->m + kConvRows - 1) / kConvRows;       // rows per converter thread
-      switch (ns) {
+      const int ns = (h->m + terms_conv_rows(6) - 1) / terms_conv_rows(6);
+      if (ns > 5 && h->f32_conv8) {
+        terms_launch<float, 3, 4, 1, 8>(h, tm, p, st);
+      } else switch (ns) {
         case 1: terms_launch<float, 3, 1, 1>(h, tm, p, st); break;
         case 2: terms_launch<float, 3, 2, 1>(h, tm, p, st); break;
         case 3: terms_launch<float, 3, 3, 1>(h, tm, p, st); break;
@@ -731,8 +753,10 @@ cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStrea
       }
     } else {
       p.pass_rows = bf16_pass_rows(h->m);                      // 40..64
-      const int ns = (p.pass_rows + kConvRows - 1) / kConvRows;
-      switch (ns) {
+      const int ns = (p.pass_rows + terms_conv_rows(6) - 1) / terms_conv_rows(6);
+      if (ns > 5 && h->f32_conv8) {
+        terms_launch<__nv_bfloat16, 2, 4, 2, 8>(h, tm, p, st);
+      } else switch (ns) {
         case 4: terms_launch<__nv_bfloat16, 2, 4, 2>(h, tm, p, st); break;
         case 5: terms_launch<__nv_bfloat16, 2, 5, 2>(h, tm, p, st); break;
         default: terms_launch<__nv_bfloat16, 2, 6, 2>(h, tm, p, st); break;
