@@ -150,6 +150,7 @@ struct cdgrab_ctx {
   int f32_nops;            // operand buffers
   int f32_stages;
   int f32_drain;           // 64-column blocks per TMEM accumulation chunk
+  int f32_mma_m;           // MMA M of the term-splitting kernel: 64 for fp32 with m <= 32, else 128
   int f32_conv8;           // 1: eight converter warps where six would take 6 rows per thread and pass
   int f32_ctas;
   size_t f32_smem;

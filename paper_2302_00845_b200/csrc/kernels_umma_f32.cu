@@ -7,19 +7,20 @@
 // bf16 terms are exact in the fp32 accumulator, so <c_k, c_i> is the sum of the nine term
 // products; the lo x lo one (below 2^-32 of the product) is left out, the other eight come out
 // of ONE product per 16 columns:  D = A B^T with B = [hi_0..hi_{m-1} | mid_0.. | lo_0..] (3m
-// rows, the MMA's N) and A = the first 128 of those rows (hi and mid, the MMA's M):
+// rows, the MMA's N) and A = the first 128 of those rows (hi and mid, the MMA's M; M = 64 when
+// 2m <= 64, which halves the A bytes each MMA reads from shared memory):
 //     G_ki = D[k][i] + D[k][m+i] + D[k][2m+i] + D[m+k][i] + D[m+k][m+i] + D[m+k][2m+i]
 //            + D[i][2m+k] + D[m+i][2m+k]          (the last two are lo_k x hi_i and lo_k x mid_i).
 // The terms are formed inside the kernel: TMA brings fp32 tiles [2m rows][64 s columns] and the
-// matching piece of r into a ring of stages; six converter warps read them, subtract, split,
+// matching piece of r into a ring of stages; six (or eight) converter warps read them, subtract, split,
 // and store the bf16 terms into an operand buffer in the K-major 128-byte-swizzled layout the
 // MMA reads ([8-row group][8 rows][128 B], 16-byte chunk c of row q at chunk c ^ (q & 7)).  The
 // same warps add up b_i = <r, c_i> on the FMA pipe (fp32 products, moved into fp64 every 32
 // blocks), so r needs no bf16 copy on this path.  Nothing but the caller's rows and r is read
 // from HBM: 2mde + 4d bytes per launch.
 //
-// Roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2..7
-// converters, warps 8..15 read the accumulator back.  The sum stays in TMEM for `drain` blocks
+// Roles (512 or 576 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2..7
+// (2..9) converters, the last eight warps read the accumulator back.  The sum stays in TMEM for `drain` blocks
 // of 64 columns only (the tensor core's fp32 accumulation truncates), then the read-back warps
 // add the chunk to fp32 registers (round to nearest) while the MMAs fill the other buffer.
 // One persistent CTA per SM owns a contiguous range of 64-column blocks; its partial D and b
@@ -67,6 +68,7 @@ struct F32Params {
   int drain;           // blocks accumulated in TMEM before the sum is read back
   long long nblk;      // ceil(d / 64)
   int pass_rows;       // rows per converter pass (a multiple of 8; = m rounded up when there is one pass)
+  int mma_m;           // MMA M: 128, or 64 when the 2m rows of A fit (half the A bytes read from shared memory per MMA)
 };
 
 template <typename T>
@@ -237,8 +239,8 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer: the warp loops converged, an elected lane issues ----------------
-    // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = npad
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)p.npad >> 3) << 17) | ((128u >> 4) << 24);
+    // kind::f16, D = f32, A = B = bf16, both K-major, M = 128 (64 when A has at most 64 rows), N = npad
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)p.npad >> 3) << 17) | (((uint32_t)p.mma_m >> 4) << 24);
     bool ok = true;
     int o = 0, c = 0, in_chunk = 0;
     uint32_t op_parity = 0;
@@ -407,10 +409,13 @@ gram_umma_f32_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_cons
     const int dw = warp - (2 + kConvWarps);          // 0..7
     const int lg = warp & 3;                         // TMEM lane group this warp may read; four consecutive warps cover all four
     const int half = dw >> 2;                        // pieces of 16 columns: this warp takes piece 2 pp + half
-    const int row = lg * 32 + lane;
+    // M = 128: row r of D lies in TMEM lane r.  M = 64: in lane 32 (r / 16) + r % 16, the first 16
+    // lanes of each lane group (the other lanes hold nothing of this product: row 128 = none).
+    int row = lg * 32 + lane;
+    if (p.mma_m == 64) row = (lane < 16) ? lg * 16 + lane : 128;
     const int nchunks = (nsb + p.drain - 1) / p.drain;
     const int rows_needed = (NT == 3) ? 2 * m : m;   // rows of D the combine reads
-    float *dst = partials + ((size_t)blockIdx.x * 128 + row) * (size_t)p.npad;
+    float *dst = partials + ((size_t)blockIdx.x * 128 + (row & 127)) * (size_t)p.npad;
     // NT == 3 (N <= 192): the chunks are added in fp32 registers and stored once.  NT == 2
     // (N <= 256): each chunk is added to the partial in global memory (first chunk: stored).
     constexpr int kPieces = (NT == 3) ? 6 : 8;       // pieces of 16 columns per warp
@@ -704,6 +709,13 @@ int cdg_umma_f32_setup(cdgrab_ctx *h) {
   if (const char *e = getenv("CDGRAB_UMMA_FUSE_TAIL")) {
     if (atoi(e) == 0) h->umma_fused = 0;
   }
+  // fp32 with at most 32 workers: hi and mid terms are 2m <= 64 rows, so M = 64 reads half the A
+  // bytes per MMA (pass 1 is bound by shared-memory bandwidth there: 4 % faster at m = 32);
+  // CDGRAB_F32_M64=0 keeps M = 128
+  h->f32_mma_m = (nt == 3 && 2 * m <= 64) ? 64 : 128;
+  if (const char *e = getenv("CDGRAB_F32_M64")) {
+    if (atoi(e) == 0) h->f32_mma_m = 128;
+  }
   h->f32_conv8 = 1;                      // CDGRAB_F32_CONV8=0: six converter warps at every size
   if (const char *e = getenv("CDGRAB_F32_CONV8")) h->f32_conv8 = atoi(e) ? 1 : 0;
   h->umma_f32 = 1;
@@ -734,6 +746,7 @@ cudaError_t cdg_launch_gram_umma_f32(cdgrab_ctx *h, const void *grads, cudaStrea
   p.nops = h->f32_nops;
   p.drain = h->f32_drain;
   p.nblk = (h->d + kBlockCols - 1) / kBlockCols;
+  p.mma_m = h->f32_mma_m;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     const CUtensorMap &tm = h->tm_f32g.maps[slot][0];
