@@ -17,6 +17,12 @@
  *     Calls that take a stream only enqueue work; they do not synchronise the host.
  *   - All device work of one handle must be issued on one stream (or on streams the
  *     caller orders itself).  One handle is used by one host thread at a time.
+ *   - The library's kernels are chained with programmatic dependent launch and the last
+ *     kernel of a step lets its dependents be scheduled early.  Ordinary launches, copies
+ *     and events after a library call are ordered as usual; a caller's kernel that is itself
+ *     launched with programmatic stream serialization directly after a library call must
+ *     execute griddepcontrol.wait (cudaGridDependencySynchronize) before it touches anything
+ *     the call reads or writes.
  *   - Return value: CDGRAB_OK (0) or a negative CDGRAB_ERR_* code.  Argument and state
  *     errors leave the handle unchanged.  Conditions found on the device (non-finite
  *     reductions, an expired bounded wait) are written to a device status word and

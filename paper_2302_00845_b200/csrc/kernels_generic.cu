@@ -238,6 +238,10 @@ update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__re
               int sign_stride, int m, long long d, __nv_bfloat16 *__restrict__ r_split,
               long long d_pad, float *__restrict__ mean_out) {
   extern __shared__ float ssh[];  // [m] signs as +-1.0f
+  // The next launch in the stream (pass 1 of the next step) may be scheduled as this grid's blocks
+  // leave; it waits for this grid's completion before it reads r.  (The pass-1 kernels do not
+  // trigger early: pass 2's blocks would pile up on the SMs that finished first.)
+  cdg_grid_dep_trigger();
   cdg_grid_dep_wait();            // the signs come from the launch before this one
   for (int i = threadIdx.x; i < m; i += blockDim.x) ssh[i] = (float)signs[(size_t)i * sign_stride];
   __syncthreads();
