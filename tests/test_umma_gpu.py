@@ -37,6 +37,10 @@ def run(m, n, d, seed, mean=0.0, scale=1.0):
     (43, 4, 70_004),         # 129 term rows: past one 128-row tile; d a multiple of 4 only
     (50, 4, 100_000),
     (64, 4, 8192),           # the largest m: 192 term rows; fewer blocks than SMs
+    (61, 4, 150_000),        # eight converter warps (six would take six rows per thread), 3 idle row slots
+    (60, 4, 150_000),        # the last m on six converter warps
+    (32, 4, 150_000),        # the last m with MMA M = 64 (2m = 64 rows of A)
+    (33, 4, 150_000),        # the first m with M = 128
     (64, 6, 1_000_000 + 4),  # many accumulator chunks per CTA, ragged last block
     (64, 4, 64 * 148 * 2 + 12),  # two blocks per CTA, odd tail
     (33, 4, 300_000),
@@ -128,6 +132,8 @@ def test_umma_long_rows_with_common_mean(mean, scale, monkeypatch):
     (100, 4, 300_000),
     (128, 4, 64 * 148 * 2 + 8),   # the largest m: N = 256, both TMEM buffers full width
     (128, 6, 1_000_000),      # several accumulator chunks per CTA
+    (113, 4, 120_000),        # eight converter warps, passes of 64 rows of which 57 / 56 are real
+    (112, 4, 120_000),        # the last m on six converter warps (passes of 56 rows)
 ])
 def test_bf16_more_than_64_workers_on_the_tensor_cores(m, n, d):
     """bf16 gradients with 65..128 workers: the differences go through the MMA as two bf16 terms
