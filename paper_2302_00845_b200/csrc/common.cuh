@@ -134,6 +134,9 @@ struct cdgrab_ctx {
   size_t umma_smem;
   CUtensorMap tm_r;        // 3-D tensor map over r_split
   CUtensorMap tm_r2;       // 2-D map over r_split (ragged last block)
+  CUtensorMap tm_r32;      // 2-D map over r itself (fp32), when pass 1 forms the bf16 rows in shared memory
+  int umma_rconv;          // 1: pass 1 reads r as fp32 and splits it in the kernel (no r_split in HBM)
+  int umma_rbox;           // 64-column blocks of r per fp32 copy
   // maps over the gradient rows of the last few buffers: [0] 3-D, [1] 2-D (ragged last block),
   // [2] 4-D over the full 8-row groups
   CdgMapCache<3> tm_g;

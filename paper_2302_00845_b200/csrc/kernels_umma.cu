@@ -5,10 +5,14 @@
 // accumulator, so no difference has to be rounded to bf16.  The Gram matrix of the pair
 // differences c_i = z1_i - z2_i follows afterwards in fp64:
 //     G_ki = H[k][i] - H[k][m+i] - H[m+k][i] + H[m+k][m+i].
-// The running sum r (fp32) is kept as three bf16 rows hi + mid + lo = r exactly (3 x 8
-// significand bits), written by pass 2; they are appended to operand B, so
+// The running sum r (fp32) goes in as three bf16 rows hi + mid + lo = r exactly (3 x 8
+// significand bits) appended to operand B, so
 //     b_i = <r, c_i> = sum_j (H[i][R+j] - H[m+i][R+j])
-// falls out of the same MMA.
+// falls out of the same MMA.  The rows are formed inside the kernel: the TMA brings the fp32
+// piece of r of a stage (4 bytes per column), a converter warp splits it and writes the three
+// rows into the stage's r row group in the swizzled layout the TMA would have produced.
+// (CDGRAB_UMMA_RCONV=0: pass 2 keeps a bf16 copy [3][d] of r in HBM and the TMA brings its rows;
+// 12 instead of 4 bytes of r traffic per column and step on top of pass 2's own 8.)
 //
 // One persistent CTA per SM owns a contiguous K range (split-K) in blocks of 64 columns.
 // A pipeline stage holds `subs` consecutive blocks.  Rows are loaded in groups of 8: a TMA box
@@ -25,7 +29,7 @@
 // With 2m <= 64 one MMA takes two blocks at once (N = 160; layout at the top of the kernel).
 // Roles: warp 0 TMA producer, warp 1 MMA issuer (the warp loops converged, an elected lane
 // issues) and TMEM owner, warps 2..5 drain the accumulator (tcgen05.ld) chunk by chunk into
-// fp32 registers and write the CTA's partial H.  The combine kernel's last block also takes the
+// fp32 registers and write the CTA's partial H, warp 6 converts r.  The combine kernel's last block also takes the
 // step's decisions.
 // Every wait is bounded: on expiry the CTA raises the time-out bit of the status word,
 // drains the copies it has in flight, frees its TMEM and returns.
@@ -39,7 +43,7 @@
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;           // TMA producer, MMA issuer, four read-back warps, one converter of r
 constexpr int kMaxStages = 8;
 constexpr int kSubCols = 64;             // bf16 columns per TMA box = one 128-byte swizzle row
 constexpr int kRBoxRows = 16;
@@ -57,6 +61,8 @@ struct UmmaParams {
   int drain;           // pipeline iterations accumulated in TMEM before the sum is drained
   int g4;              // full 8-row groups fetched by one 4-D copy (0: per-group copies only)
   int paired;          // 2m <= 64: blocks j and j + subs/2 of a stage share one MMA (see the kernel)
+  int rconv;           // 1: r arrives as fp32 and warp 6 writes its three bf16 rows; 0: the rows come from HBM
+  int rbox;            // 64-column blocks of r per fp32 copy (a divisor of the blocks per (half) stage, at most 4)
 };
 
 // K-major, 128-byte swizzle: rows 128 B apart, 8-row groups `sbo` bytes apart
@@ -89,10 +95,13 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __global__ void __launch_bounds__(kThreads, 1)
 gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constant__ CUtensorMap tm_r3,
                  const __grid_constant__ CUtensorMap tm_g2, const __grid_constant__ CUtensorMap tm_r2,
-                 const __grid_constant__ CUtensorMap tm_g4, const UmmaParams p, float *__restrict__ partials, int *__restrict__ status) {
+                 const __grid_constant__ CUtensorMap tm_g4, const __grid_constant__ CUtensorMap tm_r32,
+                 const UmmaParams p, float *__restrict__ partials, int *__restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
+  __shared__ __align__(8) uint64_t bar_r32[kMaxStages];   // the fp32 piece of r of stage s has landed (rconv)
+  __shared__ __align__(8) uint64_t bar_conv[kMaxStages];  // ... and its bf16 rows are written
   __shared__ __align__(8) uint64_t bar_acc_full[2];    // accumulator buffer b holds a finished chunk
   __shared__ __align__(8) uint64_t bar_acc_empty[2];   // ... has been read back and may be overwritten
   __shared__ uint32_t tmem_base_sh;
@@ -112,6 +121,10 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   const int ngroups = paired ? 20 : (p.ncols >> 3);
   const int ggroups = p.box_rows >> 3;                           // gradient row groups
   const uint32_t stage_bytes = group_bytes * ngroups;
+  // rconv: the fp32 pieces of r (256 bytes per block, subs blocks per stage) lie behind the
+  // stages and the slack operand A may read past the last stage
+  const int rconv = p.rconv;
+  const uint32_t r32_off = (uint32_t)p.stages * stage_bytes + (ngroups < 16 ? (uint32_t)(16 - ngroups) * group_bytes : 0u);
 
   // this CTA's K range in full blocks; the last CTA also owns the ragged block, taken first.
   // Paired: whole stages per CTA, so that both halves of a stage belong to the same CTA (blocks
@@ -132,6 +145,8 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
+      mbar_init(smem_u32(&bar_r32[s]), 1);
+      mbar_init(smem_u32(&bar_conv[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bar_acc_full[b]), 1);
@@ -139,12 +154,14 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
     }
     mbar_init_fence();
   }
-  // row groups that are never loaded (gradient groups wholly past row 2m, and the padding
-  // group after the r rows) are zeroed once
+  // row groups that are never loaded (gradient groups wholly past row 2m, the padding group
+  // after the r rows, and with rconv the r groups themselves, of which the converter rewrites
+  // rows 0..2 only) are zeroed once
   const int lgroups = (p.rows_used + 7) >> 3;                    // gradient row groups that get loaded
   for (int s = 0; s < p.stages; ++s) {
     for (int g = 0; g < ngroups; ++g) {
-      const bool loaded = paired ? (g < 16 ? (g & 7) < lgroups : !(g & 1)) : (g < lgroups || g == ggroups);
+      const bool loaded = paired ? (g < 16 ? (g & 7) < lgroups : (!(g & 1) && !rconv))
+                                 : (g < lgroups || (g == ggroups && !rconv));
       if (loaded) continue;
       uint8_t *z = smem_raw + (tiles - smem_u32(smem_raw)) + (size_t)s * stage_bytes + (size_t)g * group_bytes;
       for (uint32_t o = threadIdx.x * 16; o < group_bytes; o += kThreads * 16)
@@ -176,44 +193,67 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
         const uint32_t full = smem_u32(&bar_full[s]);
         const uint32_t base = tiles + s * stage_bytes;
         const uint32_t rbase = base + (paired ? 16 : ggroups) * group_bytes;   // the r rows (first half)
+        // rconv: fp32 r of the nb blocks of a (half) stage, rbox blocks per copy, instead of the r rows
+        const int nb = paired ? hb : p.subs;
+        const uint32_t r32 = tiles + r32_off + (uint32_t)(s * p.subs) * 256u;
+        const uint32_t rg_tx = rconv ? 0u : 1u;                               // r row groups a copy fills
+        const uint32_t rbar = smem_u32(&bar_r32[s]);
+        // the small copies of r go first and complete a barrier of their own, so that the
+        // converter works while the rows of the stage are still landing
+        if (rconv) mbar_expect_tx(rbar, (uint32_t)(paired ? 2 * nb : nb) * 256u);
         if (has_tail && it == 0) {
           // ragged block: 8-row 2-D boxes into block slot 0 of every loaded row group
           const int col = (int)(p.nblk_full * kSubCols);   // 128-byte aligned
-          mbar_expect_tx(full, (uint32_t)(lgroups + 1) * (1024u + (paired ? group_bytes : 0u)));
+          if (rconv) {
+            for (int q = 0; q < nb; q += p.rbox) tma_load_2d(r32 + q * 256u, &tm_r32, col + q * kSubCols, 0, rbar);
+            if (paired)      // the other half: columns past the end, read as zeros
+              for (int q = 0; q < nb; q += p.rbox)
+                tma_load_2d(r32 + (uint32_t)(nb + q) * 256u, &tm_r32, (int)((p.nblk_full + 1 + q) * kSubCols), 0, rbar);
+          }
+          mbar_expect_tx(full, (uint32_t)(lgroups + rg_tx) * (1024u + (paired ? group_bytes : 0u)));
           for (int g = 0; g < lgroups; ++g) tma_load_2d(base + g * group_bytes, &tm_g2, col, g * 8, full);
-          tma_load_2d(rbase, &tm_r2, col, 0, full);
+          if (!rconv) tma_load_2d(rbase, &tm_r2, col, 0, full);
           if (paired) {
             // the other half of the pair: blocks past the end, which the copies fill with zeros
             const int past = (int)p.nblk_full;
             const uint32_t hbase = base + 8 * group_bytes;
             if (p.g4 > 0) tma_load_4d(hbase, &tm_g4, 0, 0, past, 0, full);
             for (int g = p.g4; g < lgroups; ++g) tma_load_3d(hbase + g * group_bytes, &tm_g3, 0, g * 8, past, full);
-            tma_load_3d(rbase + 2 * group_bytes, &tm_r3, 0, 0, past, full);
+            if (!rconv) tma_load_3d(rbase + 2 * group_bytes, &tm_r3, 0, 0, past, full);
           }
         } else if (paired) {
           const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
-          mbar_expect_tx(full, 2u * (uint32_t)(lgroups + 1) * group_bytes);
+          if (rconv)
+            for (int hf = 0; hf < 2; ++hf)
+              for (int q = 0; q < nb; q += p.rbox)
+                tma_load_2d(r32 + (uint32_t)(hf * nb + q) * 256u, &tm_r32, (int)(first + (long long)hf * hb + q) * kSubCols, 0, rbar);
+          mbar_expect_tx(full, 2u * (uint32_t)(lgroups + rg_tx) * group_bytes);
           for (int hf = 0; hf < 2; ++hf) {
             const int blk = (int)(first + (long long)hf * hb);
             const uint32_t hbase = base + hf * 8 * group_bytes;
             if (p.g4 > 0) tma_load_4d(hbase, &tm_g4, 0, 0, blk, 0, full);
             for (int g = p.g4; g < lgroups; ++g) tma_load_3d(hbase + g * group_bytes, &tm_g3, 0, g * 8, blk, full);
-            tma_load_3d(rbase + hf * 2 * group_bytes, &tm_r3, 0, 0, blk, full);
+            if (!rconv) tma_load_3d(rbase + hf * 2 * group_bytes, &tm_r3, 0, 0, blk, full);
           }
         } else {
           const long long first = blk_lo + (long long)(it - has_tail) * p.subs;
-          mbar_expect_tx(full, (uint32_t)(lgroups + 1) * group_bytes);
+          if (rconv)
+            for (int q = 0; q < nb; q += p.rbox)
+              tma_load_2d(r32 + q * 256u, &tm_r32, (int)(first + q) * kSubCols, 0, rbar);
+          mbar_expect_tx(full, (uint32_t)(lgroups + rg_tx) * group_bytes);
           if (p.g4 > 0) tma_load_4d(base, &tm_g4, 0, 0, (int)first, 0, full);
           for (int g = p.g4; g < lgroups; ++g) tma_load_3d(base + g * group_bytes, &tm_g3, 0, g * 8, (int)first, full);
-          tma_load_3d(rbase, &tm_r3, 0, 0, (int)first, full);
+          if (!rconv) tma_load_3d(rbase, &tm_r3, 0, 0, (int)first, full);
         }
         issued = it + 1;
       }
       if (!ok) {
         atomicOr(status, CDG_ST_TIMEOUT);
         // let the copies already issued land before the CTA gives up its shared memory
-        for (int it = max(0, issued - p.stages); it < issued; ++it)
+        for (int it = max(0, issued - p.stages); it < issued; ++it) {
           mbar_wait(smem_u32(&bar_full[it % p.stages]), (it / p.stages) & 1, clock64() + kWaitCycles);
+          if (rconv) mbar_wait(smem_u32(&bar_r32[it % p.stages]), (it / p.stages) & 1, clock64() + kWaitCycles);
+        }
       }
     }
   } else if (warp == 1) {
@@ -237,6 +277,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       const bool chunk_start = in_chunk == 0;
       if (chunk_start && c >= 2) ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), ((c >> 1) - 1) & 1, deadline);
       if (ok) ok = mbar_wait(smem_u32(&bar_full[s]), full_parity, deadline);
+      if (ok && rconv) ok = mbar_wait(smem_u32(&bar_conv[s]), full_parity, deadline);   // the r rows are in place
       ok = __all_sync(0xffffffffu, ok);      // the lanes leave together
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -265,6 +306,57 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       if (++s == p.stages) { s = 0; full_parity ^= 1u; }
     }
     if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+  } else if (warp == 6) {
+    // ---------------- converter of r: fp32 piece -> three bf16 rows hi + mid + lo = r ----------------
+    // Written where the TMA would have put them: row t of the 8-row r group of block q, 16-byte
+    // chunk (c / 8) ^ t of its 128-byte row (the 128-byte swizzle; rows 3..7 stay zero).  Same
+    // three roundings as everywhere else r is split, so the products come out bit for bit alike.
+    if (rconv) {
+      const int nb = paired ? hb : p.subs;
+      uint8_t *smem_tiles = smem_raw + (tiles - smem_u32(smem_raw));
+      bool ok = true;
+      int s = 0;
+      uint32_t parity = 0;
+      for (int it = 0; it < n_iter; ++it) {
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_r32[s]), parity, deadline));
+        if (!ok) break;
+        for (int hf = 0; hf < (paired ? 2 : 1); ++hf) {
+          const float *src = reinterpret_cast<const float *>(smem_tiles + r32_off + (size_t)(s * p.subs + hf * nb) * 256);
+          uint8_t *rg = smem_tiles + (size_t)s * stage_bytes + (size_t)((paired ? 16 : ggroups) + hf * 2) * group_bytes;
+          for (int idx = lane * 8; idx < nb * kSubCols; idx += 256) {
+            const int q = idx >> 6, chunk = (idx & 63) >> 3;
+            const float4 f0 = *reinterpret_cast<const float4 *>(src + idx);
+            const float4 f1 = *reinterpret_cast<const float4 *>(src + idx + 4);
+            const float v[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+            uint32_t hi[4], mid[4], lo[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              __nv_bfloat16 h2[2], m2[2], l2[2];
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const float x = v[2 * j + e];
+                h2[e] = __float2bfloat16_rn(x);
+                const float r1 = x - __bfloat162float(h2[e]);
+                m2[e] = __float2bfloat16_rn(r1);
+                l2[e] = __float2bfloat16_rn(r1 - __bfloat162float(m2[e]));
+              }
+              hi[j] = (uint32_t)__bfloat16_as_ushort(h2[0]) | ((uint32_t)__bfloat16_as_ushort(h2[1]) << 16);
+              mid[j] = (uint32_t)__bfloat16_as_ushort(m2[0]) | ((uint32_t)__bfloat16_as_ushort(m2[1]) << 16);
+              lo[j] = (uint32_t)__bfloat16_as_ushort(l2[0]) | ((uint32_t)__bfloat16_as_ushort(l2[1]) << 16);
+            }
+            uint8_t *blk = rg + (size_t)q * 1024;
+            *reinterpret_cast<uint4 *>(blk + 0 * 128 + ((chunk ^ 0) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4 *>(blk + 1 * 128 + ((chunk ^ 1) << 4)) = make_uint4(mid[0], mid[1], mid[2], mid[3]);
+            *reinterpret_cast<uint4 *>(blk + 2 * 128 + ((chunk ^ 2) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads these bytes through the async proxy
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bar_conv[s]));
+        if (++s == p.stages) { s = 0; parity ^= 1u; }
+      }
+      if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
+    }
   } else {
     // ---------------- accumulator read-back: TMEM chunks -> fp32 registers -> partial H ----------------
     const int lg = warp & 3;                 // TMEM lane group this warp may read
@@ -453,6 +545,20 @@ bool encode_map_4d(CUtensorMap *map, const void *base, long long nblk, int group
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D fp32 map over r viewed as one row of d columns, box {blocks x 64 columns, 1 row}, no swizzle;
+// columns past d read as zeros
+bool encode_map_r32(CUtensorMap *map, const void *base, long long d, int blocks) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)d, 1};
+  cuuint64_t strides[1] = {(cuuint64_t)d * 4};
+  cuuint32_t box[2] = {(cuuint32_t)(blocks * kSubCols), 1};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 // Self-test of the bounded wait every TMA-fed kernel here relies on: one thread waits on a
@@ -524,12 +630,24 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   const int ngroups = h->umma_paired ? 20 : h->umma_ncols / 8;
   const size_t stage_bytes = group_bytes * ngroups;
   const size_t slack = (ngroups < 16) ? (16 - ngroups) * group_bytes : 0;  // operand A spans 16 row groups
+  // r reaches the MMA as three bf16 rows.  Default: pass 1 reads r itself (fp32, 4 bytes per
+  // column) and one warp writes the rows in shared memory; CDGRAB_UMMA_RCONV=0: pass 2 keeps a
+  // bf16 copy [3][d_pad] in HBM (6 bytes per column written, 6 read) and the TMA brings its rows.
+  h->umma_rconv = 1;
+  if (const char *e = getenv("CDGRAB_UMMA_RCONV")) h->umma_rconv = atoi(e) ? 1 : 0;
+  {
+    const int nb = h->umma_paired ? subs / 2 : subs;       // blocks per (half) stage
+    int rbox = nb < 4 ? nb : 4;                            // at most 256 fp32 columns per copy
+    while (nb % rbox) --rbox;
+    h->umma_rbox = rbox;
+  }
+  const size_t r32_stage = h->umma_rconv ? (size_t)subs * 256 : 0;         // fp32 r of a stage
   const size_t budget = 226 * 1024 - 1024 - slack;
-  int stages = (int)(budget / stage_bytes);
+  int stages = (int)(budget / (stage_bytes + r32_stage));
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return CDGRAB_ERR_INVALID;
   h->umma_stages = stages;
-  h->umma_smem = stages * stage_bytes + slack + 1024;
+  h->umma_smem = stages * (stage_bytes + r32_stage) + slack + 1024;
   const long long nblk_full = h->d / kSubCols;
   const long long total_sub = (h->d + kSubCols - 1) / kSubCols;
   h->umma_ctas = (int)((nblk_full < h->num_sms) ? (nblk_full > 0 ? nblk_full : 1) : h->num_sms);
@@ -538,17 +656,24 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     h->umma_ctas = (int)(units < h->num_sms ? (units > 0 ? units : 1) : h->num_sms);
   }
   h->d_pad = total_sub * kSubCols;
-  if (cdg_alloc(h, &h->r_split, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
-      cdg_alloc(h, &h->umma_partials, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess) {
+  if (cdg_alloc(h, &h->umma_partials, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess ||
+      (!h->umma_rconv && cdg_alloc(h, &h->r_split, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess)) {
     cudaGetLastError();
     return CDGRAB_ERR_NOMEM;
   }
-  if (cudaMemset(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess ||
-      cudaMemset(h->umma_partials, 0, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess)
+  if (cudaMemset(h->umma_partials, 0, sizeof(float) * 128 * (size_t)h->umma_ncols * h->umma_ctas) != cudaSuccess)
     return CDGRAB_ERR_CUDA;
-  if (!encode_map_3d(&h->tm_r, h->r_split, nblk_full, 3, h->d_pad, h->umma_paired ? subs / 2 : subs))
-    return CDGRAB_ERR_CUDA;
-  if (!encode_map_2d(&h->tm_r2, h->r_split, h->d, 3, h->d_pad)) return CDGRAB_ERR_CUDA;
+  if (h->umma_rconv) {
+    if (!encode_map_r32(&h->tm_r32, h->r, h->d, h->umma_rbox)) return CDGRAB_ERR_CUDA;
+    h->tm_r = h->tm_r32;               // unused by the kernel in this mode; any valid map will do
+    h->tm_r2 = h->tm_r32;
+  } else {
+    if (cudaMemset(h->r_split, 0, sizeof(__nv_bfloat16) * 3 * (size_t)h->d_pad) != cudaSuccess) return CDGRAB_ERR_CUDA;
+    if (!encode_map_3d(&h->tm_r, h->r_split, nblk_full, 3, h->d_pad, h->umma_paired ? subs / 2 : subs))
+      return CDGRAB_ERR_CUDA;
+    if (!encode_map_2d(&h->tm_r2, h->r_split, h->d, 3, h->d_pad)) return CDGRAB_ERR_CUDA;
+    h->tm_r32 = h->tm_r;               // unused by the kernel in this mode
+  }
   if (cdg_open_smem_limit(gram_umma_kernel) !=
       cudaSuccess) {
     cudaGetLastError();
@@ -605,10 +730,12 @@ cudaError_t cdg_launch_gram_umma(cdgrab_ctx *h, const void *grads, cudaStream_t 
   p.drain = h->umma_drain;
   p.g4 = h->umma_g4;
   p.paired = h->umma_paired;
+  p.rconv = h->umma_rconv;
+  p.rbox = h->umma_rbox;
   {
     CdgProfScope ps(h, CDGRAB_K_GRAM, st);
     cdg_launch_dep(h, gram_umma_kernel, dim3(h->umma_ctas), dim3(kThreads), h->umma_smem, st, mp[0], h->tm_r,
-                   mp[1], h->tm_r2, mp[2], p, h->umma_partials, h->status);
+                   mp[1], h->tm_r2, mp[2], h->tm_r32, p, h->umma_partials, h->status);
   }
   {
     CdgProfScope ps(h, CDGRAB_K_COMBINE, st);
