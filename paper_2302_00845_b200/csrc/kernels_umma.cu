@@ -115,10 +115,13 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
   // A = groups 0..15 (M = 128), B = all 20 (N = 160).  D rows 0..63 x columns 0..63 and 128..143
   // hold block j's products, rows 64..127 x columns 64..127 and 144..159 block j''s; the other
   // entries are cross terms nobody reads.
+  // When the r rows are written by the converter warp (rconv), both blocks' rows share group 16
+  // (rows 0..2 r of j, rows 3..5 r of j') and group 17 is the zero padding: 18 groups, N = 144,
+  // block j's b in columns 128..130 of rows 0..63 and block j''s in columns 131..133 of rows 64..127.
   const int paired = p.paired;
   const int hb = p.subs >> 1;                                    // blocks per half stage (paired)
   const uint32_t group_bytes = (uint32_t)(paired ? hb : p.subs) * 1024u;   // one row group of a stage
-  const int ngroups = paired ? 20 : (p.ncols >> 3);
+  const int ngroups = paired ? (p.rconv ? 18 : 20) : (p.ncols >> 3);
   const int ggroups = p.box_rows >> 3;                           // gradient row groups
   const uint32_t stage_bytes = group_bytes * ngroups;
   // rconv: the fp32 pieces of r (256 bytes per block, subs blocks per stage) lie behind the
@@ -262,7 +265,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
     // tcgen05.mma computed under a lane test would have to be moved into uniform registers one
     // by one (84 cycles per MMA were measured that way), operands of converged code start there.
     // kind::f16, D = f32, A = B = bf16, both K-major, M = 128, N = ncols
-    const uint32_t mma_n = paired ? 160u : (uint32_t)p.ncols;
+    const uint32_t mma_n = paired ? (rconv ? 144u : 160u) : (uint32_t)p.ncols;
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((mma_n >> 3) << 17) | ((128u >> 4) << 24);
     // The fp32 accumulation inside the tensor core truncates; over hundreds of thousands of
     // columns that becomes a visible bias on sums of same-sign products.  So the sum is kept
@@ -308,8 +311,9 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
     if (!ok && lane == 0) atomicOr(status, CDG_ST_TIMEOUT);
   } else if (warp == 6) {
     // ---------------- converter of r: fp32 piece -> three bf16 rows hi + mid + lo = r ----------------
-    // Written where the TMA would have put them: row t of the 8-row r group of block q, 16-byte
-    // chunk (c / 8) ^ t of its 128-byte row (the 128-byte swizzle; rows 3..7 stay zero).  Same
+    // Written in the layout a TMA copy would have produced: row t (paired, second block: 3 + t)
+    // of the 8-row r group of block q, 16-byte chunk (c / 8) ^ row of its 128-byte row (the
+    // 128-byte swizzle; the other rows stay zero).  Same
     // three roundings as everywhere else r is split, so the products come out bit for bit alike.
     if (rconv) {
       const int nb = paired ? hb : p.subs;
@@ -322,7 +326,8 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
         if (!ok) break;
         for (int hf = 0; hf < (paired ? 2 : 1); ++hf) {
           const float *src = reinterpret_cast<const float *>(smem_tiles + r32_off + (size_t)(s * p.subs + hf * nb) * 256);
-          uint8_t *rg = smem_tiles + (size_t)s * stage_bytes + (size_t)((paired ? 16 : ggroups) + hf * 2) * group_bytes;
+          uint8_t *rg = smem_tiles + (size_t)s * stage_bytes + (size_t)(paired ? 16 : ggroups) * group_bytes;
+          const int r0 = 3 * hf;                     // paired: the second block's rows follow the first's
           for (int idx = lane * 8; idx < nb * kSubCols; idx += 256) {
             const int q = idx >> 6, chunk = (idx & 63) >> 3;
             const float4 f0 = *reinterpret_cast<const float4 *>(src + idx);
@@ -345,9 +350,9 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
               lo[j] = (uint32_t)__bfloat16_as_ushort(l2[0]) | ((uint32_t)__bfloat16_as_ushort(l2[1]) << 16);
             }
             uint8_t *blk = rg + (size_t)q * 1024;
-            *reinterpret_cast<uint4 *>(blk + 0 * 128 + ((chunk ^ 0) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4 *>(blk + 1 * 128 + ((chunk ^ 1) << 4)) = make_uint4(mid[0], mid[1], mid[2], mid[3]);
-            *reinterpret_cast<uint4 *>(blk + 2 * 128 + ((chunk ^ 2) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            *reinterpret_cast<uint4 *>(blk + (r0 + 0) * 128 + ((chunk ^ (r0 + 0)) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4 *>(blk + (r0 + 1) * 128 + ((chunk ^ (r0 + 1)) << 4)) = make_uint4(mid[0], mid[1], mid[2], mid[3]);
+            *reinterpret_cast<uint4 *>(blk + (r0 + 2) * 128 + ((chunk ^ (r0 + 2)) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
           }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads these bytes through the async proxy
@@ -376,7 +381,8 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
         if (piece * 16 < p.ncols) {
           uint32_t v[16];
           // paired: rows 0..63 own D columns 0..63 and 128..143, rows 64..127 own 64..127 and 144..159
-          const int src = paired ? (piece < 4 ? piece + 4 * (lg >> 1) : 8 + (lg >> 1)) : piece;
+          // (rconv: both halves' b columns lie in piece 8, the upper rows' three at offset 3)
+          const int src = paired ? (piece < 4 ? piece + 4 * (lg >> 1) : 8 + (rconv ? 0 : (lg >> 1))) : piece;
           const uint32_t taddr = tmem_acc + (uint32_t)buf * 256u + ((uint32_t)(lg * 32) << 16) + (uint32_t)(src * 16);
           asm volatile(
               "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -401,6 +407,10 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tm_g3, const __grid_constan
       // rows 0..63 through the (now idle) stage ring; only the four read-back warps take part
       float *xch = reinterpret_cast<float *>(smem_raw + (tiles - smem_u32(smem_raw)));
       if (lg >= 2) {
+        if (rconv) {       // the upper rows' b columns sit three to the right of the lower rows'
+#pragma unroll
+          for (int j = 64; j < 67; ++j) accr[j] = accr[j + 3];
+        }
 #pragma unroll
         for (int j = 0; j < 80; ++j) xch[(row & 63) * 81 + j] = accr[j];
       }
@@ -612,7 +622,7 @@ int cdg_umma_setup(cdgrab_ctx *h) {
   // 6-8 at m = 32); CDGRAB_UMMA_SUBS overrides
   int subs = 76 / (h->umma_ncols / 8);
   subs = subs < 2 ? 2 : (subs > 8 ? 8 : subs);
-  if (h->umma_paired) subs = 6;                  // three stages of 60 KB
+  if (h->umma_paired) subs = 6;                  // four stages of 54 KB (three of 60 KB with the r rows from HBM)
   if (const char *e = getenv("CDGRAB_UMMA_SUBS")) {
     const int v = atoi(e);
     if (v >= 1 && v <= (h->umma_paired ? 10 : 8)) subs = v;
@@ -626,10 +636,6 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     const int v = atoi(e);
     if (v >= 1 && v <= (1 << 20)) h->umma_drain = v;
   }
-  const size_t group_bytes = (size_t)(h->umma_paired ? subs / 2 : subs) * 1024;
-  const int ngroups = h->umma_paired ? 20 : h->umma_ncols / 8;
-  const size_t stage_bytes = group_bytes * ngroups;
-  const size_t slack = (ngroups < 16) ? (16 - ngroups) * group_bytes : 0;  // operand A spans 16 row groups
   // r reaches the MMA as three bf16 rows.  Default: pass 1 reads r itself (fp32, 4 bytes per
   // column) and one warp writes the rows in shared memory; CDGRAB_UMMA_RCONV=0: pass 2 keeps a
   // bf16 copy [3][d_pad] in HBM (6 bytes per column written, 6 read) and the TMA brings its rows.
@@ -641,6 +647,11 @@ int cdg_umma_setup(cdgrab_ctx *h) {
     while (nb % rbox) --rbox;
     h->umma_rbox = rbox;
   }
+  const size_t group_bytes = (size_t)(h->umma_paired ? subs / 2 : subs) * 1024;
+  // paired: 20 row groups per stage, 18 when the converter packs both blocks' r rows into one
+  const int ngroups = h->umma_paired ? (h->umma_rconv ? 18 : 20) : h->umma_ncols / 8;
+  const size_t stage_bytes = group_bytes * ngroups;
+  const size_t slack = (ngroups < 16) ? (16 - ngroups) * group_bytes : 0;  // operand A spans 16 row groups
   const size_t r32_stage = h->umma_rconv ? (size_t)subs * 256 : 0;         // fp32 r of a stage
   const size_t budget = 226 * 1024 - 1024 - slack;
   int stages = (int)(budget / (stage_bytes + r32_stage));
