@@ -46,13 +46,18 @@ __device__ __forceinline__ void ldr(const float *p, float (&v)[VEC]) {
   }
 }
 
-constexpr int kIndepUnroll = 4;   // column groups a thread has in flight
+// Column groups a thread has in flight: 4 for 16-byte groups of fp32 rows, 2 for bf16 rows read 8
+// columns at a time (their groups carry twice the columns, and with 4 of them the kernels need 128
+// registers: two blocks per SM; measured 8 % (m = 32, d = 13.5 M) to 22 % (m = 64, d = 31 M) slower).
+template <typename T, int VEC>
+struct IndepUnroll { static constexpr int value = (sizeof(T) == 2 && VEC == 8) ? 2 : 4; };
 
 // grid (chunks, m).  partials[(i * chunks + chunk) * 3 + {t, rr, cc}]
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
 indep_dot_kernel(const T *__restrict__ g, const float *__restrict__ r, int m, long long d,
                  double *__restrict__ partials) {
+  constexpr int kIndepUnroll = IndepUnroll<T, VEC>::value;
   cdg_grid_dep_wait();            // the sums were updated by the launch before this one
   const int i = blockIdx.y;
   const T *z1 = g + (size_t)i * (size_t)d, *z2 = g + ((size_t)m + i) * (size_t)d;
@@ -134,6 +139,7 @@ template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
 indep_update_kernel(const T *__restrict__ g, float *__restrict__ r, const int8_t *__restrict__ signs,
                     int sign_stride, int m, long long d) {
+  constexpr int kIndepUnroll = IndepUnroll<T, VEC>::value;
   cdg_grid_dep_wait();            // the signs come from the launch before this one
   const int i = blockIdx.y;
   const float s = (float)signs[(size_t)i * sign_stride];
